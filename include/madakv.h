@@ -1,0 +1,160 @@
+/*
+ * madakv.h — C ABI of the MadaKV prefill-to-decode KV-cache eviction pass for NVIDIA B200 (sm_100a).
+ *
+ * The pass follows arXiv 2506.15724 (MadaKV), Section 3:
+ *   stage 1  madakv_score        importance psi(i) of every cached key under the proxy-token window   (Eq. 7, scale of Eq. 5)
+ *   stage 2  madakv_allocate     modality preference w_v, w_t and per-head modality budgets            (Eq. 6, Eq. 8)
+ *   stage 3  madakv_allocate     sparsity counts k_v, k_t, layer compensation K^l and phi^{l+1}        (Eq. 9, Eq. 10, Eq. 11)
+ *   stage 4  madakv_select       per-head, per-modality eviction: keep the budgeted top-psi tokens     (Section 3.3, text after Eq. 8)
+ *            madakv_compact      gather the kept K/V rows into a ragged per-head cache
+ *   stage 5  madakv_decode_attn  cache append and decode attention over the ragged cache                (Eq. 4, Eq. 5)
+ *
+ * General rules for every entry point
+ *   - Every data pointer is a DEVICE pointer owned by the caller (the only host pointers are `cfg` and the
+ *     `size_t* / int32_t*` result arguments of madakv_workspace_bytes / madakv_poll_status). The library allocates no
+ *     device memory, keeps no state between calls other than what lives in the caller's buffers, and only
+ *     enqueues work on `stream`.
+ *   - Return value: MADAKV_OK or a host-detected error (null or misaligned pointer, bad shape, unsupported
+ *     dtype/head_dim, workspace or capacity too small). Host-detected errors are raised before any kernel launch.
+ *   - Conditions only the device can see (a ragged segment that would overflow its capacity, a bounded wait that
+ *     expired) set a status word at the head of the workspace; the offending write is skipped, never performed out
+ *     of bounds. madakv_poll_status reads that word (it is the only call that synchronises the stream).
+ *   - Layouts: the innermost dimension (head_dim) is contiguous; all other strides are passed in ELEMENTS through
+ *     madakv_strides. Every row (head_dim elements) must start on a 16-byte boundary.
+ *   - Notation: B sequences, L layers, H_q query heads, H_kv KV heads, g = H_q / H_kv, d = head_dim, n_max =
+ *     max_seq_len, w = window. A "unit" is one (sequence b, layer l, KV head h); its flat index is
+ *     u = (b * L + l) * H_kv + h. Modality index 0 = visual, 1 = text.
+ */
+#ifndef MADAKV_H_
+#define MADAKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum madakv_status {
+  MADAKV_OK = 0,
+  MADAKV_EINVAL = 1,       /* null pointer, bad struct_size, bad flag value                         */
+  MADAKV_ESHAPE = 2,       /* non-positive or inconsistent dimension, H_q not a multiple of H_kv     */
+  MADAKV_EALIGN = 3,       /* a pointer or stride breaks the 16-byte row alignment rule              */
+  MADAKV_EWORKSPACE = 4,   /* workspace smaller than madakv_workspace_bytes reports                   */
+  MADAKV_ECAPACITY = 5,    /* ragged cache capacity exceeded (host- or device-detected)              */
+  MADAKV_EUNSUPPORTED = 6, /* dtype / head_dim / window*g outside the supported set                  */
+  MADAKV_ECUDA = 7,        /* a CUDA runtime call failed (launch configuration, missing sm_100 device) */
+  MADAKV_ETIMEOUT = 8      /* device-detected: a bounded wait inside a kernel ran out                */
+} madakv_status;
+
+enum { MADAKV_F32 = 0, MADAKV_BF16 = 1 };
+
+/* Layer-compensation modes (Eq. 10-11). phi^l is a per-head token budget; H below means KV heads.
+ *   OFF      phi^l = phi^1 for every layer (ablation "without HCC", Table 3)
+ *   PAPER    phi^{l+1} = phi^l - K^l / (H * (L - l)); the factor H reconciles Eq. 8 (phi^l per head) with Eq. 10
+ *            (K^l summed over heads)
+ *   LITERAL  phi^{l+1} = phi^l - K^l / (L - l), Eq. 11 exactly as printed                                     */
+enum { MADAKV_HCC_OFF = 0, MADAKV_HCC_PAPER = 1, MADAKV_HCC_LITERAL = 2 };
+
+typedef struct madakv_config {
+  uint32_t struct_size;     /* sizeof(madakv_config), checked                                            */
+  int32_t dtype;            /* MADAKV_F32 or MADAKV_BF16: element type of q, K, V, the ragged cache, out   */
+  int32_t batch;            /* B                                                                          */
+  int32_t n_layers;         /* L                                                                          */
+  int32_t n_q_heads;        /* H_q                                                                        */
+  int32_t n_kv_heads;       /* H_kv, divides H_q                                                          */
+  int32_t head_dim;         /* d, 64 or 128                                                               */
+  int32_t max_seq_len;      /* n_max: row count of the token dimension of K, V, psi, mask                  */
+  int32_t window;           /* w = |P|, the proxy tokens are the last w prompt positions (Section 3.3)     */
+  int32_t causal;           /* 1: window query at position p sees keys 0..p; 0: every window query sees all */
+  int32_t mpa;              /* 1: Eq. 8 modality split; 0: one budget per head, modality ignored (Table 3) */
+  int32_t hcc_mode;         /* MADAKV_HCC_*                                                               */
+  int32_t max_new_tokens;   /* rows of headroom left after every ragged segment for Eq. 4 appends          */
+  float theta;              /* threshold of Eq. 9, 0 <= theta <= 1                                        */
+  float softmax_scale;      /* 0 means 1/sqrt(head_dim) (Eq. 5)                                           */
+} madakv_config;
+
+/* Strides in elements of a [B, L, H, tokens, d] tensor; d is contiguous. */
+typedef struct madakv_strides {
+  int64_t batch, layer, head, token;
+} madakv_strides;
+
+/* Bytes of caller-provided scratch every other call expects in `ws` (a device buffer, 256-byte aligned).
+ * The first 256 bytes hold the device status word and counters; the caller zeroes the buffer once after
+ * allocating it (cudaMemsetAsync) and may then reuse it across calls on one stream. Two calls that run
+ * concurrently on different streams need separate workspaces.                                             */
+int madakv_workspace_bytes(const madakv_config* cfg, size_t* bytes_out);
+
+/* Stage 1 (Eq. 7 with the softmax of Eq. 5). For unit (b,l,h) and key i < seq_len[b]:
+ *   psi[u][i] = sum over the g query heads of the KV group and over window rows r of
+ *               softmax_i( scale * q_win[b,l,hq,r,:] . k[b,l,h,i,:] )
+ * Window row r stands at absolute position seq_len[b] - w + r; rows with a negative position are skipped; with
+ * cfg->causal the row sees keys 0..position. psi[u][i] = 0 for i >= seq_len[b]. Accumulation is fp32.
+ *   q_win   [B, L, H_q, w, d]  dtype, strides sq
+ *   k       [B, L, H_kv, n_max, d] dtype, strides sk
+ *   seq_len [B] int32, 0 <= seq_len[b] <= n_max
+ *   lse     [B, L, H_q, w] fp32, natural-log sum-exp of every window row's scaled logits. The call computes
+ *           these values and stores them here when `lse` is non-null (may be null).
+ *   psi     [B, L, H_kv, n_max] fp32, contiguous, written in full
+ * Deterministic: a fixed reduction order, no floating-point atomics.                                       */
+int madakv_score(const madakv_config* cfg, const void* q_win, madakv_strides sq, const void* k, madakv_strides sk,
+                 const int32_t* seq_len, float* lse, float* psi, void* ws, size_t ws_bytes, void* stream);
+
+/* Stages 2-3 (Eq. 6, 8, 9, 10, 11). All sums of psi are taken exactly, in 2^-32 fixed point:
+ *   Q(x) = floor(x * 2^32) for x > 0, else 0;   W_m = sum_{i in X_m} Q(psi[u][i])                 (Eq. 6)
+ *   pref[u][m] = W_m / (W_v + W_t)  (0 if the denominator is 0)                                    (Eq. 8 ratio)
+ *   demand[u][m] = smallest c such that the c largest Q of modality m sum to >= theta * W_m,
+ *                  0 when theta * W_m = 0                                                          (Eq. 9)
+ *   per sequence, l = 1..L (fp64): Phi^l = clamp(floor(phi^l + 1/2), 1, n);
+ *                  K^l = sum_h (k_v + k_t) - H * phi^l;                                             (Eq. 10)
+ *                  phi^{l+1} per cfg->hcc_mode, clamped to [1, n];  phi^1 = budget[b]               (Eq. 11)
+ *   budgets[u][0] = floor(pref_v * Phi^l + 1/2), budgets[u][1] = Phi^l - budgets[u][0]; a modality with fewer
+ *                  tokens than its share passes the surplus to the other one (both capped by their token counts).
+ *                  With cfg->mpa = 0: budgets[u] = {0, min(Phi^l, n)}.
+ *   psi [B,L,H_kv,n_max] fp32; mask [B,n_max] uint8 (1 = visual token); seq_len [B]; budget [B] int32 >= 1
+ *   mass, pref [B,L,H_kv,2] fp64 (mass = W_m / 2^32); demand, budgets [B,L,H_kv,2] int32; phi [B,L] fp64      */
+int madakv_allocate(const madakv_config* cfg, const float* psi, const uint8_t* mask, const int32_t* seq_len,
+                    const int32_t* budget, double* mass, double* pref, int32_t* demand, double* phi, int32_t* budgets,
+                    void* ws, size_t ws_bytes, void* stream);
+
+/* Stage 4a (Section 3.3: modality-specific eviction for each head). For every unit keep, of each modality m,
+ * the budgets[u][m] tokens with the largest psi (equal psi: the lower position wins) and list the kept positions
+ * in ascending order:
+ *   kept_len[u] = budgets[u][0] + budgets[u][1]
+ *   seg_off[u]  = sum_{u' < u} (kept_len[u'] + cfg->max_new_tokens), seg_off has B*L*H_kv + 1 entries (rows)
+ *   kept_idx[seg_off[u] + j], j < kept_len[u]: the j-th kept position
+ * With cfg->mpa = 0 the mask is ignored and budgets[u][1] positions are kept. A segment that would end beyond
+ * `capacity` rows is not written and sets MADAKV_ECAPACITY in the status word.                             */
+int madakv_select(const madakv_config* cfg, const float* psi, const uint8_t* mask, const int32_t* seq_len,
+                  const int32_t* budgets, int32_t* kept_len, int64_t* seg_off, int32_t* kept_idx, int64_t capacity,
+                  void* ws, size_t ws_bytes, void* stream);
+
+/* Stage 4b: k_c[seg_off[u] + j, :] = k[b,l,h, kept_idx[seg_off[u] + j], :] and the same for v (bit copies).
+ *   k, v [B,L,H_kv,n_max,d] dtype with strides skv; k_c, v_c [capacity, d] dtype, contiguous.             */
+int madakv_compact(const madakv_config* cfg, const void* k, const void* v, madakv_strides skv, const int32_t* kept_idx,
+                   const int64_t* seg_off, const int32_t* kept_len, void* k_c, void* v_c, int64_t capacity,
+                   void* ws, size_t ws_bytes, void* stream);
+
+/* Stage 5 (Eq. 4-5). For every unit of layer `layer` (all layers when layer = -1):
+ *   if k_new is non-null: row kept_len[u] of the segment := k_new[b,l,h,:] / v_new[b,l,h,:], kept_len[u] += 1
+ *                         (a full segment is left unchanged and sets MADAKV_ECAPACITY)              (Eq. 4)
+ *   out[b,l,hq,:] = softmax( scale * q[b,l,hq,:] . K_seg^T ) V_seg for the g query heads of the group (Eq. 5)
+ *   q, out [B,L,H_q,d] dtype contiguous; k_new, v_new [B,L,H_kv,d] dtype contiguous or both null;
+ *   lse_out [B,L,H_q] fp32 or null. An empty segment gives out = 0, lse = -inf.
+ * Accumulation is fp32; out is rounded to dtype once.                                                     */
+int madakv_decode_attn(const madakv_config* cfg, int32_t layer, const void* q, const void* k_new, const void* v_new,
+                       void* k_c, void* v_c, const int64_t* seg_off, int32_t* kept_len, int64_t capacity, void* out,
+                       float* lse_out, void* ws, size_t ws_bytes, void* stream);
+
+/* Synchronises `stream`, copies the device status word (a madakv_status) to *status_out and clears it. */
+int madakv_poll_status(void* ws, void* stream, int32_t* status_out);
+
+const char* madakv_status_string(int status);
+
+/* Library version, bumped when the ABI changes. */
+int madakv_abi_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MADAKV_H_ */
