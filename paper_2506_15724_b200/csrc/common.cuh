@@ -1,0 +1,136 @@
+// Shared declarations of the MadaKV CUDA library (host-side validation helpers, workspace layout, small device helpers).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "madakv.h"
+
+namespace madakv {
+
+// ---------------------------------------------------------------------------------------------------------------
+// Workspace layout (device memory owned by the caller)
+//   [0, 256)                 header: int32 status, then counters used by persistent kernels
+//   [256, ..)                stage 4 scratch: visual-token count per sequence [B] int32
+//   [.., .. + score)         stage 1 scratch: log2-domain row log-sum-exp [units * g * w] fp32, then per-chunk partial
+//                            (max, sum) pairs [units * chunks * g * w] float2
+//   [.., .. + decode)        stage 5 scratch: split partials [B * L * H_q * splits * (d + 2)] fp32
+// Stages 2-3 keep their scratch in shared memory.
+// ---------------------------------------------------------------------------------------------------------------
+constexpr size_t kHeaderBytes = 256;
+constexpr int kScoreChunk = 1024;   // keys per (max, sum) partial of the generic scoring path
+constexpr int kDecodeChunk = 512;   // cache rows per split of decode attention
+
+struct WsHeader {
+  int32_t status;        // madakv_status set by device code
+  int32_t work_counter;  // dynamic work distribution of persistent kernels
+  int32_t reserved[62];
+};
+static_assert(sizeof(WsHeader) == kHeaderBytes, "header size");
+
+struct WsLayout {
+  size_t seq_nv_off, score_lse_off, score_part_off, decode_off, total;
+  int score_chunks, decode_splits;
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline WsLayout ws_layout(const madakv_config& c) {
+  WsLayout w;
+  const size_t units = (size_t)c.batch * c.n_layers * c.n_kv_heads;
+  const size_t rows = (size_t)(c.n_q_heads / c.n_kv_heads) * c.window;
+  w.score_chunks = (c.max_seq_len + kScoreChunk - 1) / kScoreChunk;
+  w.decode_splits = (c.max_seq_len + c.max_new_tokens + kDecodeChunk - 1) / kDecodeChunk;
+  size_t off = kHeaderBytes;
+  w.seq_nv_off = off;
+  off = align_up(off + (size_t)c.batch * sizeof(int32_t), 256);
+  w.score_lse_off = off;
+  off = align_up(off + units * rows * sizeof(float), 256);
+  w.score_part_off = off;
+  off = align_up(off + units * rows * (size_t)w.score_chunks * sizeof(float2), 256);
+  w.decode_off = off;
+  off = align_up(off + (size_t)c.batch * c.n_layers * c.n_q_heads * (size_t)w.decode_splits * (c.head_dim + 2) *
+                           sizeof(float), 256);
+  w.total = off;
+  return w;
+}
+
+// Host-side checks shared by all entry points. Returns MADAKV_OK or the first violated rule.
+inline int check_config(const madakv_config* c) {
+  if (!c) return MADAKV_EINVAL;
+  if (c->struct_size != sizeof(madakv_config)) return MADAKV_EINVAL;
+  if (c->dtype != MADAKV_F32 && c->dtype != MADAKV_BF16) return MADAKV_EUNSUPPORTED;
+  if (c->batch <= 0 || c->n_layers <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->max_seq_len <= 0 ||
+      c->window <= 0)
+    return MADAKV_ESHAPE;
+  if (c->n_q_heads % c->n_kv_heads) return MADAKV_ESHAPE;
+  if (c->head_dim != 64 && c->head_dim != 128) return MADAKV_EUNSUPPORTED;
+  if (c->window > 1024 || (int64_t)(c->n_q_heads / c->n_kv_heads) * c->window > 4096) return MADAKV_EUNSUPPORTED;
+  if (c->max_seq_len > (1 << 20)) return MADAKV_EUNSUPPORTED;
+  if (c->causal != 0 && c->causal != 1) return MADAKV_EINVAL;
+  if (c->mpa != 0 && c->mpa != 1) return MADAKV_EINVAL;
+  if (c->hcc_mode < MADAKV_HCC_OFF || c->hcc_mode > MADAKV_HCC_LITERAL) return MADAKV_EINVAL;
+  if (c->max_new_tokens < 0) return MADAKV_ESHAPE;
+  if (!(c->theta >= 0.0f && c->theta <= 1.0f)) return MADAKV_EINVAL;
+  if (!(c->softmax_scale >= 0.0f)) return MADAKV_EINVAL;
+  return MADAKV_OK;
+}
+
+inline int elem_bytes(const madakv_config& c) { return c.dtype == MADAKV_F32 ? 4 : 2; }
+inline bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+inline bool strides_ok(const madakv_config& c, const madakv_strides& s) {
+  const int64_t e = elem_bytes(c);
+  return s.token >= c.head_dim && (s.batch * e) % 16 == 0 && (s.layer * e) % 16 == 0 && (s.head * e) % 16 == 0 &&
+         (s.token * e) % 16 == 0 && s.batch >= 0 && s.layer >= 0 && s.head >= 0;
+}
+inline int check_ws(const madakv_config& c, const void* ws, size_t ws_bytes) {
+  if (!ws) return MADAKV_EINVAL;
+  if ((uintptr_t)ws & 255) return MADAKV_EALIGN;
+  if (ws_bytes < ws_layout(c).total) return MADAKV_EWORKSPACE;
+  return MADAKV_OK;
+}
+inline float scale_of(const madakv_config& c) {
+  return c.softmax_scale > 0.0f ? c.softmax_scale : 1.0f / sqrtf((float)c.head_dim);
+}
+inline int launch_status() { return cudaGetLastError() == cudaSuccess ? MADAKV_OK : MADAKV_ECUDA; }
+
+// ---------------------------------------------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ float ld_f32(const float* p) { return *p; }
+__device__ __forceinline__ float ld_f32(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+
+// Order-preserving integer image of a non-negative importance value; anything not > 0 (incl. NaN) maps to 0.
+__device__ __forceinline__ uint32_t psi_key(float x) { return x > 0.0f ? __float_as_uint(x) : 0u; }
+// floor(x * 2^32) of a key produced by psi_key.
+__device__ __forceinline__ unsigned long long psi_fix(uint32_t key) {
+  return key ? __float2ull_rz(__uint_as_float(key) * 4294967296.0f) : 0ull;
+}
+
+__device__ __forceinline__ void set_status(void* ws, int code) { atomicCAS((int*)ws, 0, code); }
+#endif
+
+// Stage launchers implemented in the .cu files (all return a madakv_status).
+int launch_score(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                 const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st);
+int launch_score_generic(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                         const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st);
+int launch_allocate(const madakv_config& c, const float* psi, const uint8_t* mask, const int32_t* seq_len,
+                    const int32_t* budget, double* mass, double* pref, int32_t* demand, double* phi, int32_t* budgets,
+                    void* ws, cudaStream_t st);
+int launch_select(const madakv_config& c, const float* psi, const uint8_t* mask, const int32_t* seq_len,
+                  const int32_t* budgets, int32_t* kept_len, int64_t* seg_off, int32_t* kept_idx, int64_t capacity,
+                  void* ws, cudaStream_t st);
+int launch_compact(const madakv_config& c, const void* k, const void* v, madakv_strides s, const int32_t* kept_idx,
+                   const int64_t* seg_off, const int32_t* kept_len, void* k_c, void* v_c, int64_t capacity, void* ws,
+                   cudaStream_t st);
+int launch_decode(const madakv_config& c, int layer, const void* q, const void* k_new, const void* v_new, void* k_c,
+                  void* v_c, const int64_t* seg_off, int32_t* kept_len, int64_t capacity, void* out, float* lse_out,
+                  void* ws, cudaStream_t st);
+
+}  // namespace madakv

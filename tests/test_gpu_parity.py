@@ -1,0 +1,257 @@
+"""GPU parity: every stage of the CUDA library against the CPU oracle, element by element, through the C ABI.
+
+Staged tests feed each CUDA stage the ORACLE's output of the stage before, so integer results must be bit-exact.
+End-to-end tests run the CUDA pipeline on its own outputs and re-run each oracle stage on what the CUDA stage before
+it produced; scores are compared within the stated tolerance, everything downstream exactly.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_15724_b200 import binding as mk
+from paper_2506_15724_b200 import synth
+from helpers import (assert_segments_equal, capacity_of, config_of, dcode, oracle_stages_from, psi_close, to_np)
+
+pytestmark = pytest.mark.gpu
+
+PSI_RTOL = 1e-3      # the stated bar for scores and preferences (fp32 accumulation)
+PSI_RTOL_SEEN = 2e-5  # what this implementation is expected to reach; a regression beyond it fails too
+DEC_ATOL = {"bf16": 2e-2, "f32": 2e-5}
+
+TINY = synth.CONFIGS["tiny"]
+SHAPES = {
+    "tiny": TINY,
+    "tiny_gqa_ragged": synth.scaled(TINY, B=3, L=2, Hq=6, Hkv=2, n=389, w=5, budget=60, theta=0.3),
+    "bf16_d128": synth.scaled(TINY, dtype="bf16", L=3, Hq=4, Hkv=4, d=128, n=1100, w=32, budget=200, theta=0.3,
+                              n_needles=8),
+    "bf16_gqa7": synth.scaled(TINY, dtype="bf16", L=2, Hq=14, Hkv=2, d=128, n=700, w=32, budget=150, theta=0.3),
+    "bf16_d64_long_window": synth.scaled(TINY, dtype="bf16", L=1, Hq=8, Hkv=2, d=64, n=2500, w=64, budget=300,
+                                         theta=0.2),
+    "f32_d128": synth.scaled(TINY, L=2, Hq=2, Hkv=1, d=128, n=450, w=8, budget=100),
+}
+
+
+def make_case(wl, ragged=True):
+    inp = synth.make_inputs(wl, device="cpu")
+    if ragged and wl.B > 1:  # shorten all but the first sequence; the tail of the window must stay text
+        sl = inp["seq_len"].clone()
+        for b in range(1, wl.B):
+            sl[b] = max(wl.w // 2, wl.n - 97 * b - 1)
+        inp["seq_len"] = sl
+    return inp
+
+
+def dev(inp):
+    return {k: (v.cuda() if isinstance(v, torch.Tensor) else v) for k, v in inp.items()}
+
+
+@pytest.mark.parametrize("name", list(SHAPES))
+@pytest.mark.parametrize("causal", [1, 0])
+def test_score_matches_oracle(name, causal):
+    wl = SHAPES[name]
+    inp = make_case(wl)
+    cfg = config_of(wl, causal=causal)
+    g = dev(inp)
+    buf = mk.EvictionBuffers(cfg, capacity_of(wl), want_lse=True)
+    buf.psi.fill_(7.0)  # the call must overwrite every element, padding included
+    mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], buf.lse, buf.psi, buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    want, want_lse = oracle.score(dcode(wl), to_np(inp["q_win"]), to_np(inp["k"]), to_np(inp["seq_len"]),
+                                  causal=causal, want_lse=True)
+    got = buf.psi.cpu().numpy()
+    worst = psi_close(got, want, PSI_RTOL)
+    assert worst < PSI_RTOL_SEEN, worst
+    for b in range(wl.B):
+        assert (got[b, :, :, int(inp["seq_len"][b]):] == 0).all()
+    lse = buf.lse.cpu().numpy().astype(np.float64)
+    fin = np.isfinite(want_lse)
+    assert (np.isneginf(lse) == ~fin).all()
+    np.testing.assert_allclose(lse[fin], want_lse[fin], rtol=0, atol=2e-5)
+    # run to run bit-identical (fixed reduction order)
+    again = torch.empty_like(buf.psi)
+    mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], None, again, buf.ws)
+    assert torch.equal(again, buf.psi)
+
+
+@pytest.mark.parametrize("name", list(SHAPES))
+@pytest.mark.parametrize("mpa,hcc", [(1, mk.HCC_PAPER), (1, mk.HCC_LITERAL), (0, mk.HCC_OFF), (0, mk.HCC_PAPER)])
+def test_staged_allocate_select_compact_are_bit_exact(name, mpa, hcc):
+    wl = SHAPES[name]
+    inp = make_case(wl)
+    cfg = config_of(wl, mpa=mpa, hcc_mode=hcc)
+    mask, sl, bud = to_np(inp["mask"]), to_np(inp["seq_len"]), to_np(inp["budget"])
+    psi32 = oracle.score(dcode(wl), to_np(inp["q_win"]), to_np(inp["k"]), sl).astype(np.float32)
+    ref = oracle_stages_from(wl, cfg, psi32, mask, sl, bud, to_np(inp["k"]), to_np(inp["v"]))
+    g = dev(inp)
+    buf = mk.EvictionBuffers(cfg, ref["capacity"])
+    buf.psi.copy_(torch.from_numpy(psi32))
+    mk.madakv_allocate(cfg, buf.psi, g["mask"], g["seq_len"], g["budget"], buf.mass, buf.pref, buf.demand, buf.phi,
+                       buf.budgets, buf.ws)
+    for key in ("mass", "pref", "demand", "phi", "budgets"):
+        assert np.array_equal(getattr(buf, key).cpu().numpy(), ref[key]), key
+    # stage 4a on the oracle's budgets
+    buf.budgets.copy_(torch.from_numpy(ref["budgets"]))
+    mk.madakv_select(cfg, buf.psi, g["mask"], g["seq_len"], buf.budgets, buf.kept_len, buf.seg_off, buf.kept_idx,
+                     buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    assert np.array_equal(buf.kept_len.cpu().numpy(), ref["kept_len"])
+    assert np.array_equal(buf.seg_off.cpu().numpy(), ref["seg_off"])
+    assert_segments_equal(ref["kept_len"], ref["seg_off"], buf.kept_idx.cpu().numpy(), ref["kept_idx"], "kept_idx")
+    # stage 4b on the oracle's indices
+    buf.kept_idx.copy_(torch.from_numpy(ref["kept_idx"]))
+    mk.madakv_compact(cfg, g["k"], g["v"], buf.kept_idx, buf.seg_off, buf.kept_len, buf.k_c, buf.v_c, buf.ws)
+    assert_segments_equal(ref["kept_len"], ref["seg_off"], to_np(buf.k_c), ref["k_c"], "k_c")
+    assert_segments_equal(ref["kept_len"], ref["seg_off"], to_np(buf.v_c), ref["v_c"], "v_c")
+
+
+@pytest.mark.parametrize("name", list(SHAPES))
+def test_end_to_end_pass_and_decode(name):
+    wl = SHAPES[name]
+    inp = make_case(wl)
+    cfg = config_of(wl)
+    g = dev(inp)
+    buf = mk.EvictionBuffers(cfg, capacity_of(wl))
+    buf.run_eviction(g["q_win"], g["k"], g["v"], g["mask"], g["seq_len"], g["budget"])
+    assert mk.madakv_poll_status(buf.ws) == 0
+    mask, sl, bud = to_np(inp["mask"]), to_np(inp["seq_len"]), to_np(inp["budget"])
+    # scores against the oracle within tolerance
+    want_psi = oracle.score(dcode(wl), to_np(inp["q_win"]), to_np(inp["k"]), sl)
+    psi_gpu = buf.psi.cpu().numpy()
+    psi_close(psi_gpu, want_psi, PSI_RTOL)
+    # every later stage: the oracle re-run on the CUDA path's own scores must agree exactly
+    ref = oracle_stages_from(wl, cfg, psi_gpu, mask, sl, bud, to_np(inp["k"]), to_np(inp["v"]))
+    for key in ("mass", "pref", "demand", "phi", "budgets", "kept_len", "seg_off"):
+        assert np.array_equal(getattr(buf, key).cpu().numpy(), ref[key]), key
+    np.testing.assert_allclose(buf.pref.cpu().numpy().sum(-1), 1.0, rtol=1e-12)
+    assert_segments_equal(ref["kept_len"], ref["seg_off"], buf.kept_idx.cpu().numpy(), ref["kept_idx"], "kept_idx")
+    assert_segments_equal(ref["kept_len"], ref["seg_off"], to_np(buf.k_c), ref["k_c"], "k_c")
+    assert_segments_equal(ref["kept_len"], ref["seg_off"], to_np(buf.v_c), ref["v_c"], "v_c")
+    # pure-oracle pipeline: identical kept sets except at ties within 1e-5 relative of the k-th score
+    pure = oracle_stages_from(wl, cfg, want_psi.astype(np.float32), mask, sl, bud, to_np(inp["k"]), to_np(inp["v"]))
+    if np.array_equal(pure["budgets"], ref["budgets"]):
+        psi_u = want_psi.reshape(wl.units, wl.n)
+        for u in range(wl.units):
+            a = set(pure["kept_idx"][pure["seg_off"][u]: pure["seg_off"][u] + pure["kept_len"][u]].tolist())
+            b = set(ref["kept_idx"][ref["seg_off"][u]: ref["seg_off"][u] + ref["kept_len"][u]].tolist())
+            for i in a ^ b:
+                m = mask[u // (wl.L * wl.Hkv), i]
+                kept_m = [j for j in a if mask[u // (wl.L * wl.Hkv), j] == m]
+                kth = min(psi_u[u, j] for j in kept_m)
+                assert abs(psi_u[u, i] - kth) <= 1e-5 * kth, (u, i)
+    # decode: three steps with append, against the oracle on the same ragged cache
+    k_c, v_c, kept_len = ref["k_c"].copy(), ref["v_c"].copy(), ref["kept_len"].copy()
+    for step in range(3):
+        q, kn, vn = synth.make_decode_step(wl, step)
+        rc, want, want_lse = oracle.decode(dcode(wl), to_np(q), to_np(kn), to_np(vn), k_c, v_c, ref["seg_off"],
+                                           kept_len, Hkv=wl.Hkv)
+        assert rc == 0
+        buf.run_decode(q.cuda(), kn.cuda(), vn.cuda())
+        assert mk.madakv_poll_status(buf.ws) == 0
+        assert np.array_equal(buf.kept_len.cpu().numpy(), kept_len)
+        got = buf.out.float().cpu().numpy()
+        assert np.abs(got - want).max() <= DEC_ATOL[wl.dtype], np.abs(got - want).max()
+        np.testing.assert_allclose(buf.lse_dec.cpu().numpy(), want_lse, rtol=0, atol=1e-4)
+    assert_segments_equal(kept_len, ref["seg_off"], to_np(buf.k_c), k_c, "k_c after append")
+    # one layer only: other layers' outputs stay untouched
+    if wl.L > 1:
+        q, _, _ = synth.make_decode_step(wl, 9)
+        before = buf.out.clone()
+        buf.run_decode(q.cuda(), layer=1)
+        rc, want, _ = oracle.decode(dcode(wl), to_np(q), None, None, k_c, v_c, ref["seg_off"], kept_len, Hkv=wl.Hkv,
+                                    layer=1)
+        got = buf.out.float().cpu().numpy()
+        assert np.abs(got[:, 1] - want[:, 1]).max() <= DEC_ATOL[wl.dtype]
+        assert torch.equal(buf.out[:, 0], before[:, 0])
+
+
+def test_edge_cases_budget_extremes_and_single_modality():
+    wl = synth.scaled(TINY, L=2, n=330, w=8)
+    inp = make_case(wl)
+    g = dev(inp)
+    mask, sl = to_np(inp["mask"]), to_np(inp["seq_len"])
+    for budget, theta, flip in ((1, 0.5, None), (10_000, 1.0, None), (40, 0.0, None), (40, 0.5, 0), (40, 0.5, 1)):
+        cfg = config_of(wl, theta=theta)
+        m = mask if flip is None else np.full_like(mask, flip)
+        bud = np.array([budget], np.int32)
+        buf = mk.EvictionBuffers(cfg, capacity_of(wl))
+        buf.run_eviction(g["q_win"], g["k"], g["v"], torch.from_numpy(m).cuda(), g["seq_len"],
+                         torch.from_numpy(bud).cuda())
+        assert mk.madakv_poll_status(buf.ws) == 0
+        ref = oracle_stages_from(wl, cfg, buf.psi.cpu().numpy(), m, sl, bud, to_np(inp["k"]), to_np(inp["v"]))
+        for key in ("demand", "phi", "budgets", "kept_len", "seg_off"):
+            assert np.array_equal(getattr(buf, key).cpu().numpy(), ref[key]), (key, budget, theta, flip)
+        assert_segments_equal(ref["kept_len"], ref["seg_off"], buf.kept_idx.cpu().numpy(), ref["kept_idx"], "kept_idx")
+        if budget >= wl.n:
+            assert (ref["kept_len"] == wl.n).all()
+
+
+def test_short_sequences_and_empty_sequence():
+    wl = synth.scaled(TINY, B=4, L=1, n=320 + 8, w=8, budget=16)
+    inp = synth.make_inputs(wl)
+    inp["seq_len"] = torch.tensor([wl.n, 3, 0, 8], dtype=torch.int32)  # shorter than the window, empty, == window
+    cfg = config_of(wl)
+    g = dev(inp)
+    buf = mk.EvictionBuffers(cfg, capacity_of(wl))
+    buf.run_eviction(g["q_win"], g["k"], g["v"], g["mask"], g["seq_len"], g["budget"])
+    assert mk.madakv_poll_status(buf.ws) == 0
+    sl = to_np(inp["seq_len"])
+    want_psi = oracle.score(0, to_np(inp["q_win"]), to_np(inp["k"]), sl)
+    psi_close(buf.psi.cpu().numpy(), want_psi, PSI_RTOL)
+    ref = oracle_stages_from(wl, cfg, buf.psi.cpu().numpy(), to_np(inp["mask"]), sl, to_np(inp["budget"]),
+                             to_np(inp["k"]), to_np(inp["v"]))
+    for key in ("demand", "phi", "budgets", "kept_len", "seg_off"):
+        assert np.array_equal(getattr(buf, key).cpu().numpy(), ref[key]), key
+    q, _, _ = synth.make_decode_step(wl, 0)
+    buf.run_decode(q.cuda())
+    kept_len = ref["kept_len"].copy()
+    rc, want, want_lse = oracle.decode(0, to_np(q), None, None, ref["k_c"], ref["v_c"], ref["seg_off"], kept_len,
+                                       Hkv=wl.Hkv)
+    assert np.abs(buf.out.cpu().numpy() - want).max() <= 2e-5
+    got_lse = buf.lse_dec.cpu().numpy()
+    assert (np.isneginf(got_lse) == np.isneginf(want_lse)).all()
+    assert (buf.out[2] == 0).all()  # empty sequence: zeros
+
+
+def test_capacity_overflow_is_reported_not_written():
+    wl = synth.scaled(TINY, L=1, max_new_tokens=1)
+    inp = make_case(wl)
+    cfg = config_of(wl)
+    g = dev(inp)
+    small = 100  # rows: far below 4 units x 129
+    buf = mk.EvictionBuffers(cfg, small)
+    guard = torch.full((small + 64,), -7, dtype=torch.int32, device="cuda")
+    buf.kept_idx = guard[:small]
+    buf.run_eviction(g["q_win"], g["k"], g["v"], g["mask"], g["seq_len"], g["budget"])
+    assert mk.madakv_poll_status(buf.ws) == mk.ECAPACITY
+    assert mk.madakv_poll_status(buf.ws) == 0  # cleared by the poll
+    assert (guard[small:] == -7).all()
+    # appending beyond the headroom: first append fits, second is refused and leaves the cache unchanged
+    buf = mk.EvictionBuffers(cfg, capacity_of(wl))
+    buf.run_eviction(g["q_win"], g["k"], g["v"], g["mask"], g["seq_len"], g["budget"])
+    q, kn, vn = [t.cuda() for t in synth.make_decode_step(wl, 0)]
+    buf.run_decode(q, kn, vn)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    lens, kc = buf.kept_len.clone(), buf.k_c.clone()
+    buf.run_decode(q, kn, vn)
+    assert mk.madakv_poll_status(buf.ws) == mk.ECAPACITY
+    assert torch.equal(buf.kept_len, lens) and torch.equal(buf.k_c, kc)
+
+
+def test_strided_kv_layout():
+    # K/V stored per layer as [B, H, n, d] inside a larger allocation (token stride > d)
+    wl = synth.scaled(TINY, dtype="bf16", L=2, Hq=4, Hkv=2, d=128, n=340, w=8, budget=50)
+    inp = make_case(wl)
+    cfg = config_of(wl)
+    g = dev(inp)
+    big_k = torch.zeros((wl.L, wl.B, wl.Hkv, wl.n, wl.d + 64), dtype=torch.bfloat16, device="cuda")
+    big_v = torch.zeros_like(big_k)
+    big_k[..., : wl.d] = g["k"].permute(1, 0, 2, 3, 4)
+    big_v[..., : wl.d] = g["v"].permute(1, 0, 2, 3, 4)
+    kv, vv = big_k[..., : wl.d].permute(1, 0, 2, 3, 4), big_v[..., : wl.d].permute(1, 0, 2, 3, 4)
+    a = mk.EvictionBuffers(cfg, capacity_of(wl))
+    a.run_eviction(g["q_win"], g["k"], g["v"], g["mask"], g["seq_len"], g["budget"])
+    b = mk.EvictionBuffers(cfg, capacity_of(wl))
+    b.run_eviction(g["q_win"], kv, vv, g["mask"], g["seq_len"], g["budget"])
+    assert torch.equal(a.psi, b.psi) and torch.equal(a.kept_idx, b.kept_idx)
+    assert torch.equal(a.k_c, b.k_c) and torch.equal(a.v_c, b.v_c)
