@@ -28,7 +28,7 @@ def build(force=False, verbose=False):
         "nvcc", "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
         "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", os.path.join(HERE, "csrc"),
         "-o", LIB,
-    ] + (["-Xptxas", "-v"] if verbose else []) + sources() + ["-lcuda"]
+    ] + (["-Xptxas", "-v"] if verbose else []) + sources()
     subprocess.check_call(cmd)
     return LIB
 

@@ -13,13 +13,14 @@ namespace madakv {
 // Workspace layout (device memory owned by the caller)
 //   [0, 256)                 header: int32 status, then counters used by persistent kernels
 //   [256, ..)                stage 4 scratch: visual-token count per sequence [B] int32
-//   [.., .. + score)         stage 1 scratch: log2-domain row log-sum-exp [units * g * w] fp32, then per-chunk partial
-//                            (max, sum) pairs [units * chunks * g * w] float2
+//   [.., .. + score)         stage 1 scratch: finished-item counters [units] int32, log2-domain row log-sum-exp
+//                            [units * g * w] fp32, per-chunk partial (max, sum) pairs [units * chunks * rows] float2
 //   [.., .. + decode)        stage 5 scratch: split partials [B * L * H_q * splits * (d + 2)] fp32
 // Stages 2-3 keep their scratch in shared memory.
 // ---------------------------------------------------------------------------------------------------------------
 constexpr size_t kHeaderBytes = 256;
 constexpr int kScoreChunk = 1024;   // keys per (max, sum) partial of the generic scoring path
+constexpr int kScoreTcChunk = 512;  // keys per work item (and per partial) of the tensor-core scoring path
 constexpr int kDecodeChunk = 512;   // cache rows per split of decode attention
 
 struct WsHeader {
@@ -30,8 +31,8 @@ struct WsHeader {
 static_assert(sizeof(WsHeader) == kHeaderBytes, "header size");
 
 struct WsLayout {
-  size_t seq_nv_off, score_lse_off, score_part_off, decode_off, total;
-  int score_chunks, decode_splits;
+  size_t seq_nv_off, score_done_off, score_lse_off, score_part_off, decode_off, total;
+  int score_chunks, score_tc_chunks, decode_splits;
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -45,10 +46,14 @@ inline WsLayout ws_layout(const madakv_config& c) {
   size_t off = kHeaderBytes;
   w.seq_nv_off = off;
   off = align_up(off + (size_t)c.batch * sizeof(int32_t), 256);
+  w.score_done_off = off;
+  off = align_up(off + units * sizeof(int32_t), 256);
   w.score_lse_off = off;
   off = align_up(off + units * rows * sizeof(float), 256);
   w.score_part_off = off;
-  off = align_up(off + units * rows * (size_t)w.score_chunks * sizeof(float2), 256);
+  w.score_tc_chunks = (c.max_seq_len + kScoreTcChunk - 1) / kScoreTcChunk;
+  const size_t rows_pad = (rows + 31) / 32 * 32;  // the tensor-core path pads the row count
+  off = align_up(off + units * rows_pad * (size_t)w.score_tc_chunks * sizeof(float2), 256);
   w.decode_off = off;
   off = align_up(off + (size_t)c.batch * c.n_layers * c.n_q_heads * (size_t)w.decode_splits * (c.head_dim + 2) *
                            sizeof(float), 256);
@@ -118,6 +123,9 @@ __device__ __forceinline__ void set_status(void* ws, int code) { atomicCAS((int*
 // Stage launchers implemented in the .cu files (all return a madakv_status).
 int launch_score(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
                  const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st);
+bool score_tc_supported(const madakv_config& c, madakv_strides sq, madakv_strides sk);
+int launch_score_tc(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                    const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st);
 int launch_score_generic(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
                          const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st);
 int launch_allocate(const madakv_config& c, const float* psi, const uint8_t* mask, const int32_t* seq_len,

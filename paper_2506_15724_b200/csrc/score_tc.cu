@@ -1,0 +1,695 @@
+// Stage 1, Blackwell tensor-core path (Eq. 7 with the softmax of Eq. 5) for bf16 inputs with g * w <= 64 window rows.
+//
+// One persistent kernel streams every K tile exactly once from HBM and a second time from L2:
+//   - the window-QK^T tile is a tcgen05.mma with the 128 keys of a tile on M, the g*w window rows on N and head_dim
+//     on K; operands are staged in shared memory by TMA (128-byte swizzle), the fp32 accumulator lives in TMEM;
+//   - a softmax over keys needs every row's log-sum-exp before any normalised weight can be summed over rows, so
+//     the work is cut into items of kItemTiles tiles in two phases: phase-1 items produce per-row (max, sum exp2)
+//     partials, phase-2 items recompute the logits and emit psi. The item list interleaves phase 2 of chunk t with
+//     phase 1 of chunk t + lag, so the second read of a K chunk comes a bounded number of chunks after the first
+//     and is served by the L2 (phase-1 loads ask L2 to keep the lines, phase-2 loads to drop them);
+//   - a phase-2 item waits (bounded) until all phase-1 items of its unit have published their partials. Every item
+//     only depends on items earlier in the global order and every CTA walks its items in that order, so with all
+//     CTAs resident (grid <= SM count, one CTA per SM) the waits always end.
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-5 epilogue (one TMEM lane quarter each;
+// a thread owns one key of the tile and all window rows of it, so psi(i) is an in-thread sum over N).
+// Every wait is bounded: on expiry the kernel records MADAKV_ETIMEOUT, lets its copies drain, frees TMEM and returns.
+#include <cuda.h>
+#include <cstdlib>
+
+#include "common.cuh"
+
+namespace madakv {
+namespace {
+
+constexpr int kTileKeys = 128;
+constexpr int kItemTiles = 4;                       // tiles per work item
+constexpr int kItemKeys = kTileKeys * kItemTiles;   // == kScoreTcChunk
+constexpr int kStagesD128 = 5;
+constexpr int kTmemCols = 256;
+constexpr int kTmemBufCols = 64;
+constexpr int kTmemBufs = kTmemCols / kTmemBufCols;
+constexpr int kThreads = 192;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kEmptyMax = -1.0e30f;               // "no key seen yet" marker of a running maximum
+constexpr long long kWaitCycles = 4000000000ll;     // ~2 s at B200 clocks: bound of every device-side wait
+
+static_assert(kItemKeys == kScoreTcChunk, "partials are indexed by kScoreTcChunk keys");
+
+struct TcParams {
+  const int32_t* seq_len;
+  float* psi;        // [units, n_max]
+  float* lse_out;    // natural log [B,L,Hq,w] or null
+  float2* part;      // ws: [units, cpu, NPAD]
+  int32_t* done;     // ws: [units] phase-1 items finished
+  int32_t* status;   // ws header
+  int units, L, Hq, Hkv, g, w, R, n_max, cpu, causal, lag;
+  float scale2;
+};
+
+// ------------------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait. Returns false if the wait was abandoned (own timeout or another role's abort flag).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  int spins = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++spins & 63) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) {
+        *abort_flag = 1;
+        atomicCAS(status, 0, (int)MADAKV_ETIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+
+// 5-D tiled TMA load into this CTA's shared memory, completion signalled on an mbarrier.
+__device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2,
+                                            int c3, int c4, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(policy)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes packed densely
+// (8-row groups 1024 bytes apart), descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);  // start address
+  d |= (uint64_t)1 << 16;                    // leading byte offset (unused with swizzle), in 16-byte units
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset
+  d |= (uint64_t)1 << 46;                    // version
+  d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Barrier of the 128 epilogue threads on an mbarrier (count 128), so that it is bounded like every other wait.
+// The result is made uniform over the warp.
+__device__ __forceinline__ bool epi_sync(uint64_t* ebar, uint32_t& parity, volatile int* abort_flag, int32_t* status) {
+  mbar_arrive(ebar);
+  const bool ok = mbar_wait(ebar, parity, abort_flag, status);
+  parity ^= 1;
+  return __all_sync(0xffffffffu, ok);
+}
+
+// (max, sum) merge of two partial softmax statistics in the log2 domain.
+__device__ __forceinline__ void merge_stats(float& m, float& z, float mo, float zo) {
+  const float mn = fmaxf(m, mo);
+  z = z * ex2(m - mn) + zo * ex2(mo - mn);
+  m = mn;
+}
+
+// ------------------------------------------------------------------------------------------------ work list
+struct Item {
+  int phase;  // 1 or 2
+  int unit, chunk;
+};
+
+// The idx-th item of CTA `cta` (grid G): first its share of the phase-1 prologue (the first `lag` chunks), then its
+// super-items t = cta, cta + G, ...: phase 2 of chunk t followed by phase 1 of chunk t + lag.
+__device__ __forceinline__ bool get_item(int cta, int G, int idx, int total_chunks, int lag, int cpu, Item& it) {
+  const int pro = min(lag, total_chunks);
+  const int my_pro = cta < pro ? (pro - cta + G - 1) / G : 0;
+  int j, phase;
+  if (idx < my_pro) {
+    j = cta + idx * G;
+    phase = 1;
+  } else {
+    const int k = idx - my_pro;
+    // super-item slots: 2 per t while t + lag < total, then 1
+    const int two = max(total_chunks - lag, 0);               // t in [0, two) have both halves
+    const int my_two = cta < two ? (two - cta + G - 1) / G : 0;
+    if (k < 2 * my_two) {
+      const int t = cta + (k >> 1) * G;
+      if (k & 1) { j = t + lag; phase = 1; } else { j = t; phase = 2; }
+    } else {
+      const int k2 = k - 2 * my_two;
+      const int t = cta + (my_two + k2) * G;
+      if (t >= total_chunks) return false;
+      j = t;
+      phase = 2;
+    }
+  }
+  it.phase = phase;
+  it.unit = j / cpu;
+  it.chunk = j % cpu;
+  return true;
+}
+
+template <int D, int NPAD>
+struct SmemLayout {
+  static constexpr int kStages = D == 128 ? kStagesD128 : 2 * kStagesD128;
+  static constexpr int kKBlocks = D / 64;
+  static constexpr int kStageBytes = kTileKeys * D * 2;
+  static constexpr int kQBytes = NPAD * D * 2;
+  static constexpr int kKOff = 0;
+  static constexpr int kQOff = kStages * kStageBytes;
+  static constexpr int kBarOff = kQOff + 2 * kQBytes;
+  static constexpr int kNumBars = 2 * kStages + 4 + 2 * kTmemBufs + 1;
+  static constexpr int kMiscOff = kBarOff + kNumBars * 8;
+  // misc: tmem base (4), abort flag (4), lse2[NPAD], vis[NPAD], red[4][NPAD] float2
+  static constexpr int kLseOff = kMiscOff + 16;
+  static constexpr int kVisOff = kLseOff + NPAD * 4;
+  static constexpr int kRedOff = kVisOff + NPAD * 4;
+  static constexpr int kTotal = kRedOff + 4 * NPAD * 8;
+  static constexpr int kAlloc = kTotal + 1024;  // slack for the 1024-byte alignment of the operand tiles
+};
+
+template <int D, int NPAD>
+__global__ void __launch_bounds__(kThreads, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_q, TcParams p) {
+  using SL = SmemLayout<D, NPAD>;
+  constexpr int kStages = SL::kStages;
+  constexpr int kKBlocks = SL::kKBlocks;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* k_s = smem + SL::kKOff;
+  uint8_t* q_s = smem + SL::kQOff;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kBarOff);
+  uint64_t* full = bars;                       // [kStages]   TMA -> MMA
+  uint64_t* empty = bars + kStages;            // [kStages]   MMA -> TMA
+  uint64_t* qfull = bars + 2 * kStages;        // [2]
+  uint64_t* qempty = qfull + 2;                // [2]
+  uint64_t* tfull = qempty + 2;                // [kTmemBufs] MMA -> epilogue
+  uint64_t* tempty = tfull + kTmemBufs;        // [kTmemBufs] epilogue -> MMA
+  uint64_t* ebar = tempty + kTmemBufs;         // barrier of the epilogue threads
+  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(smem + SL::kMiscOff);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::kMiscOff + 4);
+  float* lse_s = reinterpret_cast<float*>(smem + SL::kLseOff);
+  int* vis_s = reinterpret_cast<int*>(smem + SL::kVisOff);
+  float2* red_s = reinterpret_cast<float2*>(smem + SL::kRedOff);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_chunks = p.units * p.cpu;
+
+  // ---- set-up
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&qfull[i], 1);
+      mbar_init(&qempty[i], 1);
+    }
+    for (int i = 0; i < kTmemBufs; ++i) {
+      mbar_init(&tfull[i], 1);
+      mbar_init(&tempty[i], 128);
+    }
+    mbar_init(ebar, 128);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // rows R..NPAD-1 of both Q buffers are never written by TMA: keep them zero so their logits are 0
+  for (int x = threadIdx.x; x < 2 * SL::kQBytes / 16; x += kThreads)
+    reinterpret_cast<uint4*>(q_s)[x] = make_uint4(0, 0, 0, 0);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_s)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_s;
+
+  if (warp == 0) {
+    // ================================================================ TMA producer
+    if (lane == 0) {
+      const uint64_t pol_keep = l2_policy_evict_last(), pol_drop = l2_policy_evict_first();
+      int stage = 0;
+      uint32_t stage_par = 0;
+      int qi = 0;
+      uint32_t q_par = 0;
+      bool ok = true;
+      Item it;
+      for (int idx = 0; ok && get_item(blockIdx.x, gridDim.x, idx, total_chunks, p.lag, p.cpu, it); ++idx) {
+        const int h = it.unit % p.Hkv, l = (it.unit / p.Hkv) % p.L, b = it.unit / (p.Hkv * p.L);
+        const int n = min(p.seq_len[b], p.n_max);
+        const int key_begin = it.chunk * kItemKeys;
+        if (key_begin >= n) continue;  // nothing to load for this item
+        // window queries of the unit
+        ok = mbar_wait(&qempty[qi], q_par ^ 1, abort_flag, p.status);
+        if (!ok) break;
+        mbar_expect_tx(&qfull[qi], (uint32_t)(p.R * 128 * kKBlocks));
+        for (int kb = 0; kb < kKBlocks; ++kb)
+          tma_load_5d(q_s + qi * SL::kQBytes + kb * NPAD * 128, &tmap_q, &qfull[qi], kb * 64, 0, h * p.g, l, b,
+                      pol_keep);
+        qi ^= 1;
+        if (qi == 0) q_par ^= 1;
+        const uint64_t pol = it.phase == 1 ? pol_keep : pol_drop;
+        for (int t = 0; t < kItemTiles; ++t) {
+          const int key0 = key_begin + t * kTileKeys;
+          if (key0 >= n) break;
+          ok = mbar_wait(&empty[stage], stage_par ^ 1, abort_flag, p.status);
+          if (!ok) break;
+          mbar_expect_tx(&full[stage], (uint32_t)SL::kStageBytes);
+          for (int kb = 0; kb < kKBlocks; ++kb)
+            tma_load_5d(k_s + stage * SL::kStageBytes + kb * kTileKeys * 128, &tmap_k, &full[stage], kb * 64, key0, h,
+                        l, b, pol);
+          if (++stage == kStages) {
+            stage = 0;
+            stage_par ^= 1;
+          }
+        }
+      }
+      if (!ok) {  // abandoned: give copies in flight time to land before the CTA's shared memory goes away
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    // ================================================================ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc_bf16(NPAD);
+      int stage = 0;
+      uint32_t stage_par = 0;
+      int qi = 0;
+      uint32_t q_par = 0;
+      int tb = 0;
+      uint32_t tb_par = 0;
+      bool ok = true;
+      Item it;
+      for (int idx = 0; ok && get_item(blockIdx.x, gridDim.x, idx, total_chunks, p.lag, p.cpu, it); ++idx) {
+        const int b = it.unit / (p.Hkv * p.L);
+        const int n = min(p.seq_len[b], p.n_max);
+        const int key_begin = it.chunk * kItemKeys;
+        if (key_begin >= n) continue;
+        ok = mbar_wait(&qfull[qi], q_par, abort_flag, p.status);
+        if (!ok) break;
+        const uint32_t q_addr = smem_u32(q_s + qi * SL::kQBytes);
+        for (int t = 0; t < kItemTiles; ++t) {
+          const int key0 = key_begin + t * kTileKeys;
+          if (key0 >= n) break;
+          ok = mbar_wait(&full[stage], stage_par, abort_flag, p.status) &&
+               mbar_wait(&tempty[tb], tb_par ^ 1, abort_flag, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t k_addr = smem_u32(k_s + stage * SL::kStageBytes);
+          const uint32_t d_tmem = tmem_base + tb * kTmemBufCols;
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const int kb = ks >> 2, kk = ks & 3;
+            const uint64_t a = smem_desc_sw128(k_addr + kb * kTileKeys * 128 + kk * 32);
+            const uint64_t bq = smem_desc_sw128(q_addr + kb * NPAD * 128 + kk * 32);
+            umma_bf16(d_tmem, a, bq, idesc, ks > 0 ? 1u : 0u);
+          }
+          umma_commit(&empty[stage]);  // the K stage may be refilled once these MMAs have read it
+          umma_commit(&tfull[tb]);     // the accumulator is complete
+          if (++stage == kStages) {
+            stage = 0;
+            stage_par ^= 1;
+          }
+          if (++tb == kTmemBufs) {
+            tb = 0;
+            tb_par ^= 1;
+          }
+        }
+        if (!ok) break;
+        umma_commit(&qempty[qi]);  // the Q buffer may be refilled once this item's MMAs are done
+        qi ^= 1;
+        if (qi == 0) q_par ^= 1;
+      }
+    }
+  } else {
+    // ================================================================ epilogue (128 threads, one key each)
+    const int quarter = warp & 3;                 // TMEM lanes [32 * quarter, 32 * quarter + 32)
+    const int et = (quarter << 5) | lane;         // key index inside the tile
+    const int ethread = threadIdx.x - 64;         // 0..127 in launch order (used for row-parallel steps)
+    int tb = 0;
+    uint32_t tb_par = 0, e_par = 0;
+    bool ok = true;
+    Item it;
+    for (int idx = 0; ok && get_item(blockIdx.x, gridDim.x, idx, total_chunks, p.lag, p.cpu, it); ++idx) {
+      const int h = it.unit % p.Hkv, bl = it.unit / p.Hkv, b = bl / p.L;
+      const int n = min(p.seq_len[b], p.n_max);
+      const int key_begin = it.chunk * kItemKeys;
+      float* psi = p.psi + (int64_t)it.unit * p.n_max;
+      if (key_begin >= n) {
+        if (it.phase == 2)  // beyond the sequence: psi = 0
+          for (int t = 0; t < kItemTiles; ++t) {
+            const int key = key_begin + t * kTileKeys + et;
+            if (key < p.n_max) psi[key] = 0.f;
+          }
+        continue;
+      }
+      // per-row visibility bound (exclusive key index) of this unit
+      ok = epi_sync(ebar, e_par, abort_flag, p.status);  // previous item's readers of the shared arrays are done
+      if (!ok) break;
+      if (ethread < NPAD) {
+        int vis = 0;
+        if (ethread < p.R) {
+          const int pos = n - p.w + ethread % p.w;
+          if (pos >= 0) vis = p.causal ? pos + 1 : n;
+        }
+        vis_s[ethread] = vis;
+      }
+      const int n_chunks_active = (n + kItemKeys - 1) / kItemKeys;
+      if (it.phase == 2) {
+        // wait until every phase-1 item of this unit has published its partials
+        if (ethread == 0) {
+          const long long t0 = clock64();
+          int spins = 0;
+          while (true) {
+            int v;
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p.done + it.unit) : "memory");
+            if (v >= n_chunks_active) break;
+            if (*abort_flag) break;
+            __nanosleep(64);
+            if ((++spins & 255) == 0 && clock64() - t0 > kWaitCycles) {
+              *abort_flag = 1;
+              atomicCAS(p.status, 0, (int)MADAKV_ETIMEOUT);
+              break;
+            }
+          }
+        }
+        ok = epi_sync(ebar, e_par, abort_flag, p.status);
+        ok = __all_sync(0xffffffffu, ok && !*abort_flag);
+        if (!ok) break;
+        if (ethread < NPAD) {
+          float M = kEmptyMax, Z = 0.f;
+          const float2* part = p.part + (int64_t)it.unit * p.cpu * NPAD + ethread;
+          for (int c = 0; c < n_chunks_active; ++c) {
+            const float2 pz = __ldcg(part + c * NPAD);
+            merge_stats(M, Z, pz.x, pz.y);
+          }
+          const float lse2 = (Z > 0.f) ? M + log2f(Z) : 0.f;
+          lse_s[ethread] = lse2;
+          if (p.lse_out && it.chunk == 0 && ethread < p.R) {
+            const int hq = h * p.g + ethread / p.w, wr = ethread % p.w;
+            p.lse_out[((int64_t)bl * p.Hq + hq) * p.w + wr] = (Z > 0.f) ? lse2 * 0.6931471805599453f : -INFINITY;
+          }
+        }
+      }
+      ok = epi_sync(ebar, e_par, abort_flag, p.status);
+      if (!ok) break;
+
+      float st_m[NPAD], st_z[NPAD];  // phase 1: this lane's running statistics per window row
+      if (it.phase == 1) {
+#pragma unroll
+        for (int c = 0; c < NPAD; ++c) {
+          st_m[c] = kEmptyMax;
+          st_z[c] = 0.f;
+        }
+      }
+      for (int t = 0; t < kItemTiles; ++t) {
+        const int key0 = key_begin + t * kTileKeys;
+        if (key0 >= n) {
+          if (it.phase == 2 && key0 + et < p.n_max) psi[key0 + et] = 0.f;
+          continue;
+        }
+        ok = __all_sync(0xffffffffu, mbar_wait(&tfull[tb], tb_par, abort_flag, p.status));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + tb * kTmemBufCols;
+        const int key = key0 + et;
+        // all rows see every key of this tile when its last key is not beyond the first window position
+        const bool all_visible = (n >= p.w) && (key0 + kTileKeys - 1 <= (p.causal ? n - p.w : n - 1)) &&
+                                 (key0 + kTileKeys <= n);
+        float psi_acc = 0.f;
+#pragma unroll
+        for (int cb = 0; cb < NPAD; cb += 32) {
+          float acc[32];
+          tmem_ld32(taddr + cb, acc);
+          if (cb + 32 >= NPAD) {  // accumulator fully read: hand the TMEM buffer back to the MMA warp
+            tc_fence_before();
+            mbar_arrive(&tempty[tb]);
+          }
+          if (it.phase == 1) {
+            if (all_visible) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) {
+                const float s2 = acc[c] * p.scale2;
+                const float mn = fmaxf(st_m[cb + c], s2);
+                st_z[cb + c] = st_z[cb + c] * ex2(st_m[cb + c] - mn) + ex2(s2 - mn);
+                st_m[cb + c] = mn;
+              }
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) {
+                if (key < vis_s[cb + c]) {
+                  const float s2 = acc[c] * p.scale2;
+                  const float mn = fmaxf(st_m[cb + c], s2);
+                  st_z[cb + c] = st_z[cb + c] * ex2(st_m[cb + c] - mn) + ex2(s2 - mn);
+                  st_m[cb + c] = mn;
+                }
+              }
+            }
+          } else {
+            if (all_visible) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (cb + c < p.R) psi_acc += ex2(fmaf(acc[c], p.scale2, -lse_s[cb + c]));
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (key < vis_s[cb + c]) psi_acc += ex2(fmaf(acc[c], p.scale2, -lse_s[cb + c]));
+            }
+          }
+        }
+        if (it.phase == 2 && key < p.n_max) psi[key] = (key < n) ? psi_acc : 0.f;
+        if (++tb == kTmemBufs) {
+          tb = 0;
+          tb_par ^= 1;
+        }
+      }
+      if (!ok) break;
+      if (it.phase == 1) {
+        // reduce the 32 lanes of the warp: after the exchange lane j holds row cb + j
+#pragma unroll
+        for (int cb = 0; cb < NPAD; cb += 32) {
+#pragma unroll
+          for (int s = 16; s >= 1; s >>= 1) {
+#pragma unroll
+            for (int j = 0; j < s; ++j) {
+              const bool up = (lane & s) != 0;
+              const float keep_m = up ? st_m[cb + j + s] : st_m[cb + j];
+              const float keep_z = up ? st_z[cb + j + s] : st_z[cb + j];
+              const float give_m = up ? st_m[cb + j] : st_m[cb + j + s];
+              const float give_z = up ? st_z[cb + j] : st_z[cb + j + s];
+              const float mo = __shfl_xor_sync(0xffffffffu, give_m, s);
+              const float zo = __shfl_xor_sync(0xffffffffu, give_z, s);
+              float m = keep_m, z = keep_z;
+              merge_stats(m, z, mo, zo);
+              st_m[cb + j] = m;
+              st_z[cb + j] = z;
+            }
+          }
+          red_s[quarter * NPAD + cb + lane] = make_float2(st_m[cb], st_z[cb]);
+        }
+        ok = epi_sync(ebar, e_par, abort_flag, p.status);
+        if (!ok) break;
+        if (ethread < NPAD) {
+          float2 a = red_s[ethread];
+#pragma unroll
+          for (int qd = 1; qd < 4; ++qd) {
+            const float2 o = red_s[qd * NPAD + ethread];
+            merge_stats(a.x, a.y, o.x, o.y);
+          }
+          __stcg(p.part + ((int64_t)it.unit * p.cpu + it.chunk) * NPAD + ethread, a);
+          __threadfence();
+        }
+        ok = epi_sync(ebar, e_par, abort_flag, p.status);
+        if (!ok) break;
+        if (ethread == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.done + it.unit) : "memory");
+      }
+    }
+  }
+
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// [B, L, H, tokens, d] bf16 tensor with element strides -> 5-D map, box = {64, box_tokens, box_heads, 1, 1}.
+bool make_map(CUtensorMap* map, const void* base, int d, int tokens, int heads, int L, int B, madakv_strides s,
+              int box_tokens, int box_heads) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[5] = {(cuuint64_t)d, (cuuint64_t)tokens, (cuuint64_t)heads, (cuuint64_t)L, (cuuint64_t)B};
+  // a dimension of extent 1 never advances; give it a harmless valid stride if the caller's is 0
+  auto st = [&](int64_t v, int64_t fallback) { return (cuuint64_t)((v > 0 ? v : fallback) * 2); };
+  const int64_t tok = s.token;
+  const cuuint64_t strides[4] = {st(s.token, d), st(s.head, tok * tokens), st(s.layer, tok * tokens * heads),
+                                 st(s.batch, tok * tokens * heads * L)};
+  for (int i = 0; i < 4; ++i)
+    if (strides[i] % 16 || strides[i] >= ((cuuint64_t)1 << 40)) return false;
+  const cuuint32_t box[5] = {64, (cuuint32_t)box_tokens, (cuuint32_t)box_heads, 1, 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D, int NPAD>
+int run_tc(const CUtensorMap& mk, const CUtensorMap& mq, const TcParams& p, int grid, cudaStream_t st) {
+  using SL = SmemLayout<D, NPAD>;
+  if (cudaFuncSetAttribute(score_tc_kernel<D, NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kAlloc) !=
+      cudaSuccess)
+    return MADAKV_ECUDA;
+  score_tc_kernel<D, NPAD><<<grid, kThreads, SL::kAlloc, st>>>(mk, mq, p);
+  return launch_status();
+}
+
+}  // namespace
+
+bool score_tc_supported(const madakv_config& c, madakv_strides sq, madakv_strides sk) {
+  const int g = c.n_q_heads / c.n_kv_heads;
+  if (c.dtype != MADAKV_BF16 || g * c.window > 64 || c.window > 256 || g > 256) return false;
+  (void)sq;
+  (void)sk;
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess || major != 10)
+    return false;
+  const char* force = getenv("MADAKV_SCORE_PATH");
+  if (force && force[0] == 'g') return false;
+  return encode_fn() != nullptr;
+}
+
+int launch_score_tc(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                    const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st) {
+  const WsLayout wl = ws_layout(c);
+  const int g = c.n_q_heads / c.n_kv_heads;
+  TcParams p;
+  p.seq_len = seq_len;
+  p.psi = psi;
+  p.lse_out = lse;
+  p.part = reinterpret_cast<float2*>((char*)ws + wl.score_part_off);
+  p.done = reinterpret_cast<int32_t*>((char*)ws + wl.score_done_off);
+  p.status = reinterpret_cast<int32_t*>(ws);
+  p.units = c.batch * c.n_layers * c.n_kv_heads;
+  p.L = c.n_layers;
+  p.Hq = c.n_q_heads;
+  p.Hkv = c.n_kv_heads;
+  p.g = g;
+  p.w = c.window;
+  p.R = g * c.window;
+  p.n_max = c.max_seq_len;
+  p.cpu = wl.score_tc_chunks;
+  p.causal = c.causal;
+  p.scale2 = scale_of(c) * kLog2e;
+  const int npad = p.R <= 32 ? 32 : 64;
+
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return MADAKV_ECUDA;
+  const long long total = (long long)p.units * p.cpu;
+  if (total > 0x3fffffff) return MADAKV_EUNSUPPORTED;
+  const int grid = (int)(total < sms ? total : sms);
+  int lag = 2 * grid;
+  if (const char* e = getenv("MADAKV_SCORE_LAG")) lag = atoi(e);
+  if (lag < p.cpu) lag = p.cpu;
+  p.lag = lag;
+
+  CUtensorMap mk, mq;
+  if (!make_map(&mk, k, c.head_dim, c.max_seq_len, c.n_kv_heads, c.n_layers, c.batch, sk, kTileKeys, 1) ||
+      !make_map(&mq, q, c.head_dim, c.window, c.n_q_heads, c.n_layers, c.batch, sq, c.window, g))
+    return MADAKV_EUNSUPPORTED;
+  if (cudaMemsetAsync(p.done, 0, (size_t)p.units * sizeof(int32_t), st) != cudaSuccess) return MADAKV_ECUDA;
+  if (c.head_dim == 128) return npad == 32 ? run_tc<128, 32>(mk, mq, p, grid, st) : run_tc<128, 64>(mk, mq, p, grid, st);
+  return npad == 32 ? run_tc<64, 32>(mk, mq, p, grid, st) : run_tc<64, 64>(mk, mq, p, grid, st);
+}
+
+}  // namespace madakv

@@ -29,6 +29,12 @@ SHAPES = {
     "bf16_d64_long_window": synth.scaled(TINY, dtype="bf16", L=1, Hq=8, Hkv=2, d=64, n=2500, w=64, budget=300,
                                          theta=0.2),
     "f32_d128": synth.scaled(TINY, L=2, Hq=2, Hkv=1, d=128, n=450, w=8, budget=100),
+    # shapes the tensor-core scoring path takes (bf16, g * w <= 64)
+    "tc_d64_r24": synth.scaled(TINY, dtype="bf16", B=2, L=2, Hq=6, Hkv=2, d=64, n=700, w=8, budget=90, theta=0.4),
+    "tc_d128_r64": synth.scaled(TINY, dtype="bf16", L=2, Hq=4, Hkv=2, d=128, n=1500, w=32, budget=250, theta=0.3),
+    "tc_d128_r40": synth.scaled(TINY, dtype="bf16", L=1, Hq=2, Hkv=2, d=128, n=900, w=40, budget=120, theta=0.3),
+    "tc_d64_r64_b3": synth.scaled(TINY, dtype="bf16", B=3, L=2, Hq=2, Hkv=2, d=64, n=2100, w=64, budget=333,
+                                  theta=0.3),
 }
 
 
@@ -72,6 +78,30 @@ def test_score_matches_oracle(name, causal):
     again = torch.empty_like(buf.psi)
     mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], None, again, buf.ws)
     assert torch.equal(again, buf.psi)
+
+
+@pytest.mark.parametrize("lag", ["8", "9", "40", "1000"])
+def test_tensor_core_score_item_interleaving(lag, monkeypatch):
+    # many more work items than the phase-1 lead: exercises the interleaved phase-2 / phase-1 item order and the
+    # waits between CTAs; the result may not depend on the lead (fixed reduction order)
+    wl = synth.scaled(TINY, dtype="bf16", B=2, L=3, Hq=8, Hkv=8, d=128, n=4096, w=32, budget=500, n_needles=8)
+    inp = make_case(wl)
+    cfg = config_of(wl)
+    g = dev(inp)
+    buf = mk.EvictionBuffers(cfg, capacity_of(wl), want_lse=True)
+    mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], buf.lse, buf.psi, buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    base = buf.psi.clone()
+    monkeypatch.setenv("MADAKV_SCORE_LAG", lag)
+    buf.psi.fill_(-1.0)
+    mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], buf.lse, buf.psi, buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    assert torch.equal(buf.psi, base)
+    want = oracle.score(1, to_np(inp["q_win"]), to_np(inp["k"]), to_np(inp["seq_len"]))
+    assert psi_close(buf.psi.cpu().numpy(), want, PSI_RTOL) < PSI_RTOL_SEEN
+    monkeypatch.setenv("MADAKV_SCORE_PATH", "generic")
+    mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], buf.lse, buf.psi, buf.ws)
+    assert psi_close(buf.psi.cpu().numpy(), want, PSI_RTOL) < PSI_RTOL_SEEN
 
 
 @pytest.mark.parametrize("name", list(SHAPES))
