@@ -166,8 +166,12 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-full-cache", action="store_true", help="skip the full-cache decode comparison")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--layers", type=int, default=0, help="profiling only: run a reduced-depth copy of the workload")
     args = ap.parse_args()
     wl = synth.CONFIGS[args.workload]
+    if args.layers > 0:
+        wl = synth.scaled(wl, L=args.layers, name=f"{wl.name}[L={args.layers}]")
     if args.impl == "reference":
         run_reference(args, wl)
         return
@@ -268,12 +272,15 @@ def main():
     dec_gbs = decode_bytes / (stage_ms[4] * 1e-3) / 1e9
 
     # ---- end to end through the C ABI with host buffers (pinned): H2D of the step's inputs, D2H of its result
-    host = {k: v.cpu().pin_memory() for k, v in inp.items()}
-    hdec = [tuple(x.cpu().pin_memory() for x in d) for d in dec]
-    h_out = torch.empty_like(buf.out, device="cpu").pin_memory()
-    h_len = torch.empty_like(buf.kept_len, device="cpu").pin_memory()
-    h2d = sum(v.numel() * v.element_size() for v in host.values()) + sum(x.numel() * x.element_size() for x in hdec[0])
-    d2h = h_out.numel() * h_out.element_size() + h_len.numel() * h_len.element_size()
+    h2d = d2h = 0
+    if not args.no_e2e:
+        host = {k: v.cpu().pin_memory() for k, v in inp.items()}
+        hdec = [tuple(x.cpu().pin_memory() for x in d) for d in dec]
+        h_out = torch.empty_like(buf.out, device="cpu").pin_memory()
+        h_len = torch.empty_like(buf.kept_len, device="cpu").pin_memory()
+        h2d = sum(v.numel() * v.element_size() for v in host.values()) + sum(x.numel() * x.element_size()
+                                                                             for x in hdec[0])
+        d2h = h_out.numel() * h_out.element_size() + h_len.numel() * h_len.element_size()
 
     def e2e_step(i):
         for k_, v_ in host.items():
@@ -284,19 +291,21 @@ def main():
         h_out.copy_(buf.out, non_blocking=True)
         h_len.copy_(buf.kept_len, non_blocking=True)
 
-    e2e_step(0)
-    sync_all()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(args.e2e_steps):
-        e2e_step(i)
-    e1.record()
-    sync_all()
-    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item()) / args.e2e_steps
-    e2e_value = world * tokens / (e2e_ms * 1e-3)
+    e2e_ms = e2e_value = None
+    if not args.no_e2e:
+        e2e_step(0)
+        sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.e2e_steps):
+            e2e_step(i)
+        e1.record()
+        sync_all()
+        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item()) / args.e2e_steps
+        e2e_value = world * tokens / (e2e_ms * 1e-3)
 
     # ---- decode-step latency: compressed cache (per step, all layers in one call) against the full cache
     def time_decode(b, steps=20):

@@ -11,8 +11,10 @@
 //   - a phase-2 item waits (bounded) until all phase-1 items of its unit have published their partials. Every item
 //     only depends on items earlier in the global order and every CTA walks its items in that order, so with all
 //     CTAs resident (grid <= SM count, one CTA per SM) the waits always end.
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-5 epilogue (one TMEM lane quarter each;
-// a thread owns one key of the tile and all window rows of it, so psi(i) is an in-thread sum over N).
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 two epilogue groups that take
+// alternate work items (four warps = the four TMEM lane quarters; a thread owns one key of a tile and all window
+// rows of it, so psi(i) is an in-thread sum over N). The accumulators of a whole item stay in TMEM, so phase 1
+// reads them twice (row maximum, then one exp2 per logit) instead of rescaling a running sum.
 // Every wait is bounded: on expiry the kernel records MADAKV_ETIMEOUT, lets its copies drain, frees TMEM and returns.
 #include <cuda.h>
 #include <cstdlib>
@@ -26,10 +28,8 @@ constexpr int kTileKeys = 128;
 constexpr int kItemTiles = 4;                       // tiles per work item
 constexpr int kItemKeys = kTileKeys * kItemTiles;   // == kScoreTcChunk
 constexpr int kStagesD128 = 5;
-constexpr int kTmemCols = 256;
-constexpr int kTmemBufCols = 64;
-constexpr int kTmemBufs = kTmemCols / kTmemBufCols;
-constexpr int kThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr int kThreads = 320;                        // TMA warp, MMA warp, two epilogue groups of four warps
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kEmptyMax = -1.0e30f;               // "no key seen yet" marker of a running maximum
 constexpr long long kWaitCycles = 4000000000ll;     // ~2 s at B200 clocks: bound of every device-side wait
@@ -217,17 +217,19 @@ struct SmemLayout {
   static constexpr int kKBlocks = D / 64;
   static constexpr int kStageBytes = kTileKeys * D * 2;
   static constexpr int kQBytes = NPAD * D * 2;
+  static constexpr int kItemBufs = kTmemCols / (kItemTiles * NPAD);  // accumulator sets (one work item each) in TMEM
   static constexpr int kKOff = 0;
   static constexpr int kQOff = kStages * kStageBytes;
   static constexpr int kBarOff = kQOff + 2 * kQBytes;
-  static constexpr int kNumBars = 2 * kStages + 4 + 2 * kTmemBufs + 1;
+  // full[kStages], empty[kStages], qfull[2], qempty[2], tfull[kItemBufs * kItemTiles], tempty[kItemBufs], ebar[2]
+  static constexpr int kNumBars = 2 * kStages + 4 + kItemBufs * kItemTiles + kItemBufs + 2;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-  // misc: tmem base (4), abort flag (4), lse2[NPAD], vis[NPAD], red[4][NPAD] float2
-  static constexpr int kLseOff = kMiscOff + 16;
-  static constexpr int kVisOff = kLseOff + NPAD * 4;
-  static constexpr int kRedOff = kVisOff + NPAD * 4;
-  static constexpr int kTotal = kRedOff + 4 * NPAD * 8;
+  // misc: tmem base (4), abort flag (4); then per epilogue group: lse2[NPAD], vis[NPAD], red[4][NPAD] float2
+  static constexpr int kGroupOff = kMiscOff + 16;
+  static constexpr int kGroupBytes = NPAD * 4 + NPAD * 4 + 4 * NPAD * 8;
+  static constexpr int kTotal = kGroupOff + 2 * kGroupBytes;
   static constexpr int kAlloc = kTotal + 1024;  // slack for the 1024-byte alignment of the operand tiles
+  static_assert(kItemBufs >= 2, "each epilogue group needs an accumulator set of its own");
 };
 
 template <int D, int NPAD>
@@ -236,23 +238,22 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
   using SL = SmemLayout<D, NPAD>;
   constexpr int kStages = SL::kStages;
   constexpr int kKBlocks = SL::kKBlocks;
+  constexpr int kItemBufs = SL::kItemBufs;
+  constexpr int kItemCols = kItemTiles * NPAD;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* k_s = smem + SL::kKOff;
   uint8_t* q_s = smem + SL::kQOff;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kBarOff);
-  uint64_t* full = bars;                       // [kStages]   TMA -> MMA
-  uint64_t* empty = bars + kStages;            // [kStages]   MMA -> TMA
-  uint64_t* qfull = bars + 2 * kStages;        // [2]
-  uint64_t* qempty = qfull + 2;                // [2]
-  uint64_t* tfull = qempty + 2;                // [kTmemBufs] MMA -> epilogue
-  uint64_t* tempty = tfull + kTmemBufs;        // [kTmemBufs] epilogue -> MMA
-  uint64_t* ebar = tempty + kTmemBufs;         // barrier of the epilogue threads
+  uint64_t* full = bars;                               // [kStages]                TMA -> MMA
+  uint64_t* empty = bars + kStages;                    // [kStages]                MMA -> TMA
+  uint64_t* qfull = bars + 2 * kStages;                // [2]
+  uint64_t* qempty = qfull + 2;                        // [2]
+  uint64_t* tfull = qempty + 2;                        // [kItemBufs][kItemTiles]  MMA -> epilogue, one per tile
+  uint64_t* tempty = tfull + kItemBufs * kItemTiles;   // [kItemBufs]              epilogue -> MMA, one per item
+  uint64_t* ebars = tempty + kItemBufs;                // [2] barrier of each epilogue group
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(smem + SL::kMiscOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::kMiscOff + 4);
-  float* lse_s = reinterpret_cast<float*>(smem + SL::kLseOff);
-  int* vis_s = reinterpret_cast<int*>(smem + SL::kVisOff);
-  float2* red_s = reinterpret_cast<float2*>(smem + SL::kRedOff);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int total_chunks = p.units * p.cpu;
@@ -266,12 +267,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
     for (int i = 0; i < 2; ++i) {
       mbar_init(&qfull[i], 1);
       mbar_init(&qempty[i], 1);
+      mbar_init(&ebars[i], 128);
     }
-    for (int i = 0; i < kTmemBufs; ++i) {
-      mbar_init(&tfull[i], 1);
-      mbar_init(&tempty[i], 128);
-    }
-    mbar_init(ebar, 128);
+    for (int i = 0; i < kItemBufs * kItemTiles; ++i) mbar_init(&tfull[i], 1);
+    for (int i = 0; i < kItemBufs; ++i) mbar_init(&tempty[i], 128);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -343,8 +342,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
       uint32_t stage_par = 0;
       int qi = 0;
       uint32_t q_par = 0;
-      int tb = 0;
-      uint32_t tb_par = 0;
+      int active = 0;  // active items issued so far; item k uses accumulator set k % kItemBufs
       bool ok = true;
       Item it;
       for (int idx = 0; ok && get_item(blockIdx.x, gridDim.x, idx, total_chunks, p.lag, p.cpu, it); ++idx) {
@@ -352,49 +350,56 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         const int n = min(p.seq_len[b], p.n_max);
         const int key_begin = it.chunk * kItemKeys;
         if (key_begin >= n) continue;
-        ok = mbar_wait(&qfull[qi], q_par, abort_flag, p.status);
+        const int ib = active % kItemBufs;
+        const uint32_t use_par = (uint32_t)(active / kItemBufs) & 1u;
+        ok = mbar_wait(&qfull[qi], q_par, abort_flag, p.status) &&
+             mbar_wait(&tempty[ib], use_par ^ 1, abort_flag, p.status);
         if (!ok) break;
         const uint32_t q_addr = smem_u32(q_s + qi * SL::kQBytes);
         for (int t = 0; t < kItemTiles; ++t) {
           const int key0 = key_begin + t * kTileKeys;
-          if (key0 >= n) break;
-          ok = mbar_wait(&full[stage], stage_par, abort_flag, p.status) &&
-               mbar_wait(&tempty[tb], tb_par ^ 1, abort_flag, p.status);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t k_addr = smem_u32(k_s + stage * SL::kStageBytes);
-          const uint32_t d_tmem = tmem_base + tb * kTmemBufCols;
+          if (key0 < n) {
+            ok = mbar_wait(&full[stage], stage_par, abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t k_addr = smem_u32(k_s + stage * SL::kStageBytes);
+            const uint32_t d_tmem = tmem_base + ib * kItemCols + t * NPAD;
 #pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            const int kb = ks >> 2, kk = ks & 3;
-            const uint64_t a = smem_desc_sw128(k_addr + kb * kTileKeys * 128 + kk * 32);
-            const uint64_t bq = smem_desc_sw128(q_addr + kb * NPAD * 128 + kk * 32);
-            umma_bf16(d_tmem, a, bq, idesc, ks > 0 ? 1u : 0u);
+            for (int ks = 0; ks < D / 16; ++ks) {
+              const int kb = ks >> 2, kk = ks & 3;
+              const uint64_t a = smem_desc_sw128(k_addr + kb * kTileKeys * 128 + kk * 32);
+              const uint64_t bq = smem_desc_sw128(q_addr + kb * NPAD * 128 + kk * 32);
+              umma_bf16(d_tmem, a, bq, idesc, ks > 0 ? 1u : 0u);
+            }
+            umma_commit(&empty[stage]);  // the K stage may be refilled once these MMAs have read it
+            if (++stage == kStages) {
+              stage = 0;
+              stage_par ^= 1;
+            }
           }
-          umma_commit(&empty[stage]);  // the K stage may be refilled once these MMAs have read it
-          umma_commit(&tfull[tb]);     // the accumulator is complete
-          if (++stage == kStages) {
-            stage = 0;
-            stage_par ^= 1;
-          }
-          if (++tb == kTmemBufs) {
-            tb = 0;
-            tb_par ^= 1;
-          }
+          umma_commit(&tfull[ib * kItemTiles + t]);  // every tile barrier completes once per use of the set
         }
         if (!ok) break;
         umma_commit(&qempty[qi]);  // the Q buffer may be refilled once this item's MMAs are done
         qi ^= 1;
         if (qi == 0) q_par ^= 1;
+        ++active;
       }
     }
   } else {
-    // ================================================================ epilogue (128 threads, one key each)
+    // ================================================================ epilogue: two groups of 128 threads; group e
+    // takes the active items of its parity. A thread owns one key of each tile (one TMEM lane).
+    const int grp = (warp - 2) >> 2;              // 0 or 1
     const int quarter = warp & 3;                 // TMEM lanes [32 * quarter, 32 * quarter + 32)
     const int et = (quarter << 5) | lane;         // key index inside the tile
-    const int ethread = threadIdx.x - 64;         // 0..127 in launch order (used for row-parallel steps)
-    int tb = 0;
-    uint32_t tb_par = 0, e_par = 0;
+    const int ethread = (((warp - 2) & 3) << 5) | lane;  // 0..127 inside the group
+    uint8_t* gbase = smem + SL::kGroupOff + grp * SL::kGroupBytes;
+    float* lse_s = reinterpret_cast<float*>(gbase);
+    int* vis_s = reinterpret_cast<int*>(gbase + NPAD * 4);
+    float2* red_s = reinterpret_cast<float2*>(gbase + NPAD * 8);
+    uint64_t* ebar = &ebars[grp];
+    uint32_t e_par = 0;
+    int active = 0;
     bool ok = true;
     Item it;
     for (int idx = 0; ok && get_item(blockIdx.x, gridDim.x, idx, total_chunks, p.lag, p.cpu, it); ++idx) {
@@ -403,15 +408,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
       const int key_begin = it.chunk * kItemKeys;
       float* psi = p.psi + (int64_t)it.unit * p.n_max;
       if (key_begin >= n) {
-        if (it.phase == 2)  // beyond the sequence: psi = 0
+        if (it.phase == 2 && grp == 0)  // beyond the sequence: psi = 0
           for (int t = 0; t < kItemTiles; ++t) {
             const int key = key_begin + t * kTileKeys + et;
             if (key < p.n_max) psi[key] = 0.f;
           }
         continue;
       }
+      const int k_item = active++;
+      if ((k_item & 1) != grp) continue;
+      const int ib = k_item % kItemBufs;
+      const uint32_t use_par = (uint32_t)(k_item / kItemBufs) & 1u;
+      const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + ib * kItemCols;
+
       // per-row visibility bound (exclusive key index) of this unit
-      ok = epi_sync(ebar, e_par, abort_flag, p.status);  // previous item's readers of the shared arrays are done
+      ok = epi_sync(ebar, e_par, abort_flag, p.status);  // the previous item's readers of the shared arrays are done
       if (!ok) break;
       if (ethread < NPAD) {
         int vis = 0;
@@ -422,7 +433,107 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         vis_s[ethread] = vis;
       }
       const int n_chunks_active = (n + kItemKeys - 1) / kItemKeys;
-      if (it.phase == 2) {
+      // keys below this bound are seen by every window row
+      const int all_bound = (n >= p.w) ? (p.causal ? n - p.w + 1 : n) : 0;
+
+      if (it.phase == 1) {
+        ok = epi_sync(ebar, e_par, abort_flag, p.status);  // vis_s is published
+        if (!ok) break;
+        // pass A: running maximum of the raw logits of this lane's keys, per window row
+        float st_m[NPAD], st_z[NPAD];
+#pragma unroll
+        for (int c = 0; c < NPAD; ++c) {
+          st_m[c] = kEmptyMax;
+          st_z[c] = 0.f;
+        }
+        for (int t = 0; t < kItemTiles; ++t) {
+          const int key0 = key_begin + t * kTileKeys;
+          if (key0 >= n) break;
+          ok = __all_sync(0xffffffffu, mbar_wait(&tfull[ib * kItemTiles + t], use_par, abort_flag, p.status));
+          if (!ok) break;
+          tc_fence_after();
+          const bool masked = key0 + kTileKeys > all_bound;
+#pragma unroll
+          for (int cb = 0; cb < NPAD; cb += 32) {
+            float acc[32];
+            tmem_ld32(tbase + t * NPAD + cb, acc);
+            if (masked) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (key0 + et >= vis_s[cb + c]) acc[c] = kEmptyMax;
+            }
+#pragma unroll
+            for (int c = 0; c < 32; ++c) st_m[cb + c] = fmaxf(st_m[cb + c], acc[c]);
+          }
+        }
+        if (!ok) break;
+        // pass B: sum of exp2 against that maximum (second read of the accumulators, still in TMEM)
+#pragma unroll
+        for (int c = 0; c < NPAD; ++c) st_m[c] *= p.scale2;
+        for (int t = 0; t < kItemTiles; ++t) {
+          const int key0 = key_begin + t * kTileKeys;
+          if (key0 >= n) break;
+          const bool masked = key0 + kTileKeys > all_bound;
+#pragma unroll
+          for (int cb = 0; cb < NPAD; cb += 32) {
+            float acc[32];
+            tmem_ld32(tbase + t * NPAD + cb, acc);
+            if (masked) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (key0 + et >= vis_s[cb + c]) acc[c] = kEmptyMax;
+            }
+#pragma unroll
+            for (int c = 0; c < 32; ++c) st_z[cb + c] += ex2(fmaf(acc[c], p.scale2, -st_m[cb + c]));
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(&tempty[ib]);  // accumulators fully read: hand the set back to the MMA warp
+        // a row for which this lane saw no visible key: exp2(0) was summed for masked entries, drop it
+#pragma unroll
+        for (int c = 0; c < NPAD; ++c)
+          if (st_m[c] < 0.5f * kEmptyMax * p.scale2) {
+            st_m[c] = kEmptyMax;
+            st_z[c] = 0.f;
+          }
+        // reduce the 32 lanes of the warp: after the exchange lane j holds row cb + j
+#pragma unroll
+        for (int cb = 0; cb < NPAD; cb += 32) {
+#pragma unroll
+          for (int s = 16; s >= 1; s >>= 1) {
+#pragma unroll
+            for (int j = 0; j < s; ++j) {
+              const bool up = (lane & s) != 0;
+              const float keep_m = up ? st_m[cb + j + s] : st_m[cb + j];
+              const float keep_z = up ? st_z[cb + j + s] : st_z[cb + j];
+              const float give_m = up ? st_m[cb + j] : st_m[cb + j + s];
+              const float give_z = up ? st_z[cb + j] : st_z[cb + j + s];
+              const float mo = __shfl_xor_sync(0xffffffffu, give_m, s);
+              const float zo = __shfl_xor_sync(0xffffffffu, give_z, s);
+              float m = keep_m, z = keep_z;
+              merge_stats(m, z, mo, zo);
+              st_m[cb + j] = m;
+              st_z[cb + j] = z;
+            }
+          }
+          red_s[(ethread >> 5) * NPAD + cb + lane] = make_float2(st_m[cb], st_z[cb]);
+        }
+        ok = epi_sync(ebar, e_par, abort_flag, p.status);
+        if (!ok) break;
+        if (ethread < NPAD) {
+          float2 a = red_s[ethread];
+#pragma unroll
+          for (int qd = 1; qd < 4; ++qd) {
+            const float2 o = red_s[qd * NPAD + ethread];
+            merge_stats(a.x, a.y, o.x, o.y);
+          }
+          __stcg(p.part + ((int64_t)it.unit * p.cpu + it.chunk) * NPAD + ethread, a);
+          __threadfence();
+        }
+        ok = epi_sync(ebar, e_par, abort_flag, p.status);
+        if (!ok) break;
+        if (ethread == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.done + it.unit) : "memory");
+      } else {
         // wait until every phase-1 item of this unit has published its partials
         if (ethread == 0) {
           const long long t0 = clock64();
@@ -457,118 +568,40 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
             p.lse_out[((int64_t)bl * p.Hq + hq) * p.w + wr] = (Z > 0.f) ? lse2 * 0.6931471805599453f : -INFINITY;
           }
         }
-      }
-      ok = epi_sync(ebar, e_par, abort_flag, p.status);
-      if (!ok) break;
-
-      float st_m[NPAD], st_z[NPAD];  // phase 1: this lane's running statistics per window row
-      if (it.phase == 1) {
-#pragma unroll
-        for (int c = 0; c < NPAD; ++c) {
-          st_m[c] = kEmptyMax;
-          st_z[c] = 0.f;
-        }
-      }
-      for (int t = 0; t < kItemTiles; ++t) {
-        const int key0 = key_begin + t * kTileKeys;
-        if (key0 >= n) {
-          if (it.phase == 2 && key0 + et < p.n_max) psi[key0 + et] = 0.f;
-          continue;
-        }
-        ok = __all_sync(0xffffffffu, mbar_wait(&tfull[tb], tb_par, abort_flag, p.status));
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + tb * kTmemBufCols;
-        const int key = key0 + et;
-        // all rows see every key of this tile when its last key is not beyond the first window position
-        const bool all_visible = (n >= p.w) && (key0 + kTileKeys - 1 <= (p.causal ? n - p.w : n - 1)) &&
-                                 (key0 + kTileKeys <= n);
-        float psi_acc = 0.f;
-#pragma unroll
-        for (int cb = 0; cb < NPAD; cb += 32) {
-          float acc[32];
-          tmem_ld32(taddr + cb, acc);
-          if (cb + 32 >= NPAD) {  // accumulator fully read: hand the TMEM buffer back to the MMA warp
-            tc_fence_before();
-            mbar_arrive(&tempty[tb]);
-          }
-          if (it.phase == 1) {
-            if (all_visible) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c) {
-                const float s2 = acc[c] * p.scale2;
-                const float mn = fmaxf(st_m[cb + c], s2);
-                st_z[cb + c] = st_z[cb + c] * ex2(st_m[cb + c] - mn) + ex2(s2 - mn);
-                st_m[cb + c] = mn;
-              }
-            } else {
-#pragma unroll
-              for (int c = 0; c < 32; ++c) {
-                if (key < vis_s[cb + c]) {
-                  const float s2 = acc[c] * p.scale2;
-                  const float mn = fmaxf(st_m[cb + c], s2);
-                  st_z[cb + c] = st_z[cb + c] * ex2(st_m[cb + c] - mn) + ex2(s2 - mn);
-                  st_m[cb + c] = mn;
-                }
-              }
-            }
-          } else {
-            if (all_visible) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (cb + c < p.R) psi_acc += ex2(fmaf(acc[c], p.scale2, -lse_s[cb + c]));
-            } else {
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (key < vis_s[cb + c]) psi_acc += ex2(fmaf(acc[c], p.scale2, -lse_s[cb + c]));
-            }
-          }
-        }
-        if (it.phase == 2 && key < p.n_max) psi[key] = (key < n) ? psi_acc : 0.f;
-        if (++tb == kTmemBufs) {
-          tb = 0;
-          tb_par ^= 1;
-        }
-      }
-      if (!ok) break;
-      if (it.phase == 1) {
-        // reduce the 32 lanes of the warp: after the exchange lane j holds row cb + j
-#pragma unroll
-        for (int cb = 0; cb < NPAD; cb += 32) {
-#pragma unroll
-          for (int s = 16; s >= 1; s >>= 1) {
-#pragma unroll
-            for (int j = 0; j < s; ++j) {
-              const bool up = (lane & s) != 0;
-              const float keep_m = up ? st_m[cb + j + s] : st_m[cb + j];
-              const float keep_z = up ? st_z[cb + j + s] : st_z[cb + j];
-              const float give_m = up ? st_m[cb + j] : st_m[cb + j + s];
-              const float give_z = up ? st_z[cb + j] : st_z[cb + j + s];
-              const float mo = __shfl_xor_sync(0xffffffffu, give_m, s);
-              const float zo = __shfl_xor_sync(0xffffffffu, give_z, s);
-              float m = keep_m, z = keep_z;
-              merge_stats(m, z, mo, zo);
-              st_m[cb + j] = m;
-              st_z[cb + j] = z;
-            }
-          }
-          red_s[quarter * NPAD + cb + lane] = make_float2(st_m[cb], st_z[cb]);
-        }
         ok = epi_sync(ebar, e_par, abort_flag, p.status);
         if (!ok) break;
-        if (ethread < NPAD) {
-          float2 a = red_s[ethread];
+        float lse_r[NPAD];
 #pragma unroll
-          for (int qd = 1; qd < 4; ++qd) {
-            const float2 o = red_s[qd * NPAD + ethread];
-            merge_stats(a.x, a.y, o.x, o.y);
+        for (int c = 0; c < NPAD; ++c) lse_r[c] = (c < p.R) ? lse_s[c] : -kEmptyMax;  // padding rows add exp2(-huge) = 0
+        for (int t = 0; t < kItemTiles; ++t) {
+          const int key0 = key_begin + t * kTileKeys;
+          const int key = key0 + et;
+          if (key0 >= n) {
+            if (key < p.n_max) psi[key] = 0.f;
+            continue;
           }
-          __stcg(p.part + ((int64_t)it.unit * p.cpu + it.chunk) * NPAD + ethread, a);
-          __threadfence();
+          ok = __all_sync(0xffffffffu, mbar_wait(&tfull[ib * kItemTiles + t], use_par, abort_flag, p.status));
+          if (!ok) break;
+          tc_fence_after();
+          const bool masked = key0 + kTileKeys > all_bound;
+          float psi_acc = 0.f;
+#pragma unroll
+          for (int cb = 0; cb < NPAD; cb += 32) {
+            float acc[32];
+            tmem_ld32(tbase + t * NPAD + cb, acc);
+            if (masked) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (key >= vis_s[cb + c]) acc[c] = kEmptyMax;
+            }
+#pragma unroll
+            for (int c = 0; c < 32; ++c) psi_acc += ex2(fmaf(acc[c], p.scale2, -lse_r[cb + c]));
+          }
+          if (key < p.n_max) psi[key] = (key < n) ? psi_acc : 0.f;
         }
-        ok = epi_sync(ebar, e_par, abort_flag, p.status);
         if (!ok) break;
-        if (ethread == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.done + it.unit) : "memory");
+        tc_fence_before();
+        mbar_arrive(&tempty[ib]);
       }
     }
   }
