@@ -4,6 +4,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
 
 #include "madakv.h"
 
@@ -98,7 +100,12 @@ inline int check_ws(const madakv_config& c, const void* ws, size_t ws_bytes) {
 inline float scale_of(const madakv_config& c) {
   return c.softmax_scale > 0.0f ? c.softmax_scale : 1.0f / sqrtf((float)c.head_dim);
 }
-inline int launch_status() { return cudaGetLastError() == cudaSuccess ? MADAKV_OK : MADAKV_ECUDA; }
+inline int launch_status() {
+  const cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) return MADAKV_OK;
+  if (getenv("MADAKV_DEBUG")) fprintf(stderr, "madakv: CUDA error %d (%s)\n", (int)e, cudaGetErrorString(e));
+  return MADAKV_ECUDA;
+}
 
 // ---------------------------------------------------------------------------------------------------------------
 // Device helpers

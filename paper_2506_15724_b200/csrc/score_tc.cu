@@ -4,7 +4,7 @@
 //   - the window-QK^T tile is a tcgen05.mma with the 128 keys of a tile on M, the g*w window rows on N and head_dim
 //     on K; operands are staged in shared memory by TMA (128-byte swizzle), the fp32 accumulator lives in TMEM;
 //   - a softmax over keys needs every row's log-sum-exp before any normalised weight can be summed over rows, so
-//     the work is cut into items of kItemTiles tiles in two phases: phase-1 items produce per-row (max, sum exp2)
+//     the work is cut into items of 4 or 8 tiles in two phases: phase-1 items produce per-row (max, sum exp2)
 //     partials, phase-2 items recompute the logits and emit psi. The item list interleaves phase 2 of chunk t with
 //     phase 1 of chunk t + lag, so the second read of a K chunk comes a bounded number of chunks after the first
 //     and is served by the L2 (phase-1 loads ask L2 to keep the lines, phase-2 loads to drop them);
@@ -25,8 +25,7 @@ namespace madakv {
 namespace {
 
 constexpr int kTileKeys = 128;
-constexpr int kItemTiles = 4;                       // tiles per work item
-constexpr int kItemKeys = kTileKeys * kItemTiles;   // == kScoreTcChunk
+constexpr int kItemCols = 256;                      // TMEM columns of one work item's accumulators
 constexpr int kStagesD128 = 5;
 constexpr int kTmemCols = 512;
 constexpr int kThreads = 320;                        // TMA warp, MMA warp, two epilogue groups of four warps
@@ -34,7 +33,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kEmptyMax = -1.0e30f;               // "no key seen yet" marker of a running maximum
 constexpr long long kWaitCycles = 4000000000ll;     // ~2 s at B200 clocks: bound of every device-side wait
 
-static_assert(kItemKeys == kScoreTcChunk, "partials are indexed by kScoreTcChunk keys");
+static_assert(kTileKeys * (kItemCols / 64) == kScoreTcChunk, "the workspace is sized for the smallest work item");
 
 struct TcParams {
   const int32_t* seq_len;
@@ -137,8 +136,8 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
-  uint32_t r[32];
+// Issue a 32-column TMEM load of this thread's lane; the registers are valid only after tmem_ld_wait on them.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -149,9 +148,52 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// Wait for this thread's outstanding TMEM loads. The registers pass through the statement so that no use of them
+// can be scheduled before the wait.
+#define MADAKV_R8(r, o) "+r"(r[o]), "+r"(r[o + 1]), "+r"(r[o + 2]), "+r"(r[o + 3]), "+r"(r[o + 4]), "+r"(r[o + 5]), \
+                        "+r"(r[o + 6]), "+r"(r[o + 7])
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&a)[32], uint32_t (&b)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : MADAKV_R8(a, 0), MADAKV_R8(a, 8), MADAKV_R8(a, 16), MADAKV_R8(a, 24), MADAKV_R8(b, 0), MADAKV_R8(b, 8),
+                 MADAKV_R8(b, 16), MADAKV_R8(b, 24)
+               :
+               : "memory");
+}
+#undef MADAKV_R8
+__device__ __forceinline__ float warp_max(float v) {
+  float r;
+  asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// packed pairs of fp32 (sm_100 f32x2 arithmetic): one instruction per two logits
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ uint64_t pack2u(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -211,25 +253,56 @@ __device__ __forceinline__ bool get_item(int cta, int G, int idx, int total_chun
   return true;
 }
 
+// exp2 of 32 scaled-and-shifted logits, summed into 16 packed accumulators: acc2[i] += exp2(raw * scale - shift)
+__device__ __forceinline__ void exp_accumulate(const uint32_t (&raw)[32], uint64_t scale2x, const uint64_t* negshift2,
+                                               uint64_t (&acc2)[16]) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    float lo, hi;
+    unpack2(fma2(pack2u(raw[2 * i], raw[2 * i + 1]), scale2x, negshift2[i]), lo, hi);
+    acc2[i] = add2(acc2[i], pack2(ex2(lo), ex2(hi)));
+  }
+}
+// the same, all 32 summed into one packed accumulator (phase 2: sum over window rows)
+__device__ __forceinline__ uint64_t exp_sum(const uint32_t (&raw)[32], uint64_t scale2x, const uint64_t* negshift2,
+                                            uint64_t acc) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    float lo, hi;
+    unpack2(fma2(pack2u(raw[2 * i], raw[2 * i + 1]), scale2x, negshift2[i]), lo, hi);
+    acc = add2(acc, pack2(ex2(lo), ex2(hi)));
+  }
+  return acc;
+}
+// logits of keys a window row may not see are replaced by a huge negative value
+__device__ __forceinline__ void mask_slab(uint32_t (&raw)[32], int key, const int* vis) {
+#pragma unroll
+  for (int c = 0; c < 32; ++c)
+    if (key >= vis[c]) raw[c] = __float_as_uint(kEmptyMax);
+}
+
 template <int D, int NPAD>
 struct SmemLayout {
-  static constexpr int kStages = D == 128 ? kStagesD128 : 2 * kStagesD128;
+  static constexpr int kStages = (D == 128 ? 1 : 2) * (NPAD == 32 ? kStagesD128 : kStagesD128 - 1);
   static constexpr int kKBlocks = D / 64;
   static constexpr int kStageBytes = kTileKeys * D * 2;
   static constexpr int kQBytes = NPAD * D * 2;
-  static constexpr int kItemBufs = kTmemCols / (kItemTiles * NPAD);  // accumulator sets (one work item each) in TMEM
+  static constexpr int kItemTiles = kItemCols / NPAD;     // tiles per work item: 8 (NPAD 32) or 4 (NPAD 64)
+  static constexpr int kItemKeys = kItemTiles * kTileKeys;
+  static constexpr int kItemBufs = kTmemCols / kItemCols;  // accumulator sets (one work item each) in TMEM
   static constexpr int kKOff = 0;
   static constexpr int kQOff = kStages * kStageBytes;
   static constexpr int kBarOff = kQOff + 2 * kQBytes;
   // full[kStages], empty[kStages], qfull[2], qempty[2], tfull[kItemBufs * kItemTiles], tempty[kItemBufs], ebar[2]
   static constexpr int kNumBars = 2 * kStages + 4 + kItemBufs * kItemTiles + kItemBufs + 2;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-  // misc: tmem base (4), abort flag (4); then per epilogue group: lse2[NPAD], vis[NPAD], red[4][NPAD] float2
+  // misc: tmem base (4), abort flag (4); then per epilogue group: lse2[NPAD], vis[NPAD], red[4][NPAD] float2 and
+  // a padded 32 x 33 transpose tile per warp
   static constexpr int kGroupOff = kMiscOff + 16;
-  static constexpr int kGroupBytes = NPAD * 4 + NPAD * 4 + 4 * NPAD * 8;
+  static constexpr int kGroupBytes = NPAD * 4 + NPAD * 4 + 4 * NPAD * 8 + 4 * 32 * 33 * 4;
   static constexpr int kTotal = kGroupOff + 2 * kGroupBytes;
   static constexpr int kAlloc = kTotal + 1024;  // slack for the 1024-byte alignment of the operand tiles
-  static_assert(kItemBufs >= 2, "each epilogue group needs an accumulator set of its own");
+  static_assert(kItemBufs == 2, "each epilogue group owns one accumulator set");
 };
 
 template <int D, int NPAD>
@@ -239,7 +312,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
   constexpr int kStages = SL::kStages;
   constexpr int kKBlocks = SL::kKBlocks;
   constexpr int kItemBufs = SL::kItemBufs;
-  constexpr int kItemCols = kItemTiles * NPAD;
+  constexpr int kItemTiles = SL::kItemTiles;
+  constexpr int kItemKeys = SL::kItemKeys;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* k_s = smem + SL::kKOff;
@@ -397,6 +471,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
     float* lse_s = reinterpret_cast<float*>(gbase);
     int* vis_s = reinterpret_cast<int*>(gbase + NPAD * 4);
     float2* red_s = reinterpret_cast<float2*>(gbase + NPAD * 8);
+    float* tr_s = reinterpret_cast<float*>(gbase + NPAD * 8 + 4 * NPAD * 8);
     uint64_t* ebar = &ebars[grp];
     uint32_t e_par = 0;
     int active = 0;
@@ -439,84 +514,118 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
       if (it.phase == 1) {
         ok = epi_sync(ebar, e_par, abort_flag, p.status);  // vis_s is published
         if (!ok) break;
-        // pass A: running maximum of the raw logits of this lane's keys, per window row
-        float st_m[NPAD], st_z[NPAD];
+        // Two 32-column slabs are in registers at a time: tiles t and t + 1 (NPAD 32) or the two column halves of
+        // tile t (NPAD 64).
+        constexpr int kTilesPerPair = NPAD == 32 ? 2 : 1;
+        int nt = 0;
+        while (nt < kItemTiles && key_begin + nt * kTileKeys < n) ++nt;
+        const uint64_t* tf = &tfull[ib * kItemTiles];
+        // pass A: maximum of the raw logits per window row over this lane's keys, then over the warp
+        float st_m[NPAD];
 #pragma unroll
-        for (int c = 0; c < NPAD; ++c) {
-          st_m[c] = kEmptyMax;
-          st_z[c] = 0.f;
-        }
-        for (int t = 0; t < kItemTiles; ++t) {
+        for (int c = 0; c < NPAD; ++c) st_m[c] = kEmptyMax;
+        for (int t = 0; t < nt; t += kTilesPerPair) {
+          uint32_t ra[32], rb[32];
           const int key0 = key_begin + t * kTileKeys;
-          if (key0 >= n) break;
-          ok = __all_sync(0xffffffffu, mbar_wait(&tfull[ib * kItemTiles + t], use_par, abort_flag, p.status));
+          const bool two = NPAD == 64 || t + 1 < nt;
+          ok = __all_sync(0xffffffffu, mbar_wait(const_cast<uint64_t*>(&tf[t]), use_par, abort_flag, p.status) &&
+                                           (NPAD == 64 || !two ||
+                                            mbar_wait(const_cast<uint64_t*>(&tf[t + 1]), use_par, abort_flag, p.status)));
           if (!ok) break;
           tc_fence_after();
-          const bool masked = key0 + kTileKeys > all_bound;
+          tmem_ld32_issue(tbase + t * NPAD, ra);
+          if (two) tmem_ld32_issue(tbase + t * NPAD + 32, rb);  // next tile (NPAD 32) or upper columns (NPAD 64)
+          tmem_ld_wait(ra, rb);
+          if (!two) {
 #pragma unroll
-          for (int cb = 0; cb < NPAD; cb += 32) {
-            float acc[32];
-            tmem_ld32(tbase + t * NPAD + cb, acc);
-            if (masked) {
+            for (int c = 0; c < 32; ++c) rb[c] = __float_as_uint(kEmptyMax);
+          }
+          if (key0 + kTilesPerPair * kTileKeys > all_bound) {
+            mask_slab(ra, key0 + et, vis_s);
+            if (two) mask_slab(rb, (NPAD == 32 ? key0 + kTileKeys : key0) + et, vis_s + (NPAD == 32 ? 0 : 32));
+          }
+          if constexpr (NPAD == 32) {
 #pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (key0 + et >= vis_s[cb + c]) acc[c] = kEmptyMax;
+            for (int c = 0; c < 32; ++c) st_m[c] = max3(st_m[c], __uint_as_float(ra[c]), __uint_as_float(rb[c]));
+          } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              st_m[c] = fmaxf(st_m[c], __uint_as_float(ra[c]));
+              st_m[32 + c] = fmaxf(st_m[32 + c], __uint_as_float(rb[c]));
             }
-#pragma unroll
-            for (int c = 0; c < 32; ++c) st_m[cb + c] = fmaxf(st_m[cb + c], acc[c]);
           }
         }
         if (!ok) break;
-        // pass B: sum of exp2 against that maximum (second read of the accumulators, still in TMEM)
+        // pass B: sum of exp2 against the warp's maximum (second read of the accumulators, still in TMEM)
+        uint64_t negm2[NPAD / 2], z2[NPAD / 2];
 #pragma unroll
-        for (int c = 0; c < NPAD; ++c) st_m[c] *= p.scale2;
-        for (int t = 0; t < kItemTiles; ++t) {
+        for (int i = 0; i < NPAD / 2; ++i) {
+          negm2[i] = pack2(-(warp_max(st_m[2 * i]) * p.scale2), -(warp_max(st_m[2 * i + 1]) * p.scale2));
+          z2[i] = 0ull;
+        }
+        const uint64_t scale2x = pack2(p.scale2, p.scale2);
+        for (int t = 0; t < nt; t += kTilesPerPair) {
+          uint32_t ra[32], rb[32];
           const int key0 = key_begin + t * kTileKeys;
-          if (key0 >= n) break;
-          const bool masked = key0 + kTileKeys > all_bound;
-#pragma unroll
-          for (int cb = 0; cb < NPAD; cb += 32) {
-            float acc[32];
-            tmem_ld32(tbase + t * NPAD + cb, acc);
-            if (masked) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (key0 + et >= vis_s[cb + c]) acc[c] = kEmptyMax;
+          const bool two = NPAD == 64 || t + 1 < nt;
+          const bool msk = key0 + kTilesPerPair * kTileKeys > all_bound;
+          tmem_ld32_issue(tbase + t * NPAD, ra);
+          tmem_ld_wait(ra, ra);
+          if (msk) mask_slab(ra, key0 + et, vis_s);
+          if constexpr (NPAD == 32) {
+            exp_accumulate(ra, scale2x, negm2, z2);
+            if (two) {
+              tmem_ld32_issue(tbase + t * NPAD + 32, ra);
+              tmem_ld_wait(ra, ra);
+              if (msk) mask_slab(ra, key0 + kTileKeys + et, vis_s);
+              exp_accumulate(ra, scale2x, negm2, z2);
             }
-#pragma unroll
-            for (int c = 0; c < 32; ++c) st_z[cb + c] += ex2(fmaf(acc[c], p.scale2, -st_m[cb + c]));
+          } else {
+            tmem_ld32_issue(tbase + t * NPAD + 32, rb);
+            tmem_ld_wait(rb, rb);
+            if (msk) mask_slab(rb, key0 + et, vis_s + 32);
+            exp_accumulate(ra, scale2x, negm2, reinterpret_cast<uint64_t(&)[16]>(z2[0]));
+            exp_accumulate(rb, scale2x, negm2 + 16, reinterpret_cast<uint64_t(&)[16]>(z2[16]));
           }
         }
         tc_fence_before();
         mbar_arrive(&tempty[ib]);  // accumulators fully read: hand the set back to the MMA warp
-        // a row for which this lane saw no visible key: exp2(0) was summed for masked entries, drop it
+        // back to scalars; a row of which the whole warp saw no visible key summed exp2(0) for its masked entries:
+        // such a row is recorded as empty
+        float st_z[NPAD];
+#pragma unroll
+        for (int i = 0; i < NPAD / 2; ++i) {
+          float a, b;
+          unpack2(negm2[i], a, b);
+          st_m[2 * i] = -a;
+          st_m[2 * i + 1] = -b;
+          unpack2(z2[i], st_z[2 * i], st_z[2 * i + 1]);
+        }
 #pragma unroll
         for (int c = 0; c < NPAD; ++c)
           if (st_m[c] < 0.5f * kEmptyMax * p.scale2) {
             st_m[c] = kEmptyMax;
             st_z[c] = 0.f;
           }
-        // reduce the 32 lanes of the warp: after the exchange lane j holds row cb + j
+        // sum over the 32 lanes of the warp through a padded shared-memory transpose (fixed order): lane j ends up
+        // with the sum of row cb + j; the maximum is already uniform over the warp
+        {
+          float* tr = tr_s + (ethread >> 5) * (32 * 33);
 #pragma unroll
-        for (int cb = 0; cb < NPAD; cb += 32) {
+          for (int cb = 0; cb < NPAD; cb += 32) {
 #pragma unroll
-          for (int s = 16; s >= 1; s >>= 1) {
+            for (int c = 0; c < 32; ++c) tr[c * 33 + lane] = st_z[cb + c];
+            if (lane == 0) {
 #pragma unroll
-            for (int j = 0; j < s; ++j) {
-              const bool up = (lane & s) != 0;
-              const float keep_m = up ? st_m[cb + j + s] : st_m[cb + j];
-              const float keep_z = up ? st_z[cb + j + s] : st_z[cb + j];
-              const float give_m = up ? st_m[cb + j] : st_m[cb + j + s];
-              const float give_z = up ? st_z[cb + j] : st_z[cb + j + s];
-              const float mo = __shfl_xor_sync(0xffffffffu, give_m, s);
-              const float zo = __shfl_xor_sync(0xffffffffu, give_z, s);
-              float m = keep_m, z = keep_z;
-              merge_stats(m, z, mo, zo);
-              st_m[cb + j] = m;
-              st_z[cb + j] = z;
+              for (int c = 0; c < 32; ++c) red_s[(ethread >> 5) * NPAD + cb + c].x = st_m[cb + c];
             }
+            __syncwarp();
+            float zsum = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) zsum += tr[lane * 33 + i];
+            red_s[(ethread >> 5) * NPAD + cb + lane].y = zsum;
+            __syncwarp();
           }
-          red_s[(ethread >> 5) * NPAD + cb + lane] = make_float2(st_m[cb], st_z[cb]);
         }
         ok = epi_sync(ebar, e_par, abort_flag, p.status);
         if (!ok) break;
@@ -570,34 +679,52 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         }
         ok = epi_sync(ebar, e_par, abort_flag, p.status);
         if (!ok) break;
-        float lse_r[NPAD];
+        constexpr int kTilesPerPair = NPAD == 32 ? 2 : 1;
+        uint64_t neglse2[NPAD / 2];
 #pragma unroll
-        for (int c = 0; c < NPAD; ++c) lse_r[c] = (c < p.R) ? lse_s[c] : -kEmptyMax;  // padding rows add exp2(-huge) = 0
-        for (int t = 0; t < kItemTiles; ++t) {
+        for (int i = 0; i < NPAD / 2; ++i)  // padding rows get a huge shift: they add exp2(-huge) = 0
+          neglse2[i] = pack2(2 * i < p.R ? -lse_s[2 * i] : kEmptyMax, 2 * i + 1 < p.R ? -lse_s[2 * i + 1] : kEmptyMax);
+        const uint64_t scale2x = pack2(p.scale2, p.scale2);
+        int nt = 0;
+        while (nt < kItemTiles && key_begin + nt * kTileKeys < n) ++nt;
+        const uint64_t* tf = &tfull[ib * kItemTiles];
+        for (int t = 0; t < nt; t += kTilesPerPair) {
+          uint32_t ra[32], rb[32];
           const int key0 = key_begin + t * kTileKeys;
-          const int key = key0 + et;
-          if (key0 >= n) {
-            if (key < p.n_max) psi[key] = 0.f;
-            continue;
-          }
-          ok = __all_sync(0xffffffffu, mbar_wait(&tfull[ib * kItemTiles + t], use_par, abort_flag, p.status));
+          const bool two = NPAD == 64 || t + 1 < nt;
+          ok = __all_sync(0xffffffffu, mbar_wait(const_cast<uint64_t*>(&tf[t]), use_par, abort_flag, p.status) &&
+                                           (NPAD == 64 || !two ||
+                                            mbar_wait(const_cast<uint64_t*>(&tf[t + 1]), use_par, abort_flag, p.status)));
           if (!ok) break;
           tc_fence_after();
-          const bool masked = key0 + kTileKeys > all_bound;
-          float psi_acc = 0.f;
-#pragma unroll
-          for (int cb = 0; cb < NPAD; cb += 32) {
-            float acc[32];
-            tmem_ld32(tbase + t * NPAD + cb, acc);
-            if (masked) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (key >= vis_s[cb + c]) acc[c] = kEmptyMax;
+          const bool msk = key0 + kTilesPerPair * kTileKeys > all_bound;
+          const int key = key0 + et;
+          float lo, hi;
+          tmem_ld32_issue(tbase + t * NPAD, ra);
+          tmem_ld_wait(ra, ra);
+          if (msk) mask_slab(ra, key, vis_s);
+          if constexpr (NPAD == 32) {
+            unpack2(exp_sum(ra, scale2x, neglse2, 0ull), lo, hi);
+            if (key < p.n_max) psi[key] = (key < n) ? lo + hi : 0.f;
+            if (two) {
+              tmem_ld32_issue(tbase + t * NPAD + 32, ra);
+              tmem_ld_wait(ra, ra);
+              if (msk) mask_slab(ra, key + kTileKeys, vis_s);
+              unpack2(exp_sum(ra, scale2x, neglse2, 0ull), lo, hi);
+              if (key + kTileKeys < p.n_max) psi[key + kTileKeys] = (key + kTileKeys < n) ? lo + hi : 0.f;
             }
-#pragma unroll
-            for (int c = 0; c < 32; ++c) psi_acc += ex2(fmaf(acc[c], p.scale2, -lse_r[cb + c]));
+          } else {
+            const uint64_t part = exp_sum(ra, scale2x, neglse2, 0ull);
+            tmem_ld32_issue(tbase + t * NPAD + 32, ra);
+            tmem_ld_wait(ra, ra);
+            if (msk) mask_slab(ra, key, vis_s + 32);
+            unpack2(exp_sum(ra, scale2x, neglse2 + 16, part), lo, hi);
+            if (key < p.n_max) psi[key] = (key < n) ? lo + hi : 0.f;
           }
-          if (key < p.n_max) psi[key] = (key < n) ? psi_acc : 0.f;
+        }
+        for (int t = nt; t < kItemTiles; ++t) {  // tiles beyond the sequence
+          const int key = key_begin + t * kTileKeys + et;
+          if (key < p.n_max) psi[key] = 0.f;
         }
         if (!ok) break;
         tc_fence_before();
@@ -699,7 +826,8 @@ int launch_score_tc(const madakv_config& c, const void* q, madakv_strides sq, co
   p.w = c.window;
   p.R = g * c.window;
   p.n_max = c.max_seq_len;
-  p.cpu = wl.score_tc_chunks;
+  const int item_keys = kTileKeys * (kItemCols / (p.R <= 32 ? 32 : 64));
+  p.cpu = (c.max_seq_len + item_keys - 1) / item_keys;
   p.causal = c.causal;
   p.scale2 = scale_of(c) * kLog2e;
   const int npad = p.R <= 32 ? 32 : 64;
