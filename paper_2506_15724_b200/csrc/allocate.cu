@@ -5,7 +5,7 @@
 // results do not depend on the order of summation or on the launch shape. Eq. 9 is a "top-p" count: a 4-pass
 // radix descent over the order-preserving bit pattern of psi with per-bucket (count, mass) histograms in shared
 // memory finds the bucket in which the descending prefix mass reaches theta * W_m; ties inside the final bucket
-// share one value, so the remaining count is a division. The layer recurrence is a scalar fp64 scan per sequence
+// share one value, so the remaining count is a division. The keys of a unit sit in registers between passes. The layer recurrence is a scalar fp64 scan per sequence
 // with explicitly rounded operations (no FMA contraction), so it is reproducible bit for bit.
 #include "common.cuh"
 
@@ -13,8 +13,10 @@ namespace madakv {
 namespace {
 
 typedef unsigned long long u64;
-typedef unsigned __int128 u128;
 constexpr int NT = 512;
+constexpr int KPT = 16;            // keys a thread holds in registers per round
+constexpr int ROUND = NT * KPT;    // keys a block takes per round
+constexpr unsigned int kFull = 0xffffffffu;
 
 struct AllocParams {
   const float* psi;
@@ -30,111 +32,243 @@ struct AllocParams {
   u64 theta_fix;  // floor(theta * 2^32)
 };
 
-__device__ __forceinline__ u64 block_sum_u64(u64 v, u64* scratch /*[NT/32]*/) {
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
-  __syncthreads();
-  u64 t = 0;
-  for (int i = 0; i < NT / 32; ++i) t += scratch[i];
-  return t;
+// Shared histograms of one radix pass: per (modality, digit) a count and an exact 64-bit mass kept as two 32-bit
+// words (32-bit shared atomics are native; the carry of the low word is detected from the value the atomic returns).
+struct Hist {
+  unsigned int cnt[512], mlo[512], mhi[512];
+};
+__device__ __forceinline__ void hist_atomic(Hist& h, int bucket, unsigned int c, u64 m) {
+  atomicAdd(&h.cnt[bucket], c);
+  const unsigned int add = (unsigned int)m;
+  const unsigned int old = atomicAdd(&h.mlo[bucket], add);
+  atomicAdd(&h.mhi[bucket], (unsigned int)(m >> 32) + ((unsigned int)(old + add) < old ? 1u : 0u));
+}
+__device__ __forceinline__ u64 hist_mass(const Hist& h, int bucket) {
+  return ((u64)h.mhi[bucket] << 32) | h.mlo[bucket];
 }
 
-__global__ void __launch_bounds__(NT) alloc_unit_kernel(AllocParams p) {
-  __shared__ unsigned int cnt[2][256];
-  __shared__ u64 msum[2][256];
-  __shared__ u64 scratch[NT / 32];
+// A lane's private accumulator for one bucket (see hist_add).
+struct Slot {
+  int tag;
+  unsigned int cnt;
+  u64 mass;
+};
+__device__ __forceinline__ void slot_flush(Hist& h, Slot& s) {
+  if (s.tag >= 0) hist_atomic(h, s.tag, s.cnt, s.mass);
+  s.tag = -1;
+  s.cnt = 0;
+  s.mass = 0;
+}
+
+// Adds one (bucket, fixed-point mass) sample per lane to the histograms; every lane of the warp calls it, a lane
+// without a sample passes bucket = -1. Importance values cluster in a few exponent buckets, where per-lane
+// atomics would serialise. So when the first sample's bucket is shared by several lanes, up to four rounds each
+// take one distinct bucket off the warp: its lanes are counted by a ballot, their masses summed by full-warp
+// reductions (three 22-bit pieces, so a sum of 32 stays below 2^32), and the result is added to a register
+// accumulator that one lane keeps for that bucket; the accumulator goes to shared memory only when its lane
+// meets another bucket or the pass ends. Whatever is left uses shared atomics directly.
+__device__ __forceinline__ void hist_add(Hist& h, Slot& slot, int bucket, u64 f) {
+  const int lane = threadIdx.x & 31;
+  unsigned int todo = __ballot_sync(kFull, bucket >= 0);
+  if (todo == 0) return;
+  int b = __shfl_sync(kFull, bucket, __ffs(todo) - 1);
+  unsigned int peers = __ballot_sync(kFull, bucket == b);
+  if (__popc(peers) >= 4) {
+    for (int it = 0;; ++it) {
+      const bool mine = bucket == b;
+      const u64 fm = mine ? f : 0ull;
+      const unsigned int s0 = __reduce_add_sync(kFull, (unsigned int)(fm & 0x3fffffu));
+      const unsigned int s1 = __reduce_add_sync(kFull, (unsigned int)((fm >> 22) & 0x3fffffu));
+      u64 tot = (u64)s0 + ((u64)s1 << 22);
+      if (__any_sync(kFull, (fm >> 44) != 0)) tot += (u64)__reduce_add_sync(kFull, (unsigned int)(fm >> 44)) << 44;
+      if (lane == (((b & 255) + 13 * (b >> 8)) & 31)) {
+        if (slot.tag != b) {
+          slot_flush(h, slot);
+          slot.tag = b;
+        }
+        slot.cnt += (unsigned int)__popc(peers);
+        slot.mass += tot;
+      }
+      if (mine) bucket = -1;
+      todo &= ~peers;
+      if (todo == 0 || it == 3) break;
+      b = __shfl_sync(kFull, bucket, __ffs(todo) - 1);
+      peers = __ballot_sync(kFull, bucket == b);
+    }
+  }
+  if (bucket >= 0) hist_atomic(h, bucket, 1u, f);
+}
+
+// One warp walks the 256 buckets of modality m from the top: the first bucket at which the running mass
+// `above + mass[dig]` reaches need_c is the one the threshold falls into (bucket 0 if none does). Lane j owns
+// buckets 8j..8j+7; a warp suffix scan supplies what lies above them. Returns the bucket, and updates above /
+// above_c to the mass / count strictly above it (identical in every lane).
+__device__ __forceinline__ int descend(const Hist& h, int m, u64 need_c, u64& above, unsigned int& above_c,
+                                       unsigned int& cnt_at) {
+  const int lane = threadIdx.x & 31;
+  u64 ms[8], lm = 0;
+  unsigned int cs[8], lc = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    ms[j] = hist_mass(h, m * 256 + lane * 8 + j);
+    cs[j] = h.cnt[m * 256 + lane * 8 + j];
+    lm += ms[j];
+    lc += cs[j];
+  }
+  u64 sm = lm;
+  unsigned int sc = lc;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const u64 tm = __shfl_down_sync(kFull, sm, off);
+    const unsigned int tc = __shfl_down_sync(kFull, sc, off);
+    if (lane + off < 32) {
+      sm += tm;
+      sc += tc;
+    }
+  }
+  u64 a = above + (sm - lm);
+  unsigned int ac = above_c + (sc - lc);
+  int found = -1;
+  unsigned int c_at = 0;
+#pragma unroll
+  for (int j = 7; j >= 0; --j) {
+    if (found < 0) {
+      if (a + ms[j] >= need_c || (lane == 0 && j == 0)) {
+        found = j;
+        c_at = cs[j];
+      } else {
+        a += ms[j];
+        ac += cs[j];
+      }
+    }
+  }
+  const unsigned int hit = __ballot_sync(kFull, found >= 0);  // lane 0 always hits
+  const int win = 31 - __clz(hit);
+  above = __shfl_sync(kFull, a, win);
+  above_c = __shfl_sync(kFull, ac, win);
+  cnt_at = __shfl_sync(kFull, c_at, win);
+  return win * 8 + __shfl_sync(kFull, found, win);
+}
+
+// One block per unit. A thread keeps KPT keys in registers (loaded once when the sequence fits one round, else
+// re-read from L2 every pass), so a pass costs no dependent global loads.
+__global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
+  __shared__ Hist hist;
   __shared__ uint32_t s_prefix[2];
-  __shared__ u64 s_above_mass[2];
-  __shared__ unsigned int s_above_cnt[2];
   __shared__ int s_done[2];
+  __shared__ u64 s_W[2];
 
   const int u = blockIdx.x;
   const int b = u / (p.Hkv * p.L);
   const int n = min(p.seq_len[b], p.n_max);
   const float* psi = p.psi + (int64_t)u * p.n_max;
   const uint8_t* mask = p.mask + (int64_t)b * p.n_max;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rounds = (n + ROUND - 1) / ROUND;
 
-  // Eq. 6: W_v, W_t
-  u64 wv = 0, wt = 0;
-  for (int i = threadIdx.x; i < n; i += NT) {
-    const u64 f = psi_fix(psi_key(psi[i]));
-    if (mask[i]) wv += f; else wt += f;
-  }
-  const u64 W[2] = {block_sum_u64(wv, scratch), block_sum_u64(wt, scratch)};
-  const u128 need[2] = {(u128)p.theta_fix * W[0], (u128)p.theta_fix * W[1]};
+  uint32_t key[KPT];
+  uint32_t flags = 0;  // bit j: key j exists; bit 16 + j: key j is a visual token
+  Slot slot;
+  slot.tag = -1;
+  slot.cnt = 0;
+  slot.mass = 0;
 
-  if (threadIdx.x < 2) {
-    s_prefix[threadIdx.x] = 0;
-    s_above_mass[threadIdx.x] = 0;
-    s_above_cnt[threadIdx.x] = 0;
-    s_done[threadIdx.x] = (need[threadIdx.x] == 0);
-  }
-  if (threadIdx.x == 0) {
-    const u64 tot = W[0] + W[1];
-    p.mass[(int64_t)u * 2 + 0] = __ull2double_rn(W[0]) / 4294967296.0;
-    p.mass[(int64_t)u * 2 + 1] = __ull2double_rn(W[1]) / 4294967296.0;
-    p.pref[(int64_t)u * 2 + 0] = tot ? __ddiv_rn(__ull2double_rn(W[0]), __ull2double_rn(tot)) : 0.0;
-    p.pref[(int64_t)u * 2 + 1] = tot ? __ddiv_rn(__ull2double_rn(W[1]), __ull2double_rn(tot)) : 0.0;
-  }
-  __syncthreads();
+  // state of the descent, kept by warp m (all lanes alike) for modality m
+  u64 need_c = 0, above = 0;
+  unsigned int above_c = 0;
 
-  // Eq. 9: radix descent, both modalities at once
+  // Eq. 9: radix descent, both modalities at once. Pass 0 sees every key, so its histogram also yields the
+  // modality masses W_v, W_t of Eq. 6.
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
     for (int x = threadIdx.x; x < 512; x += NT) {
-      (&cnt[0][0])[x] = 0;
-      (&msum[0][0])[x] = 0;
+      hist.cnt[x] = 0;
+      hist.mlo[x] = 0;
+      hist.mhi[x] = 0;
     }
     __syncthreads();
-    const uint32_t pre0 = s_prefix[0], pre1 = s_prefix[1];
-    const bool act0 = !s_done[0], act1 = !s_done[1];
-    for (int i = threadIdx.x; i < n; i += NT) {
-      const uint32_t key = psi_key(psi[i]);
-      const int m = mask[i] ? 0 : 1;
-      if ((m == 0 ? act0 : act1) && (key & himask) == (m == 0 ? pre0 : pre1)) {
-        const int dig = (key >> shift) & 255;
-        atomicAdd(&cnt[m][dig], 1u);
-        atomicAdd(&msum[m][dig], psi_fix(key));
-      }
-    }
-    __syncthreads();
-    if (threadIdx.x < 2 && !s_done[threadIdx.x]) {
-      const int m = threadIdx.x;
-      u64 above = s_above_mass[m];
-      unsigned int above_c = s_above_cnt[m];
-      int dig = 255;
-      for (; dig > 0; --dig) {
-        if (((u128)(above + msum[m][dig]) << 32) >= need[m]) break;
-        above += msum[m][dig];
-        above_c += cnt[m][dig];
-      }
-      s_above_mass[m] = above;
-      s_above_cnt[m] = above_c;
-      s_prefix[m] |= (uint32_t)dig << shift;
-      if (pass == 3) {
-        // every key in the final bucket has the same value: take as few of them as reach the threshold
-        const u64 each = psi_fix(s_prefix[m]);
-        unsigned int take = cnt[m][dig];
-        if (each > 0) {
-          const u128 rest = need[m] - ((u128)above << 32);
-          const u128 per = (u128)each << 32;
-          const u128 t = (rest + per - 1) / per;
-          if (t < (u128)take) take = (unsigned int)t;
+    const uint32_t pre0 = pass ? s_prefix[0] : 0u, pre1 = pass ? s_prefix[1] : 0u;
+    const bool act0 = pass == 0 || !s_done[0], act1 = pass == 0 || !s_done[1];
+    if (act0 || act1) {
+      for (int r = 0; r < rounds; ++r) {
+        if (pass == 0 || rounds > 1) {
+          flags = 0;
+#pragma unroll
+          for (int j = 0; j < KPT; ++j) {
+            const int i = r * ROUND + j * NT + (int)threadIdx.x;
+            key[j] = 0;
+            if (i < n) {
+              key[j] = psi_key(__ldg(psi + i));
+              flags |= (1u << j) | (__ldg(mask + i) ? (0x10000u << j) : 0u);
+            }
+          }
         }
-        p.demand[(int64_t)u * 2 + m] = (int32_t)(above_c + take);
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+          int bucket = -1;
+          u64 f = 0;
+          const int m = (flags >> (16 + j)) & 1u ? 0 : 1;
+          if (((flags >> j) & 1u) && (m == 0 ? act0 : act1) && (key[j] & himask) == (m == 0 ? pre0 : pre1)) {
+            bucket = m * 256 + (int)((key[j] >> shift) & 255u);
+            f = psi_fix(key[j]);
+          }
+          hist_add(hist, slot, bucket, f);
+        }
+      }
+      slot_flush(hist, slot);
+    }
+    __syncthreads();
+    if (warp < 2) {
+      const int m = warp;
+      if (pass == 0) {
+        u64 wsum = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) wsum += hist_mass(hist, m * 256 + lane * 8 + j);
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) wsum += __shfl_xor_sync(kFull, wsum, off);
+        const u64 W = wsum;
+        // need = theta_fix * W (96 bits); the prefix test  prefix * 2^32 >= need  is  prefix >= ceil(need / 2^32)
+        const u64 hi = __umul64hi(p.theta_fix, W), lo = p.theta_fix * W;
+        need_c = (hi << 32) + (lo >> 32) + ((lo & 0xffffffffull) ? 1ull : 0ull);
+        if (lane == 0) {
+          s_prefix[m] = 0;
+          s_done[m] = (need_c == 0);
+          s_W[m] = W;
+          p.mass[(int64_t)u * 2 + m] = __ull2double_rn(W) / 4294967296.0;
+          if (need_c == 0) p.demand[(int64_t)u * 2 + m] = 0;
+        }
+      }
+      __syncwarp();
+      if (need_c != 0) {
+        unsigned int c_at = 0;
+        const int dig = descend(hist, m, need_c, above, above_c, c_at);
+        if (lane == 0) s_prefix[m] |= (uint32_t)dig << shift;
+        if (pass == 3 && lane == 0) {
+          // every key in the final bucket has the same value: take as few of them as reach the threshold
+          const u64 each = psi_fix(s_prefix[m]);
+          unsigned int take = c_at;
+          if (each > 0) {
+            const u64 t = (need_c - above + each - 1) / each;
+            if (t < (u64)take) take = (unsigned int)t;
+          }
+          p.demand[(int64_t)u * 2 + m] = (int32_t)(above_c + take);
+        }
       }
     }
     __syncthreads();
+    if (pass == 0 && threadIdx.x == 0) {
+      const u64 W0 = s_W[0], W1 = s_W[1], tot = W0 + W1;
+      p.pref[(int64_t)u * 2 + 0] = tot ? __ddiv_rn(__ull2double_rn(W0), __ull2double_rn(tot)) : 0.0;
+      p.pref[(int64_t)u * 2 + 1] = tot ? __ddiv_rn(__ull2double_rn(W1), __ull2double_rn(tot)) : 0.0;
+    }
   }
-  if (threadIdx.x < 2 && need[threadIdx.x] == 0) p.demand[(int64_t)u * 2 + threadIdx.x] = 0;
 }
 
 // One block per sequence: Eq. 10-11 as a scalar scan over layers, then Eq. 8 integerised for every (layer, head).
 __global__ void alloc_seq_kernel(AllocParams p) {
-  extern __shared__ double s_Phi[];  // [L]
+  extern __shared__ double s_Phi[];  // [L] rounded budgets, then [L] demand sums (as long long)
+  long long* s_dem = reinterpret_cast<long long*>(s_Phi + p.L);
   __shared__ int s_nv;
   const int b = blockIdx.x;
   const int n = min(p.seq_len[b], p.n_max);
@@ -142,7 +276,18 @@ __global__ void alloc_seq_kernel(AllocParams p) {
   __syncthreads();
   int c = 0;
   for (int i = threadIdx.x; i < n; i += blockDim.x) c += p.mask[(int64_t)b * p.n_max + i] ? 1 : 0;
-  atomicAdd(&s_nv, c);
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
+  if ((threadIdx.x & 31) == 0 && c) atomicAdd(&s_nv, c);
+  // Eq. 10's sum over heads, one warp per layer (integers: any order gives the same sum)
+  for (int l = threadIdx.x >> 5; l < p.L; l += blockDim.x >> 5) {
+    long long dem = 0;
+    for (int x = threadIdx.x & 31; x < 2 * p.Hkv; x += 32)
+      dem += (long long)p.demand[((int64_t)b * p.L + l) * p.Hkv * 2 + x];
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) dem += __shfl_xor_sync(0xffffffffu, dem, off);
+    if ((threadIdx.x & 31) == 0) s_dem[l] = dem;
+  }
   __syncthreads();
   const int n_v = s_nv, n_t = n - n_v;
   if (threadIdx.x == 0) {
@@ -152,12 +297,7 @@ __global__ void alloc_seq_kernel(AllocParams p) {
       p.phi[(int64_t)b * p.L + (l - 1)] = ph;
       s_Phi[l - 1] = fmin(fmax(floor(__dadd_rn(ph, 0.5)), lo), hi);
       if (l < p.L) {
-        long long dem = 0;
-        for (int h = 0; h < p.Hkv; ++h) {
-          const int64_t u = ((int64_t)b * p.L + (l - 1)) * p.Hkv + h;
-          dem += (long long)p.demand[u * 2] + p.demand[u * 2 + 1];
-        }
-        const double K = __dsub_rn((double)dem, __dmul_rn((double)p.Hkv, ph));  // Eq. 10
+        const double K = __dsub_rn((double)s_dem[l - 1], __dmul_rn((double)p.Hkv, ph));  // Eq. 10
         double next = ph;
         if (p.hcc_mode == MADAKV_HCC_PAPER)
           next = __dsub_rn(ph, __ddiv_rn(K, (double)((long long)p.Hkv * (p.L - l))));  // Eq. 11, per-head units
@@ -212,7 +352,7 @@ int launch_allocate(const madakv_config& c, const float* psi, const uint8_t* mas
   p.theta_fix = (u64)((double)c.theta * 4294967296.0);
   const int units = c.batch * c.n_layers * c.n_kv_heads;
   alloc_unit_kernel<<<units, NT, 0, st>>>(p);
-  alloc_seq_kernel<<<c.batch, 256, c.n_layers * sizeof(double), st>>>(p);
+  alloc_seq_kernel<<<c.batch, 256, c.n_layers * (sizeof(double) + sizeof(long long)), st>>>(p);
   return launch_status();
 }
 

@@ -127,28 +127,56 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
   }
   // radix select: after the 4 passes s_prefix[m] is the want[m]-th largest key of modality m (if that many exist)
   // and s_above[m] counts the keys strictly above it
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_round = (n + 31) & ~31;  // whole warps run every iteration (the match below is a warp-wide call)
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
     for (int x = threadIdx.x; x < 512; x += NT) (&cnt[0][0])[x] = 0;
     __syncthreads();
     const uint32_t pre0 = s_prefix[0], pre1 = s_prefix[1];
-    for (int i = threadIdx.x; i < n; i += NT) {
-      const uint32_t key = psi_key(psi[i]);
-      const int m = (p.mpa && mask[i]) ? 0 : 1;
-      if ((key & himask) == (m == 0 ? pre0 : pre1)) atomicAdd(&cnt[m][(key >> shift) & 255], 1u);
+    for (int i = threadIdx.x; i < n_round; i += NT) {
+      int bucket = -1;
+      if (i < n) {
+        const uint32_t key = psi_key(psi[i]);
+        const int m = (p.mpa && mask[i]) ? 0 : 1;
+        if ((key & himask) == (m == 0 ? pre0 : pre1)) bucket = m * 256 + (int)((key >> shift) & 255u);
+      }
+      // lanes that hit the same bucket are counted by one of them: importance values cluster in a few exponent
+      // buckets, and per-lane atomics on them would serialise
+      const unsigned int peers = __match_any_sync(0xffffffffu, bucket);
+      if (bucket >= 0 && lane == __ffs(peers) - 1) atomicAdd(&(&cnt[0][0])[bucket], (unsigned int)__popc(peers));
     }
     __syncthreads();
-    if (threadIdx.x < 2) {
-      const int m = threadIdx.x;
-      unsigned int above = s_above[m];
-      int dig = 255;
-      for (; dig > 0; --dig) {
-        if (above + cnt[m][dig] >= (unsigned int)want[m]) break;
-        above += cnt[m][dig];
+    if (warp < 2) {
+      // warp m walks modality m's buckets from the top; lane j owns buckets 8j..8j+7
+      const int m = warp;
+      unsigned int cs[8], lc = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        cs[j] = cnt[m][lane * 8 + j];
+        lc += cs[j];
       }
-      s_above[m] = above;
-      s_prefix[m] |= (uint32_t)dig << shift;
+      unsigned int sc = lc;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int t = __shfl_down_sync(0xffffffffu, sc, off);
+        if (lane + off < 32) sc += t;
+      }
+      unsigned int above = s_above[m] + (sc - lc);
+      int found = -1;
+#pragma unroll
+      for (int j = 7; j >= 0; --j) {
+        if (found < 0) {
+          if (above + cs[j] >= (unsigned int)want[m] || (lane == 0 && j == 0)) found = j;
+          else above += cs[j];
+        }
+      }
+      const unsigned int hit = __ballot_sync(0xffffffffu, found >= 0);  // lane 0 always hits
+      if (lane == 31 - __clz(hit)) {
+        s_above[m] = above;
+        s_prefix[m] |= (uint32_t)(lane * 8 + found) << shift;
+      }
     }
     __syncthreads();
   }
