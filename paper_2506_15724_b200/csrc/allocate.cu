@@ -37,8 +37,8 @@ struct AllocParams {
 struct Hist {
   unsigned int cnt[512], mlo[512], mhi[512];
 };
-__device__ __forceinline__ void hist_atomic(Hist& h, int bucket, unsigned int c, u64 m) {
-  atomicAdd(&h.cnt[bucket], c);
+__device__ __forceinline__ void hist_add(Hist& h, int bucket, u64 m) {
+  atomicAdd(&h.cnt[bucket], 1u);
   const unsigned int add = (unsigned int)m;
   const unsigned int old = atomicAdd(&h.mlo[bucket], add);
   atomicAdd(&h.mhi[bucket], (unsigned int)(m >> 32) + ((unsigned int)(old + add) < old ? 1u : 0u));
@@ -47,62 +47,11 @@ __device__ __forceinline__ u64 hist_mass(const Hist& h, int bucket) {
   return ((u64)h.mhi[bucket] << 32) | h.mlo[bucket];
 }
 
-// A lane's private accumulator for one bucket (see hist_add).
-struct Slot {
-  int tag;
-  unsigned int cnt;
-  u64 mass;
-};
-__device__ __forceinline__ void slot_flush(Hist& h, Slot& s) {
-  if (s.tag >= 0) hist_atomic(h, s.tag, s.cnt, s.mass);
-  s.tag = -1;
-  s.cnt = 0;
-  s.mass = 0;
-}
-
-// Adds one (bucket, fixed-point mass) sample per lane to the histograms; every lane of the warp calls it, a lane
-// without a sample passes bucket = -1. Importance values cluster in a few exponent buckets, where per-lane
-// atomics would serialise. So when the first sample's bucket is shared by several lanes, up to four rounds each
-// take one distinct bucket off the warp: its lanes are counted by a ballot, their masses summed by full-warp
-// reductions (three 22-bit pieces, so a sum of 32 stays below 2^32), and the result is added to a register
-// accumulator that one lane keeps for that bucket; the accumulator goes to shared memory only when its lane
-// meets another bucket or the pass ends. Whatever is left uses shared atomics directly.
-__device__ __forceinline__ void hist_add(Hist& h, Slot& slot, int bucket, u64 f) {
-  const int lane = threadIdx.x & 31;
-  unsigned int todo = __ballot_sync(kFull, bucket >= 0);
-  if (todo == 0) return;
-  int b = __shfl_sync(kFull, bucket, __ffs(todo) - 1);
-  unsigned int peers = __ballot_sync(kFull, bucket == b);
-  if (__popc(peers) >= 4) {
-    for (int it = 0;; ++it) {
-      const bool mine = bucket == b;
-      const u64 fm = mine ? f : 0ull;
-      const unsigned int s0 = __reduce_add_sync(kFull, (unsigned int)(fm & 0x3fffffu));
-      const unsigned int s1 = __reduce_add_sync(kFull, (unsigned int)((fm >> 22) & 0x3fffffu));
-      u64 tot = (u64)s0 + ((u64)s1 << 22);
-      if (__any_sync(kFull, (fm >> 44) != 0)) tot += (u64)__reduce_add_sync(kFull, (unsigned int)(fm >> 44)) << 44;
-      if (lane == (((b & 255) + 13 * (b >> 8)) & 31)) {
-        if (slot.tag != b) {
-          slot_flush(h, slot);
-          slot.tag = b;
-        }
-        slot.cnt += (unsigned int)__popc(peers);
-        slot.mass += tot;
-      }
-      if (mine) bucket = -1;
-      todo &= ~peers;
-      if (todo == 0 || it == 3) break;
-      b = __shfl_sync(kFull, bucket, __ffs(todo) - 1);
-      peers = __ballot_sync(kFull, bucket == b);
-    }
-  }
-  if (bucket >= 0) hist_atomic(h, bucket, 1u, f);
-}
-
-// One warp walks the 256 buckets of modality m from the top: the first bucket at which the running mass
-// `above + mass[dig]` reaches need_c is the one the threshold falls into (bucket 0 if none does). Lane j owns
-// buckets 8j..8j+7; a warp suffix scan supplies what lies above them. Returns the bucket, and updates above /
-// above_c to the mass / count strictly above it (identical in every lane).
+// One warp walks the 256 buckets of modality m in ascending digit order (digits are taken from kmax - key, so this
+// is descending importance): the first bucket at which the running mass `above + mass[dig]` reaches need_c is the
+// one the threshold falls into (the last bucket if none does). Lane j owns buckets 8j..8j+7; a warp prefix scan
+// supplies what lies before them. Returns the bucket, and updates above / above_c to the mass / count strictly
+// before it (identical in every lane).
 __device__ __forceinline__ int descend(const Hist& h, int m, u64 need_c, u64& above, unsigned int& above_c,
                                        unsigned int& cnt_at) {
   const int lane = threadIdx.x & 31;
@@ -119,9 +68,9 @@ __device__ __forceinline__ int descend(const Hist& h, int m, u64 need_c, u64& ab
   unsigned int sc = lc;
 #pragma unroll
   for (int off = 1; off < 32; off <<= 1) {
-    const u64 tm = __shfl_down_sync(kFull, sm, off);
-    const unsigned int tc = __shfl_down_sync(kFull, sc, off);
-    if (lane + off < 32) {
+    const u64 tm = __shfl_up_sync(kFull, sm, off);
+    const unsigned int tc = __shfl_up_sync(kFull, sc, off);
+    if (lane >= off) {
       sm += tm;
       sc += tc;
     }
@@ -131,9 +80,9 @@ __device__ __forceinline__ int descend(const Hist& h, int m, u64 need_c, u64& ab
   int found = -1;
   unsigned int c_at = 0;
 #pragma unroll
-  for (int j = 7; j >= 0; --j) {
+  for (int j = 0; j < 8; ++j) {
     if (found < 0) {
-      if (a + ms[j] >= need_c || (lane == 0 && j == 0)) {
+      if (a + ms[j] >= need_c || (lane == 31 && j == 7)) {
         found = j;
         c_at = cs[j];
       } else {
@@ -142,8 +91,8 @@ __device__ __forceinline__ int descend(const Hist& h, int m, u64 need_c, u64& ab
       }
     }
   }
-  const unsigned int hit = __ballot_sync(kFull, found >= 0);  // lane 0 always hits
-  const int win = 31 - __clz(hit);
+  const unsigned int hit = __ballot_sync(kFull, found >= 0);  // lane 31 always hits
+  const int win = __ffs(hit) - 1;
   above = __shfl_sync(kFull, a, win);
   above_c = __shfl_sync(kFull, ac, win);
   cnt_at = __shfl_sync(kFull, c_at, win);
@@ -152,11 +101,17 @@ __device__ __forceinline__ int descend(const Hist& h, int m, u64 need_c, u64& ab
 
 // One block per unit. A thread keeps KPT keys in registers (loaded once when the sequence fits one round, else
 // re-read from L2 every pass), so a pass costs no dependent global loads.
+//
+// The radix digits are not taken from the key itself but from t = kmax - key, starting at the highest bit in which
+// the unit's keys differ (kmax, kmin: largest and smallest key of the unit). Importance values share their sign and
+// most exponent bits, so digits of the raw key would put nearly all keys into a handful of buckets and serialise
+// the shared atomics; the digits of t spread them over the whole histogram. Ascending t is descending importance.
 __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
   __shared__ Hist hist;
   __shared__ uint32_t s_prefix[2];
   __shared__ int s_done[2];
   __shared__ u64 s_W[2];
+  __shared__ uint32_t s_red[2][NT / 32];
 
   const int u = blockIdx.x;
   const int b = u / (p.Hkv * p.L);
@@ -168,20 +123,59 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
 
   uint32_t key[KPT];
   uint32_t flags = 0;  // bit j: key j exists; bit 16 + j: key j is a visual token
-  Slot slot;
-  slot.tag = -1;
-  slot.cnt = 0;
-  slot.mass = 0;
+  auto load_round = [&](int r) {
+    flags = 0;
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+      const int i = r * ROUND + j * NT + (int)threadIdx.x;
+      key[j] = 0;
+      if (i < n) {
+        key[j] = psi_key(__ldg(psi + i));
+        flags |= (1u << j) | (__ldg(mask + i) ? (0x10000u << j) : 0u);
+      }
+    }
+  };
+
+  // range of the unit's keys
+  uint32_t kmax = 0, kmin = 0xffffffffu;
+  for (int r = 0; r < rounds; ++r) {
+    load_round(r);
+#pragma unroll
+    for (int j = 0; j < KPT; ++j)
+      if ((flags >> j) & 1u) {
+        kmax = max(kmax, key[j]);
+        kmin = min(kmin, key[j]);
+      }
+  }
+  kmax = __reduce_max_sync(kFull, kmax);
+  kmin = __reduce_min_sync(kFull, kmin);
+  if (lane == 0) {
+    s_red[0][warp] = kmax;
+    s_red[1][warp] = kmin;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < NT / 32; ++i) {
+    kmax = max(kmax, s_red[0][i]);
+    kmin = min(kmin, s_red[1][i]);
+  }
+  if (kmin > kmax) kmin = kmax;  // no keys at all
+  // significant bits of t = kmax - key; at least one pass always runs (it also yields the masses of Eq. 6)
+  const int top = max(32 - __clz(kmax - kmin), 1);
+  if (rounds == 1) {
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
+  }
 
   // state of the descent, kept by warp m (all lanes alike) for modality m
   u64 need_c = 0, above = 0;
   unsigned int above_c = 0;
 
-  // Eq. 9: radix descent, both modalities at once. Pass 0 sees every key, so its histogram also yields the
-  // modality masses W_v, W_t of Eq. 6.
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+  // Eq. 9: radix descent, both modalities at once. The first pass sees every key, so its histogram also yields the
+  // modality masses W_v, W_t of Eq. 6. `rem` counts the bits of t not yet resolved.
+  for (int rem = top, pass = 0; rem > 0; ++pass) {
+    const int bits = min(rem, 8), shift = rem - bits;
+    const uint32_t dmask = (1u << bits) - 1u;
     for (int x = threadIdx.x; x < 512; x += NT) {
       hist.cnt[x] = 0;
       hist.mlo[x] = 0;
@@ -192,31 +186,18 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
     const bool act0 = pass == 0 || !s_done[0], act1 = pass == 0 || !s_done[1];
     if (act0 || act1) {
       for (int r = 0; r < rounds; ++r) {
-        if (pass == 0 || rounds > 1) {
-          flags = 0;
+        if (rounds > 1) {
+          load_round(r);
 #pragma unroll
-          for (int j = 0; j < KPT; ++j) {
-            const int i = r * ROUND + j * NT + (int)threadIdx.x;
-            key[j] = 0;
-            if (i < n) {
-              key[j] = psi_key(__ldg(psi + i));
-              flags |= (1u << j) | (__ldg(mask + i) ? (0x10000u << j) : 0u);
-            }
-          }
+          for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
         }
 #pragma unroll
         for (int j = 0; j < KPT; ++j) {
-          int bucket = -1;
-          u64 f = 0;
           const int m = (flags >> (16 + j)) & 1u ? 0 : 1;
-          if (((flags >> j) & 1u) && (m == 0 ? act0 : act1) && (key[j] & himask) == (m == 0 ? pre0 : pre1)) {
-            bucket = m * 256 + (int)((key[j] >> shift) & 255u);
-            f = psi_fix(key[j]);
-          }
-          hist_add(hist, slot, bucket, f);
+          if (((flags >> j) & 1u) && (m == 0 ? act0 : act1) && (key[j] >> rem) == (m == 0 ? pre0 : pre1))
+            hist_add(hist, m * 256 + (int)((key[j] >> shift) & dmask), psi_fix(kmax - key[j]));
         }
       }
-      slot_flush(hist, slot);
     }
     __syncthreads();
     if (warp < 2) {
@@ -242,17 +223,21 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
       __syncwarp();
       if (need_c != 0) {
         unsigned int c_at = 0;
-        const int dig = descend(hist, m, need_c, above, above_c, c_at);
-        if (lane == 0) s_prefix[m] |= (uint32_t)dig << shift;
-        if (pass == 3 && lane == 0) {
-          // every key in the final bucket has the same value: take as few of them as reach the threshold
-          const u64 each = psi_fix(s_prefix[m]);
-          unsigned int take = c_at;
-          if (each > 0) {
-            const u64 t = (need_c - above + each - 1) / each;
-            if (t < (u64)take) take = (unsigned int)t;
+        const int dig = min(descend(hist, m, need_c, above, above_c, c_at), (int)dmask);
+        if (lane == 0) {
+          const uint32_t prefix = (s_prefix[m] << bits) | (uint32_t)dig;
+          s_prefix[m] = prefix;
+          if (shift == 0) {
+            // t is resolved: every key in the final bucket has the value kmax - prefix; take as few of them as
+            // reach the threshold
+            const u64 each = psi_fix(kmax - prefix);
+            unsigned int take = c_at;
+            if (each > 0) {
+              const u64 t = (need_c - above + each - 1) / each;
+              if (t < (u64)take) take = (unsigned int)t;
+            }
+            p.demand[(int64_t)u * 2 + m] = (int32_t)(above_c + take);
           }
-          p.demand[(int64_t)u * 2 + m] = (int32_t)(above_c + take);
         }
       }
     }
@@ -262,6 +247,7 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
       p.pref[(int64_t)u * 2 + 0] = tot ? __ddiv_rn(__ull2double_rn(W0), __ull2double_rn(tot)) : 0.0;
       p.pref[(int64_t)u * 2 + 1] = tot ? __ddiv_rn(__ull2double_rn(W1), __ull2double_rn(tot)) : 0.0;
     }
+    rem = shift;
   }
 }
 

@@ -1,10 +1,13 @@
 // Stage 4a: per-head, per-modality top-budget selection (Section 3.3, the eviction step after Eq. 8).
 //
-//   seg_scan     one block: kept_len[u] = b_v + b_t and the exclusive scan seg_off (rows, with headroom)
+//   seg_scan     one block: visual-token count of every sequence, kept_len[u] = b_v + b_t and the exclusive scan
+//                seg_off (rows, with headroom)
 //   select_unit  one block per unit: a 4-pass shared-memory radix select over the order-preserving bit pattern of
 //                psi finds, for both modalities at once, the budget-th largest value and how many of its ties are
 //                still needed; an ordered sweep then emits the kept positions in ascending order, giving ties to
 //                the lowest positions (block-wide prefix scans provide the tie ranks and the output slots).
+//                A thread owns KPT consecutive positions and keeps their keys in registers from the first pass to
+//                the sweep (sequences longer than one chunk are re-read from L2 chunk by chunk).
 // Integer work only: results are bit-exact functions of (psi bits, mask, budgets).
 #include "common.cuh"
 
@@ -12,8 +15,9 @@ namespace madakv {
 namespace {
 
 constexpr int NT = 256;
-constexpr int ITEMS = 4;               // positions per thread per sweep step
-constexpr int STEP = NT * ITEMS;       // 1024 positions per sweep step
+constexpr int KPT = 32;                // consecutive positions per thread
+constexpr int CHUNK = NT * KPT;        // 8192 positions per chunk
+constexpr unsigned int kFull = 0xffffffffu;
 
 struct SelParams {
   const float* psi;
@@ -26,31 +30,30 @@ struct SelParams {
   int64_t capacity;
   void* ws;
   int32_t* seq_nv;  // ws: visual-token count of every sequence
-  int units, L, Hkv, n_max, mpa, headroom;
+  int units, B, L, Hkv, n_max, mpa, headroom;
 };
-
-// One block per sequence: number of visual tokens among the first seq_len[b] positions.
-__global__ void __launch_bounds__(1024) count_visual_kernel(SelParams p) {
-  __shared__ int s_cnt;
-  const int b = blockIdx.x;
-  const int n = min(p.seq_len[b], p.n_max);
-  const uint8_t* mask = p.mask + (int64_t)b * p.n_max;
-  if (threadIdx.x == 0) s_cnt = 0;
-  __syncthreads();
-  int c = 0;
-  for (int i = threadIdx.x; i < n; i += 1024) c += mask[i] ? 1 : 0;
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
-  if ((threadIdx.x & 31) == 0) atomicAdd(&s_cnt, c);
-  __syncthreads();
-  if (threadIdx.x == 0) p.seq_nv[b] = p.mpa ? s_cnt : 0;
-}
 
 __global__ void __launch_bounds__(1024) seg_scan_kernel(SelParams p) {
   __shared__ long long warp_tot[32];
   __shared__ long long carry;
+  __shared__ int s_cnt;
+  // visual tokens among the first seq_len[b] positions of every sequence
+  for (int b = 0; b < p.B; ++b) {
+    const int n = min(p.seq_len[b], p.n_max);
+    const uint8_t* mask = p.mask + (int64_t)b * p.n_max;
+    if (threadIdx.x == 0) s_cnt = 0;
+    __syncthreads();
+    int c = 0;
+    if (p.mpa)
+      for (int i = threadIdx.x; i < n; i += 1024) c += mask[i] ? 1 : 0;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) c += __shfl_xor_sync(kFull, c, off);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(&s_cnt, c);
+    __syncthreads();
+    if (threadIdx.x == 0) p.seq_nv[b] = s_cnt;
+  }
   if (threadIdx.x == 0) carry = 0;
-  __syncthreads();
+  __syncthreads();  // also orders the seq_nv stores before the loads below (same block)
   for (int base = 0; base < p.units; base += 1024) {
     const int u = base + threadIdx.x;
     long long v = 0;
@@ -65,7 +68,7 @@ __global__ void __launch_bounds__(1024) seg_scan_kernel(SelParams p) {
     long long incl = v;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
-      const long long t = __shfl_up_sync(0xffffffffu, incl, off);
+      const long long t = __shfl_up_sync(kFull, incl, off);
       if ((threadIdx.x & 31) >= off) incl += t;
     }
     if ((threadIdx.x & 31) == 31) warp_tot[threadIdx.x >> 5] = incl;
@@ -84,12 +87,12 @@ __global__ void __launch_bounds__(1024) seg_scan_kernel(SelParams p) {
   }
 }
 
-// Exclusive block scan of a packed pair of 16-bit counters (each total <= STEP < 65536).
+// Exclusive block scan of a packed pair of 16-bit counters (each total <= CHUNK < 65536).
 __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* warp_tot, uint32_t* total) {
   uint32_t incl = v;
 #pragma unroll
   for (int off = 1; off < 32; off <<= 1) {
-    const uint32_t t = __shfl_up_sync(0xffffffffu, incl, off);
+    const uint32_t t = __shfl_up_sync(kFull, incl, off);
     if ((threadIdx.x & 31) >= off) incl += t;
   }
   __syncthreads();
@@ -106,11 +109,49 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* warp_t
   return wbase + incl - v;
 }
 
+template <bool kVec>
+__device__ __forceinline__ void load_chunk(const float* psi, const uint8_t* mask, int n, int pos0, int mpa,
+                                           uint32_t (&key)[KPT], uint32_t& valid, uint32_t& vis) {
+  valid = 0;
+  vis = 0;
+  if (kVec && pos0 + KPT <= n) {
+#pragma unroll
+    for (int j = 0; j < KPT; j += 4) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(psi + pos0 + j));
+      key[j] = psi_key(v.x);
+      key[j + 1] = psi_key(v.y);
+      key[j + 2] = psi_key(v.z);
+      key[j + 3] = psi_key(v.w);
+    }
+    valid = 0xffffffffu;
+  } else {
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+      key[j] = 0;
+      if (pos0 + j < n) {
+        key[j] = psi_key(__ldg(psi + pos0 + j));
+        valid |= 1u << j;
+      }
+    }
+  }
+  if (mpa) {
+#pragma unroll
+    for (int j = 0; j < KPT; ++j)
+      if (pos0 + j < n && __ldg(mask + pos0 + j)) vis |= 1u << j;
+  }
+}
+
+// The radix digits are taken from t = kmax - key, starting at the highest bit in which the unit's keys differ
+// (kmax, kmin: largest and smallest key of the unit): importance values share their sign and most exponent bits,
+// so digits of the raw key would put nearly all keys into a handful of buckets and serialise the shared atomics.
+// Ascending t is descending importance.
+template <bool kVec>
 __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
   __shared__ unsigned int cnt[2][256];
   __shared__ uint32_t s_prefix[2];
   __shared__ unsigned int s_above[2];
   __shared__ uint32_t warp_tot[NT / 32];
+  __shared__ uint32_t s_red[2][NT / 32];
 
   const int u = blockIdx.x;
   const int b = u / (p.Hkv * p.L);
@@ -119,38 +160,71 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
   const uint8_t* mask = p.mask + (int64_t)b * p.n_max;
   const int64_t off0 = p.seg_off[u];
   if (off0 + p.kept_len[u] + p.headroom > p.capacity) return;  // seg_scan has raised MADAKV_ECAPACITY
-  const int want[2] = {p.mpa ? max(p.budgets[2 * u], 0) : 0, max(p.budgets[2 * u + 1], 0)};
+  const int want0 = p.mpa ? max(p.budgets[2 * u], 0) : 0, want1 = max(p.budgets[2 * u + 1], 0);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunks = (n + CHUNK - 1) / CHUNK;
 
+  // range of the unit's keys (the chunk stays in registers when there is only one)
+  uint32_t key[KPT], valid = 0, vis = 0;
+  uint32_t kmax = 0, kmin = 0xffffffffu;
+  for (int c = 0; c < chunks; ++c) {
+    load_chunk<kVec>(psi, mask, n, c * CHUNK + (int)threadIdx.x * KPT, p.mpa, key, valid, vis);
+#pragma unroll
+    for (int j = 0; j < KPT; ++j)
+      if ((valid >> j) & 1u) {
+        kmax = max(kmax, key[j]);
+        kmin = min(kmin, key[j]);
+      }
+  }
+  kmax = __reduce_max_sync(kFull, kmax);
+  kmin = __reduce_min_sync(kFull, kmin);
+  if (lane == 0) {
+    s_red[0][warp] = kmax;
+    s_red[1][warp] = kmin;
+  }
   if (threadIdx.x < 2) {
     s_prefix[threadIdx.x] = 0;
     s_above[threadIdx.x] = 0;
   }
-  // radix select: after the 4 passes s_prefix[m] is the want[m]-th largest key of modality m (if that many exist)
-  // and s_above[m] counts the keys strictly above it
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_round = (n + 31) & ~31;  // whole warps run every iteration (the match below is a warp-wide call)
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < NT / 32; ++i) {
+    kmax = max(kmax, s_red[0][i]);
+    kmin = min(kmin, s_red[1][i]);
+  }
+  if (kmin > kmax) kmin = kmax;  // no keys at all
+  const int top = 32 - __clz(kmax - kmin);  // significant bits of t; 0 when all keys are equal
+  if (chunks == 1) {
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
+  }
+
+  // radix select: when all bits of t are resolved, s_prefix[m] is the t of the want[m]-th largest key of modality m
+  // (if that many exist) and s_above[m] counts the keys strictly above it. `rem` counts the bits not yet resolved.
+  for (int rem = top; rem > 0;) {
+    const int bits = min(rem, 8), shift = rem - bits;
+    const uint32_t dmask = (1u << bits) - 1u;
     for (int x = threadIdx.x; x < 512; x += NT) (&cnt[0][0])[x] = 0;
     __syncthreads();
     const uint32_t pre0 = s_prefix[0], pre1 = s_prefix[1];
-    for (int i = threadIdx.x; i < n_round; i += NT) {
-      int bucket = -1;
-      if (i < n) {
-        const uint32_t key = psi_key(psi[i]);
-        const int m = (p.mpa && mask[i]) ? 0 : 1;
-        if ((key & himask) == (m == 0 ? pre0 : pre1)) bucket = m * 256 + (int)((key >> shift) & 255u);
+    for (int c = 0; c < chunks; ++c) {
+      if (chunks > 1) {
+        load_chunk<kVec>(psi, mask, n, c * CHUNK + (int)threadIdx.x * KPT, p.mpa, key, valid, vis);
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
       }
-      // lanes that hit the same bucket are counted by one of them: importance values cluster in a few exponent
-      // buckets, and per-lane atomics on them would serialise
-      const unsigned int peers = __match_any_sync(0xffffffffu, bucket);
-      if (bucket >= 0 && lane == __ffs(peers) - 1) atomicAdd(&(&cnt[0][0])[bucket], (unsigned int)__popc(peers));
+#pragma unroll
+      for (int j = 0; j < KPT; ++j) {
+        const int m = (vis >> j) & 1u ? 0 : 1;
+        if (((valid >> j) & 1u) && (key[j] >> rem) == (m == 0 ? pre0 : pre1))
+          atomicAdd(&cnt[m][(key[j] >> shift) & dmask], 1u);
+      }
     }
     __syncthreads();
     if (warp < 2) {
-      // warp m walks modality m's buckets from the top; lane j owns buckets 8j..8j+7
+      // warp m walks modality m's buckets in ascending digit order; lane j owns buckets 8j..8j+7
       const int m = warp;
+      const unsigned int want = (unsigned int)(m == 0 ? want0 : want1);
       unsigned int cs[8], lc = 0;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -160,77 +234,80 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
       unsigned int sc = lc;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
-        const unsigned int t = __shfl_down_sync(0xffffffffu, sc, off);
-        if (lane + off < 32) sc += t;
+        const unsigned int t = __shfl_up_sync(kFull, sc, off);
+        if (lane >= off) sc += t;
       }
       unsigned int above = s_above[m] + (sc - lc);
       int found = -1;
 #pragma unroll
-      for (int j = 7; j >= 0; --j) {
+      for (int j = 0; j < 8; ++j) {
         if (found < 0) {
-          if (above + cs[j] >= (unsigned int)want[m] || (lane == 0 && j == 0)) found = j;
+          if (above + cs[j] >= want || (lane == 31 && j == 7)) found = j;
           else above += cs[j];
         }
       }
-      const unsigned int hit = __ballot_sync(0xffffffffu, found >= 0);  // lane 0 always hits
-      if (lane == 31 - __clz(hit)) {
+      const unsigned int hit = __ballot_sync(kFull, found >= 0);  // lane 31 always hits
+      if (lane == __ffs(hit) - 1) {
+        // buckets beyond the pass's digit range are empty; landing there means "fewer keys than wanted"
         s_above[m] = above;
-        s_prefix[m] |= (uint32_t)(lane * 8 + found) << shift;
+        s_prefix[m] = (s_prefix[m] << bits) | min((uint32_t)(lane * 8 + found), dmask);
       }
     }
     __syncthreads();
+    rem = shift;
   }
-  const uint32_t thr[2] = {s_prefix[0], s_prefix[1]};
+  const uint32_t thr0 = s_prefix[0], thr1 = s_prefix[1];
   // ties at the threshold value that are still needed (all of them if the modality has fewer tokens than wanted)
-  const int ties[2] = {max(want[0] - (int)s_above[0], 0), max(want[1] - (int)s_above[1], 0)};
+  const int ties0 = max(want0 - (int)s_above[0], 0), ties1 = max(want1 - (int)s_above[1], 0);
 
-  // ordered sweep
-  int tie_run[2] = {0, 0};  // threshold-valued keys met so far, per modality
-  int out_run = 0;          // kept positions emitted so far
-  for (int base = 0; base < n; base += STEP) {
-    uint32_t key[ITEMS];
-    int mod[ITEMS];
-    uint32_t eq_pack = 0;
+  // ordered sweep: a thread's positions are consecutive, threads and chunks follow in position order
+  int tie_run0 = 0, tie_run1 = 0;  // threshold-valued keys met in earlier chunks, per modality
+  int out_run = 0;                 // kept positions emitted by earlier chunks
+  for (int c = 0; c < chunks; ++c) {
+    const int pos0 = c * CHUNK + (int)threadIdx.x * KPT;
+    if (chunks > 1) {
+      load_chunk<kVec>(psi, mask, n, pos0, p.mpa, key, valid, vis);
 #pragma unroll
-    for (int j = 0; j < ITEMS; ++j) {
-      const int i = base + threadIdx.x * ITEMS + j;
-      key[j] = 0;
-      mod[j] = -1;
-      if (i < n) {
-        key[j] = psi_key(psi[i]);
-        mod[j] = (p.mpa && mask[i]) ? 0 : 1;
-        if (key[j] == thr[mod[j]]) eq_pack += mod[j] == 0 ? 1u : 0x10000u;
+      for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
+    }
+    uint32_t eq_bits = 0, gt_bits = 0;
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+      const bool v = (vis >> j) & 1u;
+      const uint32_t thr = v ? thr0 : thr1;
+      if ((valid >> j) & 1u) {
+        if (key[j] == thr) eq_bits |= 1u << j;
+        if (key[j] < thr && (v ? want0 : want1) > 0) gt_bits |= 1u << j;  // smaller t: larger importance
       }
     }
+    const uint32_t eq_pack = (uint32_t)__popc(eq_bits & vis) | ((uint32_t)__popc(eq_bits & ~vis) << 16);
     uint32_t eq_total;
-    uint32_t eq_before = block_excl_scan(eq_pack, warp_tot, &eq_total);
-    int rank[2] = {tie_run[0] + (int)(eq_before & 0xffffu), tie_run[1] + (int)(eq_before >> 16)};
-    uint32_t keep_bits = 0, keep_cnt = 0;
-#pragma unroll
-    for (int j = 0; j < ITEMS; ++j) {
-      if (mod[j] < 0) continue;
-      const int m = mod[j];
-      bool keep = false;
-      if (want[m] > 0) {
-        if (key[j] > thr[m]) keep = true;
-        else if (key[j] == thr[m]) {
-          keep = rank[m] < ties[m];
-          rank[m] += 1;
-        }
+    const uint32_t eq_before = block_excl_scan(eq_pack, warp_tot, &eq_total);
+    // a threshold-valued key is kept while its rank among the modality's ties (in position order) is below ties[m]
+    const int room0 = ties0 - (tie_run0 + (int)(eq_before & 0xffffu));
+    const int room1 = ties1 - (tie_run1 + (int)(eq_before >> 16));
+    uint32_t keep_bits = gt_bits;
+    {
+      uint32_t ev = eq_bits & vis, et = eq_bits & ~vis;
+      for (int k = 0; k < room0 && ev && want0 > 0; ++k) {  // lowest positions first
+        keep_bits |= ev & (0u - ev);
+        ev &= ev - 1;
       }
-      if (keep) {
-        keep_bits |= 1u << j;
-        keep_cnt += 1;
+      for (int k = 0; k < room1 && et && want1 > 0; ++k) {
+        keep_bits |= et & (0u - et);
+        et &= et - 1;
       }
     }
     uint32_t keep_total;
-    const uint32_t slot = block_excl_scan(keep_cnt, warp_tot, &keep_total);
+    const uint32_t slot = block_excl_scan((uint32_t)__popc(keep_bits), warp_tot, &keep_total);
     int o = out_run + (int)slot;
-#pragma unroll
-    for (int j = 0; j < ITEMS; ++j)
-      if (keep_bits & (1u << j)) p.kept_idx[off0 + o++] = base + threadIdx.x * ITEMS + j;
-    tie_run[0] += (int)(eq_total & 0xffffu);
-    tie_run[1] += (int)(eq_total >> 16);
+    while (keep_bits) {
+      const int j = __ffs(keep_bits) - 1;
+      keep_bits &= keep_bits - 1;
+      p.kept_idx[off0 + o++] = pos0 + j;
+    }
+    tie_run0 += (int)(eq_total & 0xffffu);
+    tie_run1 += (int)(eq_total >> 16);
     out_run += (int)keep_total;
   }
 }
@@ -251,15 +328,17 @@ int launch_select(const madakv_config& c, const float* psi, const uint8_t* mask,
   p.capacity = capacity;
   p.ws = ws;
   p.units = c.batch * c.n_layers * c.n_kv_heads;
+  p.B = c.batch;
   p.L = c.n_layers;
   p.Hkv = c.n_kv_heads;
   p.n_max = c.max_seq_len;
   p.mpa = c.mpa;
   p.headroom = c.max_new_tokens;
   p.seq_nv = reinterpret_cast<int32_t*>((char*)ws + ws_layout(c).seq_nv_off);
-  count_visual_kernel<<<c.batch, 1024, 0, st>>>(p);
   seg_scan_kernel<<<1, 1024, 0, st>>>(p);
-  select_unit_kernel<<<p.units, NT, 0, st>>>(p);
+  // 16-byte loads of psi need every unit's row (n_max floats apart) to start on a 16-byte boundary
+  if (c.max_seq_len % 4 == 0) select_unit_kernel<true><<<p.units, NT, 0, st>>>(p);
+  else select_unit_kernel<false><<<p.units, NT, 0, st>>>(p);
   return launch_status();
 }
 
