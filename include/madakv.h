@@ -44,7 +44,8 @@ typedef enum madakv_status {
   MADAKV_ECAPACITY = 5,    /* ragged cache capacity exceeded (host- or device-detected)              */
   MADAKV_EUNSUPPORTED = 6, /* dtype / head_dim / window*g outside the supported set                  */
   MADAKV_ECUDA = 7,        /* a CUDA runtime call failed (launch configuration, missing sm_100 device) */
-  MADAKV_ETIMEOUT = 8      /* device-detected: a bounded wait inside a kernel ran out                */
+  MADAKV_ETIMEOUT = 8,     /* device-detected: a bounded wait inside a kernel ran out                */
+  MADAKV_ESTATIC = 9       /* madakv_decode_attn_static only: the problem needs more than its built-in scratch */
 } madakv_status;
 
 enum { MADAKV_F32 = 0, MADAKV_BF16 = 1 };
@@ -145,6 +146,31 @@ int madakv_compact(const madakv_config* cfg, const void* k, const void* v, madak
 int madakv_decode_attn(const madakv_config* cfg, int32_t layer, const void* q, const void* k_new, const void* v_new,
                        void* k_c, void* v_c, const int64_t* seg_off, int32_t* kept_len, int64_t capacity, void* out,
                        float* lse_out, void* ws, size_t ws_bytes, void* stream);
+
+/* Decode attention for callers that cannot allocate device memory. (No counterpart in the paper: this is the
+ * attention of Eq. 5 exactly as madakv_decode_attn computes it, packaged for a different kind of caller.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits, for example a plug-in called in the middle of an
+ * inference engine's step, whose memory pool is owned by the host application, or a real-time loop in which an
+ * allocation (which may synchronise the whole device) would break the latency budget. Such a caller has buffers
+ * for its inputs and outputs but nowhere to put the split partials the attention kernels exchange, and
+ * madakv_decode_attn asks for a workspace. This variant keeps those partials in a fixed array that is part of the
+ * library image: MADAKV_STATIC_SCRATCH_BYTES of device memory on every GPU that loads the library, held until the
+ * process exits. It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ * Arguments are those of madakv_decode_attn without k_new / v_new (no append, kept_len is only read), without the
+ * workspace, and with read-only caches. Same layouts, same result bits as madakv_decode_attn on the same inputs.
+ *   - Limit: B * L * H_q * ceil((n_max + max_new_tokens) / 512) * (d + 2) * 4 bytes must not exceed
+ *     MADAKV_STATIC_SCRATCH_BYTES; a larger problem returns MADAKV_ESTATIC before anything is launched.
+ *   - The first call on each device looks up the device address of the built-in array (a host-side query, no
+ *     allocation) with that device current; make that first call outside any stream capture.
+ *   - All calls on one device share the one array. Nothing in it has to start at zero (every partial that is read
+ *     was written earlier in the same call), but two calls whose kernels overlap on the GPU (different streams, or
+ *     different host threads) race on it: serialise them.                                                  */
+#define MADAKV_STATIC_SCRATCH_BYTES (16u << 20)
+int madakv_decode_attn_static(const madakv_config* cfg, int32_t layer, const void* q, const void* k_c, const void* v_c,
+                              const int64_t* seg_off, const int32_t* kept_len, int64_t capacity, void* out,
+                              float* lse_out, void* stream);
 
 /* Synchronises `stream`, copies the device status word (a madakv_status) to *status_out and clears it. */
 int madakv_poll_status(void* ws, void* stream, int32_t* status_out);

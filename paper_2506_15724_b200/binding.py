@@ -14,12 +14,14 @@ LIB_PATH = os.path.join(_HERE, "libmadakv.so")
 
 MADAKV_F32, MADAKV_BF16 = 0, 1
 HCC_OFF, HCC_PAPER, HCC_LITERAL = 0, 1, 2
-STATUS_NAMES = ["OK", "EINVAL", "ESHAPE", "EALIGN", "EWORKSPACE", "ECAPACITY", "EUNSUPPORTED", "ECUDA", "ETIMEOUT"]
-(OK, EINVAL, ESHAPE, EALIGN, EWORKSPACE, ECAPACITY, EUNSUPPORTED, ECUDA, ETIMEOUT) = range(9)
+STATUS_NAMES = ["OK", "EINVAL", "ESHAPE", "EALIGN", "EWORKSPACE", "ECAPACITY", "EUNSUPPORTED", "ECUDA", "ETIMEOUT",
+                "ESTATIC"]
+(OK, EINVAL, ESHAPE, EALIGN, EWORKSPACE, ECAPACITY, EUNSUPPORTED, ECUDA, ETIMEOUT, ESTATIC) = range(10)
+STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = [
     "madakv_abi_version", "madakv_status_string", "madakv_workspace_bytes", "madakv_score", "madakv_allocate",
-    "madakv_select", "madakv_compact", "madakv_decode_attn", "madakv_poll_status",
+    "madakv_select", "madakv_compact", "madakv_decode_attn", "madakv_decode_attn_static", "madakv_poll_status",
 ]
 
 
@@ -66,6 +68,7 @@ def lib():
         L.madakv_select.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, i64, vp, sz, vp]
         L.madakv_compact.argtypes = [cfgp, vp, vp, MadakvStrides, vp, vp, vp, vp, vp, i64, vp, sz, vp]
         L.madakv_decode_attn.argtypes = [cfgp, i32, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, sz, vp]
+        L.madakv_decode_attn_static.argtypes = [cfgp, i32, vp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.madakv_poll_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         for f in EXPORTS:
             if f not in ("madakv_status_string",):
@@ -139,6 +142,15 @@ def madakv_decode_attn(cfg, layer, q, k_new, v_new, k_c, v_c, seg_off, kept_len,
                                                           _ptr(k_c), _ptr(v_c), _ptr(seg_off), _ptr(kept_len),
                                                           k_c.shape[0], _ptr(out), _ptr(lse_out), _ptr(ws),
                                                           ws.numel(), _stream()))
+
+
+def madakv_decode_attn_static(cfg, layer, q, k_c, v_c, seg_off, kept_len, out, lse_out):
+    """Decode attention without a workspace: the library's built-in scratch is used, nothing is allocated. For
+    callers that may not allocate device memory; calls must not overlap on the GPU (they share the scratch)."""
+    _check("madakv_decode_attn_static", lib().madakv_decode_attn_static(ctypes.byref(cfg), layer, _ptr(q), _ptr(k_c),
+                                                                        _ptr(v_c), _ptr(seg_off), _ptr(kept_len),
+                                                                        k_c.shape[0], _ptr(out), _ptr(lse_out),
+                                                                        _stream()))
 
 
 def madakv_poll_status(ws):

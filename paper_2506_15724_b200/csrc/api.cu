@@ -19,6 +19,7 @@ const char* madakv_status_string(int s) {
     case MADAKV_EUNSUPPORTED: return "unsupported dtype, head_dim or window";
     case MADAKV_ECUDA: return "CUDA runtime error";
     case MADAKV_ETIMEOUT: return "bounded device wait expired";
+    case MADAKV_ESTATIC: return "problem exceeds the built-in scratch of madakv_decode_attn_static";
     default: return "unknown status";
   }
 }

@@ -5,6 +5,8 @@
 //            per lane), the g query heads of the KV group share every K/V row read; online softmax in the log2
 //            domain, fp32 accumulation; the block's row groups are merged in shared memory
 //   merge    one block per query head: fixed-order combination of the split partials, rounding to dtype once
+#include <mutex>
+
 #include "common.cuh"
 
 namespace madakv {
@@ -267,3 +269,83 @@ int launch_decode(const madakv_config& c, int layer, const void* q, const void* 
 }
 
 }  // namespace madakv
+
+// ---------------------------------------------------------------------------------------------------------------
+// madakv_decode_attn_static: the same attention kernels with their split partials in a fixed array of the library
+// image, for callers that have no way to provide (or allocate) a workspace.
+// ---------------------------------------------------------------------------------------------------------------
+
+// Split partials of the no-allocation entry point. One copy per GPU that loads the library, shared by all calls.
+static __device__ __align__(256) unsigned char g_static_scratch[MADAKV_STATIC_SCRATCH_BYTES];
+
+namespace madakv {
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};  // device address of g_static_scratch on each device, once looked up
+
+// In host code the name g_static_scratch is only a handle; the address kernels can use comes from the runtime,
+// per device, with that device current.
+int static_scratch(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MADAKV_ECUDA;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return MADAKV_ECUDA;
+    }
+    g_static_ptr[dev] = ptr;
+  }
+  *out = g_static_ptr[dev];
+  return MADAKV_OK;
+}
+
+}  // namespace
+}  // namespace madakv
+
+extern "C" int madakv_decode_attn_static(const madakv_config* cfg, int32_t layer, const void* q, const void* k_c,
+                                         const void* v_c, const int64_t* seg_off, const int32_t* kept_len,
+                                         int64_t capacity, void* out, float* lse_out, void* stream) {
+  using namespace madakv;
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (!q || !k_c || !v_c || !seg_off || !kept_len || !out) return MADAKV_EINVAL;
+  if (layer < -1 || layer >= cfg->n_layers) return MADAKV_ESHAPE;
+  if (capacity <= 0) return MADAKV_ECAPACITY;
+  if (!aligned16(q) || !aligned16(k_c) || !aligned16(v_c) || !aligned16(out) || ((uintptr_t)seg_off & 7) ||
+      ((uintptr_t)kept_len & 3) || ((uintptr_t)lse_out & 3))
+    return MADAKV_EALIGN;
+  const madakv_config& c = *cfg;
+  const int splits = ws_layout(c).decode_splits;
+  const size_t need = (size_t)c.batch * c.n_layers * c.n_q_heads * (size_t)splits * (c.head_dim + 2) * sizeof(float);
+  if (need > (size_t)MADAKV_STATIC_SCRATCH_BYTES) return MADAKV_ESTATIC;
+  void* scratch = nullptr;
+  if ((rc = static_scratch(&scratch))) return rc;
+
+  DecodeParams p;
+  p.q = q;
+  p.k_new = nullptr;  // no append: the caches and kept_len are only read
+  p.v_new = nullptr;
+  p.k_c = const_cast<void*>(k_c);
+  p.v_c = const_cast<void*>(v_c);
+  p.seg_off = seg_off;
+  p.kept_len = const_cast<int32_t*>(kept_len);
+  p.capacity = capacity;
+  p.out = out;
+  p.lse_out = lse_out;
+  p.part = reinterpret_cast<float*>(scratch);
+  p.ws = nullptr;  // only the append kernel reports through the workspace
+  p.L = c.n_layers;
+  p.Hq = c.n_q_heads;
+  p.Hkv = c.n_kv_heads;
+  p.g = c.n_q_heads / c.n_kv_heads;
+  p.layer = layer;
+  p.splits = splits;
+  p.scale2 = scale_of(c) * kLog2e;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (c.dtype == MADAKV_F32) return c.head_dim == 64 ? run<float, 64>(p, c, st) : run<float, 128>(p, c, st);
+  return c.head_dim == 64 ? run<__nv_bfloat16, 64>(p, c, st) : run<__nv_bfloat16, 128>(p, c, st);
+}
