@@ -15,8 +15,9 @@ namespace madakv {
 // Workspace layout (device memory owned by the caller)
 //   [0, 256)                 header: int32 status, then counters used by persistent kernels
 //   [256, ..)                stage 4 scratch: visual-token count per sequence [B] int32
-//   [.., .. + score)         stage 1 scratch: finished-item counters [units] int32, log2-domain row log-sum-exp
-//                            [units * g * w] fp32, per-chunk partial (max, sum) pairs [units * chunks * rows] float2
+//   [.., .. + score)         stage 1 scratch: finished-item counters [units * rows] int32, log2-domain row
+//                            log-sum-exp [units * rows] fp32 (rows = g * w padded to a multiple of 32), per-chunk
+//                            partial (max, sum) pairs [units * chunks * rows] float2
 //   [.., .. + decode)        stage 5 scratch: split partials [B * L * H_q * splits * (d + 2)] fp32
 // Stages 2-3 keep their scratch in shared memory.
 // ---------------------------------------------------------------------------------------------------------------
@@ -48,13 +49,13 @@ inline WsLayout ws_layout(const madakv_config& c) {
   size_t off = kHeaderBytes;
   w.seq_nv_off = off;
   off = align_up(off + (size_t)c.batch * sizeof(int32_t), 256);
+  const size_t rows_pad = (rows + 31) / 32 * 32;  // the tensor-core path pads the row count
   w.score_done_off = off;
-  off = align_up(off + units * sizeof(int32_t), 256);
+  off = align_up(off + units * rows_pad * sizeof(int32_t), 256);
   w.score_lse_off = off;
-  off = align_up(off + units * rows * sizeof(float), 256);
+  off = align_up(off + units * rows_pad * sizeof(float), 256);
   w.score_part_off = off;
   w.score_tc_chunks = (c.max_seq_len + kScoreTcChunk - 1) / kScoreTcChunk;
-  const size_t rows_pad = (rows + 31) / 32 * 32;  // the tensor-core path pads the row count
   off = align_up(off + units * rows_pad * (size_t)w.score_tc_chunks * sizeof(float2), 256);
   w.decode_off = off;
   off = align_up(off + (size_t)c.batch * c.n_layers * c.n_q_heads * (size_t)w.decode_splits * (c.head_dim + 2) *

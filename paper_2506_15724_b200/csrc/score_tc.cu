@@ -8,16 +8,21 @@
 //     partials, phase-2 items recompute the logits and emit psi. The item list interleaves phase 2 of chunk t with
 //     phase 1 of chunk t + lag, so the second read of a K chunk comes a bounded number of chunks after the first
 //     and is served by the L2 (phase-1 loads ask L2 to keep the lines, phase-2 loads to drop them);
-//   - a phase-2 item waits (bounded) until all phase-1 items of its unit have published their partials. Every item
-//     only depends on items earlier in the global order and every CTA walks its items in that order, so with all
-//     CTAs resident (grid <= SM count, one CTA per SM) the waits always end.
+//   - the thread that owns a window row publishes the row's partial of a phase-1 item and bumps that row's
+//     counter of the unit; the one whose bump completes the unit merges the row's partials (in chunk order, so the
+//     bits do not depend on who finishes) into the row's log-sum-exp and flags it. A phase-2 item waits (bounded)
+//     for the flags of its unit. Every item only depends on items earlier in the global order and every CTA walks
+//     its items in that order, so with all CTAs resident (grid <= SM count, one CTA per SM) the waits always end.
 // Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 two epilogue groups that take
 // alternate work items (four warps = the four TMEM lane quarters; a thread owns one key of a tile and all window
 // rows of it, so psi(i) is an in-thread sum over N). The accumulators of a whole item stay in TMEM, so phase 1
-// reads them twice (row maximum, then one exp2 per logit) instead of rescaling a running sum.
+// reads them twice (row maximum, then one exp2 per logit) instead of rescaling a running sum; every tile's
+// accumulator is handed back to the MMA warp right after its last read, and the TMEM load of the next 32-column
+// slab is in flight while the current one is being exponentiated.
 // Every wait is bounded: on expiry the kernel records MADAKV_ETIMEOUT, lets its copies drain, frees TMEM and returns.
 #include <cuda.h>
 #include <cstdlib>
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -32,6 +37,7 @@ constexpr int kThreads = 320;                        // TMA warp, MMA warp, two 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kEmptyMax = -1.0e30f;               // "no key seen yet" marker of a running maximum
 constexpr long long kWaitCycles = 4000000000ll;     // ~2 s at B200 clocks: bound of every device-side wait
+constexpr int kReady = 1 << 16;                     // added to a row counter when the row's log-sum-exp is published
 
 static_assert(kTileKeys * (kItemCols / 64) == kScoreTcChunk, "the workspace is sized for the smallest work item");
 
@@ -40,7 +46,8 @@ struct TcParams {
   float* psi;        // [units, n_max]
   float* lse_out;    // natural log [B,L,Hq,w] or null
   float2* part;      // ws: [units, cpu, NPAD]
-  int32_t* done;     // ws: [units] phase-1 items finished
+  int32_t* done;     // ws: [units, NPAD] phase-1 items finished per window row; + kReady once lse2 is published
+  float* lse2;       // ws: [units, NPAD] log2-domain log-sum-exp of every window row
   int32_t* status;   // ws header
   int units, L, Hq, Hkv, g, w, R, n_max, cpu, causal, lag;
   float scale2;
@@ -110,26 +117,22 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes packed densely
-// (8-row groups 1024 bytes apart), descriptor version 1.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);  // start address
-  d |= (uint64_t)1 << 16;                    // leading byte offset (unused with swizzle), in 16-byte units
-  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset
-  d |= (uint64_t)1 << 46;                    // version
-  d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
-  return d;
-}
+// (8-row groups 1024 bytes apart), descriptor version 1. Only the low word depends on the address: start address
+// in 16-byte units (bits 0-13) and the unused leading byte offset (bit 16); the high word holds the stride byte
+// offset (1024 >> 4), the version (bit 46) and SWIZZLE_128B (bits 61-63). Moving the start by x bytes (x a multiple
+// of 16, same operand buffer) adds x >> 4 to the low word, which is all the MMA issue loop has to do per instruction.
+constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | (1u << 16); }
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_desc_lo, uint32_t b_desc_lo, uint32_t idesc,
                                           uint32_t accumulate) {
   asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "{\n.reg .pred p;\n.reg .b64 da, db;\nsetp.ne.b32 p, %4, 0;\nmov.b64 da, {%1, %5};\nmov.b64 db, {%2, %5};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n}"
+      ::"r"(d_tmem), "r"(a_desc_lo), "r"(b_desc_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
@@ -157,6 +160,12 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&a)[32], uint32_t (&b)[32
   asm volatile("tcgen05.wait::ld.sync.aligned;"
                : MADAKV_R8(a, 0), MADAKV_R8(a, 8), MADAKV_R8(a, 16), MADAKV_R8(a, 24), MADAKV_R8(b, 0), MADAKV_R8(b, 8),
                  MADAKV_R8(b, 16), MADAKV_R8(b, 24)
+               :
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&a)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : MADAKV_R8(a, 0), MADAKV_R8(a, 8), MADAKV_R8(a, 16), MADAKV_R8(a, 24)
                :
                : "memory");
 }
@@ -223,7 +232,7 @@ struct Item {
 };
 
 // The idx-th item of CTA `cta` (grid G): first its share of the phase-1 prologue (the first `lag` chunks), then its
-// super-items t = cta, cta + G, ...: phase 2 of chunk t followed by phase 1 of chunk t + lag.
+// super-items t = cta, cta + G, ...: phase 2 of chunk t and phase 1 of chunk t + lag (in alternating order).
 __device__ __forceinline__ bool get_item(int cta, int G, int idx, int total_chunks, int lag, int cpu, Item& it) {
   const int pro = min(lag, total_chunks);
   const int my_pro = cta < pro ? (pro - cta + G - 1) / G : 0;
@@ -237,8 +246,10 @@ __device__ __forceinline__ bool get_item(int cta, int G, int idx, int total_chun
     const int two = max(total_chunks - lag, 0);               // t in [0, two) have both halves
     const int my_two = cta < two ? (two - cta + G - 1) / G : 0;
     if (k < 2 * my_two) {
+      // the two halves swap places in every other super-item, so that each of the two epilogue groups (which take
+      // alternate items) gets phase-1 and phase-2 items in turn: a phase-1 item costs about twice a phase-2 item
       const int t = cta + (k >> 1) * G;
-      if (k & 1) { j = t + lag; phase = 1; } else { j = t; phase = 2; }
+      if (((k & 1) != 0) != (((k >> 1) & 1) != 0)) { j = t + lag; phase = 1; } else { j = t; phase = 2; }
     } else {
       const int k2 = k - 2 * my_two;
       const int t = cta + (my_two + k2) * G;
@@ -255,7 +266,7 @@ __device__ __forceinline__ bool get_item(int cta, int G, int idx, int total_chun
 
 // exp2 of 32 scaled-and-shifted logits, summed into 16 packed accumulators: acc2[i] += exp2(raw * scale - shift)
 __device__ __forceinline__ void exp_accumulate(const uint32_t (&raw)[32], uint64_t scale2x, const uint64_t* negshift2,
-                                               uint64_t (&acc2)[16]) {
+                                               uint64_t* acc2) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     float lo, hi;
@@ -293,12 +304,12 @@ struct SmemLayout {
   static constexpr int kKOff = 0;
   static constexpr int kQOff = kStages * kStageBytes;
   static constexpr int kBarOff = kQOff + 2 * kQBytes;
-  // full[kStages], empty[kStages], qfull[2], qempty[2], tfull[kItemBufs * kItemTiles], tempty[kItemBufs], ebar[2]
-  static constexpr int kNumBars = 2 * kStages + 4 + kItemBufs * kItemTiles + kItemBufs + 2;
+  // full[kStages], qfull[2], qempty[2], tfull / tempty[kItemBufs * kItemTiles], ebar[2]
+  static constexpr int kNumBars = kStages + 4 + 2 * kItemBufs * kItemTiles + 2;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   // misc: tmem base (4), abort flag (4); then per epilogue group: lse2[NPAD], vis[NPAD], red[4][NPAD] float2 and
   // a padded 32 x 33 transpose tile per warp
-  static constexpr int kGroupOff = kMiscOff + 16;
+  static constexpr int kGroupOff = kMiscOff + 48;  // + producer's stage ring (kStages <= 10 words)
   static constexpr int kGroupBytes = NPAD * 4 + NPAD * 4 + 4 * NPAD * 8 + 4 * 32 * 33 * 4;
   static constexpr int kTotal = kGroupOff + 2 * kGroupBytes;
   static constexpr int kAlloc = kTotal + 1024;  // slack for the 1024-byte alignment of the operand tiles
@@ -320,12 +331,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
   uint8_t* q_s = smem + SL::kQOff;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kBarOff);
   uint64_t* full = bars;                               // [kStages]                TMA -> MMA
-  uint64_t* empty = bars + kStages;                    // [kStages]                MMA -> TMA
-  uint64_t* qfull = bars + 2 * kStages;                // [2]
+  uint64_t* qfull = bars + kStages;                    // [2]
   uint64_t* qempty = qfull + 2;                        // [2]
-  uint64_t* tfull = qempty + 2;                        // [kItemBufs][kItemTiles]  MMA -> epilogue, one per tile
-  uint64_t* tempty = tfull + kItemBufs * kItemTiles;   // [kItemBufs]              epilogue -> MMA, one per item
-  uint64_t* ebars = tempty + kItemBufs;                // [2] barrier of each epilogue group
+  uint64_t* tfull = qempty + 2;                        // [kItemBufs][kItemTiles]  MMA -> epilogue and TMA, per tile
+  uint64_t* tempty = tfull + kItemBufs * kItemTiles;   // [kItemBufs][kItemTiles]  epilogue -> MMA, one per tile
+  uint64_t* ebars = tempty + kItemBufs * kItemTiles;   // [2] barrier of each epilogue group
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(smem + SL::kMiscOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::kMiscOff + 4);
 
@@ -336,15 +346,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&full[s], 1);
-      mbar_init(&empty[s], 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&qfull[i], 1);
       mbar_init(&qempty[i], 1);
       mbar_init(&ebars[i], 128);
     }
-    for (int i = 0; i < kItemBufs * kItemTiles; ++i) mbar_init(&tfull[i], 1);
-    for (int i = 0; i < kItemBufs; ++i) mbar_init(&tempty[i], 128);
+    for (int i = 0; i < kItemBufs * kItemTiles; ++i) {
+      mbar_init(&tfull[i], 1);
+      mbar_init(&tempty[i], 128);
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -367,10 +378,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
     // ================================================================ TMA producer
     if (lane == 0) {
       const uint64_t pol_keep = l2_policy_evict_last(), pol_drop = l2_policy_evict_first();
+      // A K stage may be refilled once the MMAs of the tile that used it last have completed. That event is the
+      // tile's tfull barrier (the MMA warp commits once per tile); stage_user remembers which one, and its parity.
+      volatile uint32_t* stage_user = reinterpret_cast<volatile uint32_t*>(smem + SL::kMiscOff + 8);
+      for (int s2 = 0; s2 < kStages; ++s2) stage_user[s2] = 0;
       int stage = 0;
-      uint32_t stage_par = 0;
       int qi = 0;
       uint32_t q_par = 0;
+      int active = 0;
       bool ok = true;
       Item it;
       for (int idx = 0; ok && get_item(blockIdx.x, gridDim.x, idx, total_chunks, p.lag, p.cpu, it); ++idx) {
@@ -378,6 +393,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         const int n = min(p.seq_len[b], p.n_max);
         const int key_begin = it.chunk * kItemKeys;
         if (key_begin >= n) continue;  // nothing to load for this item
+        const int ib = active % kItemBufs;
+        const uint32_t use_par = (uint32_t)(active / kItemBufs) & 1u;
+        ++active;
         // window queries of the unit
         ok = mbar_wait(&qempty[qi], q_par ^ 1, abort_flag, p.status);
         if (!ok) break;
@@ -391,16 +409,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         for (int t = 0; t < kItemTiles; ++t) {
           const int key0 = key_begin + t * kTileKeys;
           if (key0 >= n) break;
-          ok = mbar_wait(&empty[stage], stage_par ^ 1, abort_flag, p.status);
+          const uint32_t prev = stage_user[stage];
+          if (prev & 0x200u) ok = mbar_wait(&tfull[prev & 0xffu], (prev >> 8) & 1u, abort_flag, p.status);
           if (!ok) break;
+          stage_user[stage] = (uint32_t)(ib * kItemTiles + t) | (use_par << 8) | 0x200u;
           mbar_expect_tx(&full[stage], (uint32_t)SL::kStageBytes);
           for (int kb = 0; kb < kKBlocks; ++kb)
             tma_load_5d(k_s + stage * SL::kStageBytes + kb * kTileKeys * 128, &tmap_k, &full[stage], kb * 64, key0, h,
                         l, b, pol);
-          if (++stage == kStages) {
-            stage = 0;
-            stage_par ^= 1;
-          }
+          if (++stage == kStages) stage = 0;
         }
       }
       if (!ok) {  // abandoned: give copies in flight time to land before the CTA's shared memory goes away
@@ -412,6 +429,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
     // ================================================================ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc_bf16(NPAD);
+      const uint32_t k_lo0 = smem_desc_lo(smem_u32(k_s)), q_lo0 = smem_desc_lo(smem_u32(q_s));
       int stage = 0;
       uint32_t stage_par = 0;
       int qi = 0;
@@ -426,31 +444,31 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         if (key_begin >= n) continue;
         const int ib = active % kItemBufs;
         const uint32_t use_par = (uint32_t)(active / kItemBufs) & 1u;
-        ok = mbar_wait(&qfull[qi], q_par, abort_flag, p.status) &&
-             mbar_wait(&tempty[ib], use_par ^ 1, abort_flag, p.status);
+        ok = mbar_wait(&qfull[qi], q_par, abort_flag, p.status);
         if (!ok) break;
-        const uint32_t q_addr = smem_u32(q_s + qi * SL::kQBytes);
+        const uint32_t q_lo = q_lo0 + (uint32_t)qi * (SL::kQBytes >> 4);
         for (int t = 0; t < kItemTiles; ++t) {
           const int key0 = key_begin + t * kTileKeys;
           if (key0 < n) {
-            ok = mbar_wait(&full[stage], stage_par, abort_flag, p.status);
+            // the tile's accumulator slot must have been read for the last time, and the K tile must have landed
+            ok = mbar_wait(&tempty[ib * kItemTiles + t], use_par ^ 1, abort_flag, p.status) &&
+                 mbar_wait(&full[stage], stage_par, abort_flag, p.status);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t k_addr = smem_u32(k_s + stage * SL::kStageBytes);
+            const uint32_t k_lo = k_lo0 + (uint32_t)stage * (SL::kStageBytes >> 4);
             const uint32_t d_tmem = tmem_base + ib * kItemCols + t * NPAD;
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
               const int kb = ks >> 2, kk = ks & 3;
-              const uint64_t a = smem_desc_sw128(k_addr + kb * kTileKeys * 128 + kk * 32);
-              const uint64_t bq = smem_desc_sw128(q_addr + kb * NPAD * 128 + kk * 32);
-              umma_bf16(d_tmem, a, bq, idesc, ks > 0 ? 1u : 0u);
+              umma_bf16(d_tmem, k_lo + ((kb * kTileKeys * 128 + kk * 32) >> 4), q_lo + ((kb * NPAD * 128 + kk * 32) >> 4),
+                        idesc, ks > 0 ? 1u : 0u);
             }
-            umma_commit(&empty[stage]);  // the K stage may be refilled once these MMAs have read it
             if (++stage == kStages) {
               stage = 0;
               stage_par ^= 1;
             }
           }
+          // one commit per tile: the accumulator is ready for the epilogue, and the K stage may be refilled
           umma_commit(&tfull[ib * kItemTiles + t]);  // every tile barrier completes once per use of the set
         }
         if (!ok) break;
@@ -462,7 +480,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
     }
   } else {
     // ================================================================ epilogue: two groups of 128 threads; group e
-    // takes the active items of its parity. A thread owns one key of each tile (one TMEM lane).
+    // takes the active items of its parity. A thread owns one key of each tile (one TMEM lane). An item is read
+    // as 32-column slabs: slab s covers tile s / kSlabsPerTile and window rows 32 * (s % kSlabsPerTile) ...
+    constexpr int kSlabsPerTile = NPAD / 32;
+    constexpr int kH1 = kSlabsPerTile - 1;          // row half of the odd slabs
     const int grp = (warp - 2) >> 2;              // 0 or 1
     const int quarter = warp & 3;                 // TMEM lanes [32 * quarter, 32 * quarter + 32)
     const int et = (quarter << 5) | lane;         // key index inside the tile
@@ -495,55 +516,80 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
       const int ib = k_item % kItemBufs;
       const uint32_t use_par = (uint32_t)(k_item / kItemBufs) & 1u;
       const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + ib * kItemCols;
+      uint64_t* tf = &tfull[ib * kItemTiles];
+      uint64_t* te = &tempty[ib * kItemTiles];
+      const int nt = min(kItemTiles, (n - key_begin + kTileKeys - 1) / kTileKeys);
+      const int nslab = nt * kSlabsPerTile;
+      const int n_chunks_active = (n + kItemKeys - 1) / kItemKeys;
+      // keys below this bound are seen by every window row
+      const int all_bound = (n >= p.w) ? (p.causal ? n - p.w + 1 : n) : 0;
+      const uint64_t scale2x = pack2(p.scale2, p.scale2);
+      auto wait_tile = [&](int t) -> bool {
+        const bool w_ok = __all_sync(0xffffffffu, mbar_wait(&tf[t], use_par, abort_flag, p.status));
+        tc_fence_after();
+        return w_ok;
+      };
+      auto release_tile = [&](int t) {  // this thread has read tile t's accumulator for the last time
+        tc_fence_before();
+        mbar_arrive(&te[t]);
+      };
 
-      // per-row visibility bound (exclusive key index) of this unit
       ok = epi_sync(ebar, e_par, abort_flag, p.status);  // the previous item's readers of the shared arrays are done
       if (!ok) break;
       if (ethread < NPAD) {
+        // per-row visibility bound (exclusive key index) of this unit
         int vis = 0;
         if (ethread < p.R) {
           const int pos = n - p.w + ethread % p.w;
           if (pos >= 0) vis = p.causal ? pos + 1 : n;
         }
         vis_s[ethread] = vis;
+        if (it.phase == 2) {
+          // wait until the row's log-sum-exp is published (all phase-1 items of the unit are done)
+          const int32_t* flag = p.done + (int64_t)it.unit * NPAD + ethread;
+          const long long t0 = clock64();
+          int spins = 0;
+          while (true) {
+            int v;
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+            if (v >= kReady) break;
+            if (*abort_flag) break;
+            __nanosleep(64);
+            if ((++spins & 255) == 0 && clock64() - t0 > kWaitCycles) {
+              *abort_flag = 1;
+              atomicCAS(p.status, 0, (int)MADAKV_ETIMEOUT);
+              break;
+            }
+          }
+          // negated for the exponent's fused multiply-add; padding rows get a huge shift (they add exp2(-huge) = 0)
+          lse_s[ethread] = ethread < p.R ? -__ldcg(p.lse2 + (int64_t)it.unit * NPAD + ethread) : kEmptyMax;
+        }
       }
-      const int n_chunks_active = (n + kItemKeys - 1) / kItemKeys;
-      // keys below this bound are seen by every window row
-      const int all_bound = (n >= p.w) ? (p.causal ? n - p.w + 1 : n) : 0;
+      ok = epi_sync(ebar, e_par, abort_flag, p.status);  // vis_s (and lse_s) are published
+      ok = __all_sync(0xffffffffu, ok && !*abort_flag);
+      if (!ok) break;
 
       if (it.phase == 1) {
-        ok = epi_sync(ebar, e_par, abort_flag, p.status);  // vis_s is published
-        if (!ok) break;
-        // Two 32-column slabs are in registers at a time: tiles t and t + 1 (NPAD 32) or the two column halves of
-        // tile t (NPAD 64).
-        constexpr int kTilesPerPair = NPAD == 32 ? 2 : 1;
-        int nt = 0;
-        while (nt < kItemTiles && key_begin + nt * kTileKeys < n) ++nt;
-        const uint64_t* tf = &tfull[ib * kItemTiles];
-        // pass A: maximum of the raw logits per window row over this lane's keys, then over the warp
+        // pass A: maximum of the raw logits per window row over this lane's keys, two slabs at a time
         float st_m[NPAD];
 #pragma unroll
         for (int c = 0; c < NPAD; ++c) st_m[c] = kEmptyMax;
-        for (int t = 0; t < nt; t += kTilesPerPair) {
+        for (int s = 0; s < nslab; s += 2) {
           uint32_t ra[32], rb[32];
-          const int key0 = key_begin + t * kTileKeys;
-          const bool two = NPAD == 64 || t + 1 < nt;
-          ok = __all_sync(0xffffffffu, mbar_wait(const_cast<uint64_t*>(&tf[t]), use_par, abort_flag, p.status) &&
-                                           (NPAD == 64 || !two ||
-                                            mbar_wait(const_cast<uint64_t*>(&tf[t + 1]), use_par, abort_flag, p.status)));
+          const bool two = s + 1 < nslab;
+          const int t0 = s / kSlabsPerTile, t1 = (s + 1) / kSlabsPerTile;
+          ok = wait_tile(t0) && (!two || t1 == t0 || wait_tile(t1));
           if (!ok) break;
-          tc_fence_after();
-          tmem_ld32_issue(tbase + t * NPAD, ra);
-          if (two) tmem_ld32_issue(tbase + t * NPAD + 32, rb);  // next tile (NPAD 32) or upper columns (NPAD 64)
+          tmem_ld32_issue(tbase + s * 32, ra);
+          if (two) tmem_ld32_issue(tbase + (s + 1) * 32, rb);
           tmem_ld_wait(ra, rb);
           if (!two) {
 #pragma unroll
             for (int c = 0; c < 32; ++c) rb[c] = __float_as_uint(kEmptyMax);
           }
-          if (key0 + kTilesPerPair * kTileKeys > all_bound) {
-            mask_slab(ra, key0 + et, vis_s);
-            if (two) mask_slab(rb, (NPAD == 32 ? key0 + kTileKeys : key0) + et, vis_s + (NPAD == 32 ? 0 : 32));
-          }
+          const int key0 = key_begin + t0 * kTileKeys, key1 = key_begin + t1 * kTileKeys;
+          if (key0 + kTileKeys > all_bound) mask_slab(ra, key0 + et, vis_s);
+          if (two && key1 + kTileKeys > all_bound) mask_slab(rb, key1 + et, vis_s + kH1 * 32);
           if constexpr (NPAD == 32) {
 #pragma unroll
             for (int c = 0; c < 32; ++c) st_m[c] = max3(st_m[c], __uint_as_float(ra[c]), __uint_as_float(rb[c]));
@@ -556,51 +602,53 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
           }
         }
         if (!ok) break;
-        // pass B: sum of exp2 against the warp's maximum (second read of the accumulators, still in TMEM)
-        uint64_t negm2[NPAD / 2], z2[NPAD / 2];
+        // pass B: sum of exp2 against the warp's maximum (second read of the accumulators, still in TMEM); the
+        // load of the next slab is in flight while the current one is processed
+        // the (negated, scaled) maxima are uniform over the warp: they go to the warp's shared-memory scratch (the
+        // transpose tile, not yet in use) and are read back as packed pairs, which keeps 32 registers free
+        uint64_t z2[NPAD / 2];
+        float* negm_s = tr_s + (ethread >> 5) * (32 * 33);
+        const uint64_t* negm2 = reinterpret_cast<const uint64_t*>(negm_s);
 #pragma unroll
-        for (int i = 0; i < NPAD / 2; ++i) {
-          negm2[i] = pack2(-(warp_max(st_m[2 * i]) * p.scale2), -(warp_max(st_m[2 * i + 1]) * p.scale2));
-          z2[i] = 0ull;
+        for (int c = 0; c < NPAD; ++c) {
+          const float wm = warp_max(st_m[c]);
+          if (lane == (c & 31)) negm_s[c] = -(wm * p.scale2);
         }
-        const uint64_t scale2x = pack2(p.scale2, p.scale2);
-        for (int t = 0; t < nt; t += kTilesPerPair) {
-          uint32_t ra[32], rb[32];
-          const int key0 = key_begin + t * kTileKeys;
-          const bool two = NPAD == 64 || t + 1 < nt;
-          const bool msk = key0 + kTilesPerPair * kTileKeys > all_bound;
-          tmem_ld32_issue(tbase + t * NPAD, ra);
-          tmem_ld_wait(ra, ra);
-          if (msk) mask_slab(ra, key0 + et, vis_s);
-          if constexpr (NPAD == 32) {
-            exp_accumulate(ra, scale2x, negm2, z2);
-            if (two) {
-              tmem_ld32_issue(tbase + t * NPAD + 32, ra);
-              tmem_ld_wait(ra, ra);
-              if (msk) mask_slab(ra, key0 + kTileKeys + et, vis_s);
-              exp_accumulate(ra, scale2x, negm2, z2);
+#pragma unroll
+        for (int i = 0; i < NPAD / 2; ++i) z2[i] = 0ull;
+        __syncwarp();
+        {
+          uint32_t ra[32];
+          auto proc = [&](uint32_t (&r)[32], int s, auto half) {
+            constexpr int H = decltype(half)::value;
+            const int t = s / kSlabsPerTile;
+            const int key0 = key_begin + t * kTileKeys;
+            if (H == kH1) release_tile(t);
+            if (key0 + kTileKeys > all_bound) mask_slab(r, key0 + et, vis_s + H * 32);
+            exp_accumulate(r, scale2x, negm2 + H * 16, z2 + H * 16);
+          };
+          for (int s = 0; s < nslab; s += 2) {
+            tmem_ld32_issue(tbase + s * 32, ra);
+            tmem_ld_wait(ra);
+            proc(ra, s, std::integral_constant<int, 0>());
+            if (s + 1 < nslab) {
+              tmem_ld32_issue(tbase + (s + 1) * 32, ra);
+              tmem_ld_wait(ra);
+              proc(ra, s + 1, std::integral_constant<int, kH1>());
             }
-          } else {
-            tmem_ld32_issue(tbase + t * NPAD + 32, rb);
-            tmem_ld_wait(rb, rb);
-            if (msk) mask_slab(rb, key0 + et, vis_s + 32);
-            exp_accumulate(ra, scale2x, negm2, reinterpret_cast<uint64_t(&)[16]>(z2[0]));
-            exp_accumulate(rb, scale2x, negm2 + 16, reinterpret_cast<uint64_t(&)[16]>(z2[16]));
           }
         }
-        tc_fence_before();
-        mbar_arrive(&tempty[ib]);  // accumulators fully read: hand the set back to the MMA warp
+        for (int t = nt; t < kItemTiles; ++t) release_tile(t);  // unused slots: keep the barrier phases in step
         // back to scalars; a row of which the whole warp saw no visible key summed exp2(0) for its masked entries:
         // such a row is recorded as empty
         float st_z[NPAD];
 #pragma unroll
         for (int i = 0; i < NPAD / 2; ++i) {
-          float a, b;
-          unpack2(negm2[i], a, b);
-          st_m[2 * i] = -a;
-          st_m[2 * i + 1] = -b;
+          st_m[2 * i] = -negm_s[2 * i];
+          st_m[2 * i + 1] = -negm_s[2 * i + 1];
           unpack2(z2[i], st_z[2 * i], st_z[2 * i + 1]);
         }
+        __syncwarp();  // negm_s is about to be overwritten by the transpose
 #pragma unroll
         for (int c = 0; c < NPAD; ++c)
           if (st_m[c] < 0.5f * kEmptyMax * p.scale2) {
@@ -630,105 +678,75 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         ok = epi_sync(ebar, e_par, abort_flag, p.status);
         if (!ok) break;
         if (ethread < NPAD) {
+          // this thread owns window row `ethread`: publish the item's partial of the row, count it, and if that
+          // completes the unit merge the row's partials into its log-sum-exp
           float2 a = red_s[ethread];
 #pragma unroll
           for (int qd = 1; qd < 4; ++qd) {
             const float2 o = red_s[qd * NPAD + ethread];
             merge_stats(a.x, a.y, o.x, o.y);
           }
-          __stcg(p.part + ((int64_t)it.unit * p.cpu + it.chunk) * NPAD + ethread, a);
-          __threadfence();
-        }
-        ok = epi_sync(ebar, e_par, abort_flag, p.status);
-        if (!ok) break;
-        if (ethread == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.done + it.unit) : "memory");
-      } else {
-        // wait until every phase-1 item of this unit has published its partials
-        if (ethread == 0) {
-          const long long t0 = clock64();
-          int spins = 0;
-          while (true) {
-            int v;
-            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p.done + it.unit) : "memory");
-            if (v >= n_chunks_active) break;
-            if (*abort_flag) break;
-            __nanosleep(64);
-            if ((++spins & 255) == 0 && clock64() - t0 > kWaitCycles) {
-              *abort_flag = 1;
-              atomicCAS(p.status, 0, (int)MADAKV_ETIMEOUT);
-              break;
-            }
-          }
-        }
-        ok = epi_sync(ebar, e_par, abort_flag, p.status);
-        ok = __all_sync(0xffffffffu, ok && !*abort_flag);
-        if (!ok) break;
-        if (ethread < NPAD) {
-          float M = kEmptyMax, Z = 0.f;
-          const float2* part = p.part + (int64_t)it.unit * p.cpu * NPAD + ethread;
-          for (int c = 0; c < n_chunks_active; ++c) {
-            const float2 pz = __ldcg(part + c * NPAD);
-            merge_stats(M, Z, pz.x, pz.y);
-          }
-          const float lse2 = (Z > 0.f) ? M + log2f(Z) : 0.f;
-          lse_s[ethread] = lse2;
-          if (p.lse_out && it.chunk == 0 && ethread < p.R) {
-            const int hq = h * p.g + ethread / p.w, wr = ethread % p.w;
-            p.lse_out[((int64_t)bl * p.Hq + hq) * p.w + wr] = (Z > 0.f) ? lse2 * 0.6931471805599453f : -INFINITY;
-          }
-        }
-        ok = epi_sync(ebar, e_par, abort_flag, p.status);
-        if (!ok) break;
-        constexpr int kTilesPerPair = NPAD == 32 ? 2 : 1;
-        uint64_t neglse2[NPAD / 2];
+          float2* part = p.part + (int64_t)it.unit * p.cpu * NPAD + ethread;
+          __stcg(part + (int64_t)it.chunk * NPAD, a);
+          int32_t* cnt = p.done + (int64_t)it.unit * NPAD + ethread;
+          int old;
+          asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(cnt) : "memory");
+          if (old == n_chunks_active - 1) {
+            float M = kEmptyMax, Z = 0.f;
+            for (int c0 = 0; c0 < n_chunks_active; c0 += 8) {
+              float2 v[8];
 #pragma unroll
-        for (int i = 0; i < NPAD / 2; ++i)  // padding rows get a huge shift: they add exp2(-huge) = 0
-          neglse2[i] = pack2(2 * i < p.R ? -lse_s[2 * i] : kEmptyMax, 2 * i + 1 < p.R ? -lse_s[2 * i + 1] : kEmptyMax);
-        const uint64_t scale2x = pack2(p.scale2, p.scale2);
-        int nt = 0;
-        while (nt < kItemTiles && key_begin + nt * kTileKeys < n) ++nt;
-        const uint64_t* tf = &tfull[ib * kItemTiles];
-        for (int t = 0; t < nt; t += kTilesPerPair) {
-          uint32_t ra[32], rb[32];
-          const int key0 = key_begin + t * kTileKeys;
-          const bool two = NPAD == 64 || t + 1 < nt;
-          ok = __all_sync(0xffffffffu, mbar_wait(const_cast<uint64_t*>(&tf[t]), use_par, abort_flag, p.status) &&
-                                           (NPAD == 64 || !two ||
-                                            mbar_wait(const_cast<uint64_t*>(&tf[t + 1]), use_par, abort_flag, p.status)));
-          if (!ok) break;
-          tc_fence_after();
-          const bool msk = key0 + kTilesPerPair * kTileKeys > all_bound;
-          const int key = key0 + et;
-          float lo, hi;
-          tmem_ld32_issue(tbase + t * NPAD, ra);
-          tmem_ld_wait(ra, ra);
-          if (msk) mask_slab(ra, key, vis_s);
-          if constexpr (NPAD == 32) {
-            unpack2(exp_sum(ra, scale2x, neglse2, 0ull), lo, hi);
-            if (key < p.n_max) psi[key] = (key < n) ? lo + hi : 0.f;
-            if (two) {
-              tmem_ld32_issue(tbase + t * NPAD + 32, ra);
-              tmem_ld_wait(ra, ra);
-              if (msk) mask_slab(ra, key + kTileKeys, vis_s);
-              unpack2(exp_sum(ra, scale2x, neglse2, 0ull), lo, hi);
-              if (key + kTileKeys < p.n_max) psi[key + kTileKeys] = (key + kTileKeys < n) ? lo + hi : 0.f;
+              for (int j = 0; j < 8; ++j)
+                v[j] = c0 + j < n_chunks_active ? __ldcg(part + (int64_t)(c0 + j) * NPAD) : make_float2(kEmptyMax, 0.f);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) merge_stats(M, Z, v[j].x, v[j].y);
             }
-          } else {
-            const uint64_t part = exp_sum(ra, scale2x, neglse2, 0ull);
-            tmem_ld32_issue(tbase + t * NPAD + 32, ra);
-            tmem_ld_wait(ra, ra);
-            if (msk) mask_slab(ra, key, vis_s + 32);
-            unpack2(exp_sum(ra, scale2x, neglse2 + 16, part), lo, hi);
-            if (key < p.n_max) psi[key] = (key < n) ? lo + hi : 0.f;
+            const float lse2 = (Z > 0.f) ? M + log2f(Z) : 0.f;
+            __stcg(p.lse2 + (int64_t)it.unit * NPAD + ethread, lse2);
+            if (p.lse_out && ethread < p.R) {
+              const int hq = h * p.g + ethread / p.w, wr = ethread % p.w;
+              p.lse_out[((int64_t)bl * p.Hq + hq) * p.w + wr] = (Z > 0.f) ? lse2 * 0.6931471805599453f : -INFINITY;
+            }
+            asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(cnt), "r"(kReady) : "memory");
           }
         }
+      } else {
+        const uint64_t* neglse2 = reinterpret_cast<const uint64_t*>(lse_s);
+        uint32_t ra[32];
+        uint64_t acc = 0ull;
+        auto proc = [&](uint32_t (&r)[32], int s, auto half) {
+          constexpr int H = decltype(half)::value;
+          const int t = s / kSlabsPerTile;
+          const int key = key_begin + t * kTileKeys + et;
+          if (H == kH1) release_tile(t);
+          if (key - et + kTileKeys > all_bound) mask_slab(r, key, vis_s + H * 32);
+          acc = exp_sum(r, scale2x, neglse2 + H * 16, H == 0 ? 0ull : acc);
+          if (H == kH1) {
+            float lo, hi;
+            unpack2(acc, lo, hi);
+            if (key < p.n_max) psi[key] = (key < n) ? lo + hi : 0.f;
+          }
+        };
+        for (int s = 0; s < nslab; s += 2) {
+          ok = wait_tile(s / kSlabsPerTile);
+          if (!ok) break;
+          tmem_ld32_issue(tbase + s * 32, ra);
+          tmem_ld_wait(ra);
+          proc(ra, s, std::integral_constant<int, 0>());
+          if (s + 1 < nslab) {
+            if (kSlabsPerTile == 1) ok = wait_tile(s + 1);
+            if (!ok) break;
+            tmem_ld32_issue(tbase + (s + 1) * 32, ra);
+            tmem_ld_wait(ra);
+            proc(ra, s + 1, std::integral_constant<int, kH1>());
+          }
+        }
+        if (!ok) break;
         for (int t = nt; t < kItemTiles; ++t) {  // tiles beyond the sequence
           const int key = key_begin + t * kTileKeys + et;
           if (key < p.n_max) psi[key] = 0.f;
+          release_tile(t);
         }
-        if (!ok) break;
-        tc_fence_before();
-        mbar_arrive(&tempty[ib]);
       }
     }
   }
@@ -817,6 +835,7 @@ int launch_score_tc(const madakv_config& c, const void* q, madakv_strides sq, co
   p.lse_out = lse;
   p.part = reinterpret_cast<float2*>((char*)ws + wl.score_part_off);
   p.done = reinterpret_cast<int32_t*>((char*)ws + wl.score_done_off);
+  p.lse2 = reinterpret_cast<float*>((char*)ws + wl.score_lse_off);
   p.status = reinterpret_cast<int32_t*>(ws);
   p.units = c.batch * c.n_layers * c.n_kv_heads;
   p.L = c.n_layers;
@@ -848,7 +867,7 @@ int launch_score_tc(const madakv_config& c, const void* q, madakv_strides sq, co
   if (!make_map(&mk, k, c.head_dim, c.max_seq_len, c.n_kv_heads, c.n_layers, c.batch, sk, kTileKeys, 1) ||
       !make_map(&mq, q, c.head_dim, c.window, c.n_q_heads, c.n_layers, c.batch, sq, c.window, g))
     return MADAKV_EUNSUPPORTED;
-  if (cudaMemsetAsync(p.done, 0, (size_t)p.units * sizeof(int32_t), st) != cudaSuccess) return MADAKV_ECUDA;
+  if (cudaMemsetAsync(p.done, 0, (size_t)p.units * npad * sizeof(int32_t), st) != cudaSuccess) return MADAKV_ECUDA;
   if (c.head_dim == 128) return npad == 32 ? run_tc<128, 32>(mk, mq, p, grid, st) : run_tc<128, 64>(mk, mq, p, grid, st);
   return npad == 32 ? run_tc<64, 32>(mk, mq, p, grid, st) : run_tc<64, 64>(mk, mq, p, grid, st);
 }
