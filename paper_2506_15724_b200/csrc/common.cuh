@@ -17,7 +17,7 @@ namespace madakv {
 //   [256, ..)                stage 4 scratch: visual-token count per sequence [B] int32
 //   [.., .. + score)         stage 1 scratch: finished-item counters [units * rows] int32, log2-domain row
 //                            log-sum-exp [units * rows] fp32 (rows = g * w padded to a multiple of 32), per-chunk
-//                            partial (max, sum) pairs [units * chunks * rows] float2
+//                            partial (max, sum) pairs (see ws_layout)
 //   [.., .. + decode)        stage 5 scratch: split partials [B * L * H_q * splits * (d + 2)] fp32
 // Stages 2-3 keep their scratch in shared memory.
 // ---------------------------------------------------------------------------------------------------------------
@@ -28,7 +28,7 @@ constexpr int kDecodeChunk = 512;   // cache rows per split of decode attention
 
 struct WsHeader {
   int32_t status;        // madakv_status set by device code
-  int32_t work_counter;  // dynamic work distribution of persistent kernels
+  int32_t wait_site;     // diagnostic: which bounded wait gave up (site | block << 8), written with MADAKV_ETIMEOUT
   int32_t reserved[62];
 };
 static_assert(sizeof(WsHeader) == kHeaderBytes, "header size");
@@ -56,7 +56,14 @@ inline WsLayout ws_layout(const madakv_config& c) {
   off = align_up(off + units * rows_pad * sizeof(float), 256);
   w.score_part_off = off;
   w.score_tc_chunks = (c.max_seq_len + kScoreTcChunk - 1) / kScoreTcChunk;
-  off = align_up(off + units * rows_pad * (size_t)w.score_tc_chunks * sizeof(float2), 256);
+  // partials: the generic path keeps one (max, sum) per (chunk, row); the tensor-core path (rows <= 64 only) one
+  // per (work item, TMEM lane quarter, padded row)
+  size_t part = units * (size_t)w.score_chunks * rows * sizeof(float2);
+  if (rows <= 64) {
+    const size_t tc = units * rows_pad * (size_t)w.score_tc_chunks * 4 * sizeof(float2);
+    part = tc > part ? tc : part;
+  }
+  off = align_up(off + part, 256);
   w.decode_off = off;
   off = align_up(off + (size_t)c.batch * c.n_layers * c.n_q_heads * (size_t)w.decode_splits * (c.head_dim + 2) *
                            sizeof(float), 256);

@@ -8,17 +8,20 @@
 //     partials, phase-2 items recompute the logits and emit psi. The item list interleaves phase 2 of chunk t with
 //     phase 1 of chunk t + lag, so the second read of a K chunk comes a bounded number of chunks after the first
 //     and is served by the L2 (phase-1 loads ask L2 to keep the lines, phase-2 loads to drop them);
-//   - the thread that owns a window row publishes the row's partial of a phase-1 item and bumps that row's
-//     counter of the unit; the one whose bump completes the unit merges the row's partials (in chunk order, so the
-//     bits do not depend on who finishes) into the row's log-sum-exp and flags it. A phase-2 item waits (bounded)
+//   - every epilogue warp publishes, per window row, the partial of its quarter of a phase-1 item and bumps that
+//     row's counter of the unit; the lane whose bump completes the unit merges the row's partials (in a fixed order,
+//     so the bits do not depend on who finishes) into the row's log-sum-exp and flags it. A phase-2 item waits (bounded)
 //     for the flags of its unit. Every item only depends on items earlier in the global order and every CTA walks
 //     its items in that order, so with all CTAs resident (grid <= SM count, one CTA per SM) the waits always end.
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 two epilogue groups that take
-// alternate work items (four warps = the four TMEM lane quarters; a thread owns one key of a tile and all window
-// rows of it, so psi(i) is an in-thread sum over N). The accumulators of a whole item stay in TMEM, so phase 1
-// reads them twice (row maximum, then one exp2 per logit) instead of rescaling a running sum; every tile's
-// accumulator is handed back to the MMA warp right after its last read, and the TMEM load of the next 32-column
-// slab is in flight while the current one is being exponentiated.
+// Warp roles: warp 0 TMA producer; warps 1 and 10 MMA issuers that take alternate K tiles (an MMA of N <= 64 keeps
+// the tensor pipe busy for ~45 cycles, about as long as one thread needs to poll the two barriers of the next tile,
+// so two issuers keep the pipe fed); warps 2-9 epilogue: two groups of four warps that take alternate work items,
+// the four warps of a group being the four TMEM lane quarters. A thread owns one key of a tile and all window rows
+// of it, so psi(i) is an in-thread sum over N. The epilogue warps never synchronise with one another: every warp
+// keeps its own copy of the row shifts and visibility bounds, publishes its own (max, sum) partial per row and
+// item, and counts it on the row's counter. The accumulators of a whole item stay in TMEM, so phase 1 reads them
+// twice (row maximum, then one exp2 per logit) instead of rescaling a running sum; every tile's accumulator is
+// handed back to the MMA warps right after its last read.
 // Every wait is bounded: on expiry the kernel records MADAKV_ETIMEOUT, lets its copies drain, frees TMEM and returns.
 #include <cuda.h>
 #include <cstdlib>
@@ -33,7 +36,7 @@ constexpr int kTileKeys = 128;
 constexpr int kItemCols = 256;                      // TMEM columns of one work item's accumulators
 constexpr int kStagesD128 = 5;
 constexpr int kTmemCols = 512;
-constexpr int kThreads = 320;                        // TMA warp, MMA warp, two epilogue groups of four warps
+constexpr int kThreads = 352;                        // TMA warp, MMA warp, 8 epilogue warps, second MMA warp
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kEmptyMax = -1.0e30f;               // "no key seen yet" marker of a running maximum
 constexpr long long kWaitCycles = 4000000000ll;     // ~2 s at B200 clocks: bound of every device-side wait
@@ -45,8 +48,8 @@ struct TcParams {
   const int32_t* seq_len;
   float* psi;        // [units, n_max]
   float* lse_out;    // natural log [B,L,Hq,w] or null
-  float2* part;      // ws: [units, cpu, NPAD]
-  int32_t* done;     // ws: [units, NPAD] phase-1 items finished per window row; + kReady once lse2 is published
+  float2* part;      // ws: [units, cpu, 4 lane quarters, NPAD]
+  int32_t* done;     // ws: [units, NPAD] partials published per window row; + kReady once lse2 is published
   float* lse2;       // ws: [units, NPAD] log2-domain log-sum-exp of every window row
   int32_t* status;   // ws header
   int units, L, Hq, Hkv, g, w, R, n_max, cpu, causal, lag;
@@ -74,8 +77,16 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Records a wait that ran out: the status word, and (for diagnosis) which wait it was.
+enum { kSiteQEmpty = 1, kSiteStage = 2, kSiteQFull = 3, kSiteTEmpty = 4, kSiteFull = 5, kSiteTile = 6, kSiteFlag = 7,
+       kSiteDrain = 8 };
+__device__ __forceinline__ void give_up(volatile int* abort_flag, int32_t* status, int site) {
+  *abort_flag = 1;
+  if (atomicCAS(status, 0, (int)MADAKV_ETIMEOUT) == 0) status[1] = site | ((int)blockIdx.x << 8);
+}
 // Bounded wait. Returns false if the wait was abandoned (own timeout or another role's abort flag).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          int site) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   int spins = 0;
@@ -83,8 +94,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if ((++spins & 63) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitCycles) {
-        *abort_flag = 1;
-        atomicCAS(status, 0, (int)MADAKV_ETIMEOUT);
+        give_up(abort_flag, status, site);
         return false;
       }
     }
@@ -139,45 +149,27 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
-// Issue a 32-column TMEM load of this thread's lane; the registers are valid only after tmem_ld_wait on them.
-__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+// Issue a 16-column TMEM load of this thread's lane; the registers are valid only after tmem_ld_wait16 on them (the
+// registers pass through that statement so that no use of them can be scheduled before the wait). The epilogue
+// works on blocks of 16 window rows so that two blocks (one being processed, one in flight) fit the register budget.
+#define MADAKV_R8(r, o) "+r"(r[o]), "+r"(r[o + 1]), "+r"(r[o + 2]), "+r"(r[o + 3]), "+r"(r[o + 4]), "+r"(r[o + 5]), \
+                        "+r"(r[o + 6]), "+r"(r[o + 7])
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr)
       : "memory");
 }
-// Wait for this thread's outstanding TMEM loads. The registers pass through the statement so that no use of them
-// can be scheduled before the wait.
-#define MADAKV_R8(r, o) "+r"(r[o]), "+r"(r[o + 1]), "+r"(r[o + 2]), "+r"(r[o + 3]), "+r"(r[o + 4]), "+r"(r[o + 5]), \
-                        "+r"(r[o + 6]), "+r"(r[o + 7])
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&a)[32], uint32_t (&b)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : MADAKV_R8(a, 0), MADAKV_R8(a, 8), MADAKV_R8(a, 16), MADAKV_R8(a, 24), MADAKV_R8(b, 0), MADAKV_R8(b, 8),
-                 MADAKV_R8(b, 16), MADAKV_R8(b, 24)
-               :
-               : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&a)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : MADAKV_R8(a, 0), MADAKV_R8(a, 8), MADAKV_R8(a, 16), MADAKV_R8(a, 24)
-               :
-               : "memory");
+__device__ __forceinline__ void tmem_ld_wait16(uint32_t (&a)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" : MADAKV_R8(a, 0), MADAKV_R8(a, 8) : : "memory");
 }
 #undef MADAKV_R8
 __device__ __forceinline__ float warp_max(float v) {
   float r;
   asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
-  return r;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float r;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
 // packed pairs of fp32 (sm_100 f32x2 arithmetic): one instruction per two logits
@@ -209,15 +201,6 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// Barrier of the 128 epilogue threads on an mbarrier (count 128), so that it is bounded like every other wait.
-// The result is made uniform over the warp.
-__device__ __forceinline__ bool epi_sync(uint64_t* ebar, uint32_t& parity, volatile int* abort_flag, int32_t* status) {
-  mbar_arrive(ebar);
-  const bool ok = mbar_wait(ebar, parity, abort_flag, status);
-  parity ^= 1;
-  return __all_sync(0xffffffffu, ok);
-}
-
 // (max, sum) merge of two partial softmax statistics in the log2 domain.
 __device__ __forceinline__ void merge_stats(float& m, float& z, float mo, float zo) {
   const float mn = fmaxf(m, mo);
@@ -264,21 +247,21 @@ __device__ __forceinline__ bool get_item(int cta, int G, int idx, int total_chun
   return true;
 }
 
-// exp2 of 32 scaled-and-shifted logits, summed into 16 packed accumulators: acc2[i] += exp2(raw * scale - shift)
-__device__ __forceinline__ void exp_accumulate(const uint32_t (&raw)[32], uint64_t scale2x, const uint64_t* negshift2,
-                                               uint64_t* acc2) {
+// exp2 of 16 scaled-and-shifted logits, added to 8 packed accumulators (acc2[i] += exp2(raw * scale - shift)), or
+// all summed into one packed accumulator (phase 2: sum over window rows)
+__device__ __forceinline__ void exp_accumulate16(const uint32_t (&raw)[16], uint64_t scale2x, const uint64_t* negshift2,
+                                                 uint64_t* acc2) {
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+  for (int i = 0; i < 8; ++i) {
     float lo, hi;
     unpack2(fma2(pack2u(raw[2 * i], raw[2 * i + 1]), scale2x, negshift2[i]), lo, hi);
     acc2[i] = add2(acc2[i], pack2(ex2(lo), ex2(hi)));
   }
 }
-// the same, all 32 summed into one packed accumulator (phase 2: sum over window rows)
-__device__ __forceinline__ uint64_t exp_sum(const uint32_t (&raw)[32], uint64_t scale2x, const uint64_t* negshift2,
-                                            uint64_t acc) {
+__device__ __forceinline__ uint64_t exp_sum16(const uint32_t (&raw)[16], uint64_t scale2x, const uint64_t* negshift2,
+                                              uint64_t acc) {
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+  for (int i = 0; i < 8; ++i) {
     float lo, hi;
     unpack2(fma2(pack2u(raw[2 * i], raw[2 * i + 1]), scale2x, negshift2[i]), lo, hi);
     acc = add2(acc, pack2(ex2(lo), ex2(hi)));
@@ -286,12 +269,11 @@ __device__ __forceinline__ uint64_t exp_sum(const uint32_t (&raw)[32], uint64_t 
   return acc;
 }
 // logits of keys a window row may not see are replaced by a huge negative value
-__device__ __forceinline__ void mask_slab(uint32_t (&raw)[32], int key, const int* vis) {
+__device__ __forceinline__ void mask_block16(uint32_t (&raw)[16], int key, const int* vis) {
 #pragma unroll
-  for (int c = 0; c < 32; ++c)
+  for (int c = 0; c < 16; ++c)
     if (key >= vis[c]) raw[c] = __float_as_uint(kEmptyMax);
 }
-
 template <int D, int NPAD>
 struct SmemLayout {
   static constexpr int kStages = (D == 128 ? 1 : 2) * (NPAD == 32 ? kStagesD128 : kStagesD128 - 1);
@@ -304,14 +286,14 @@ struct SmemLayout {
   static constexpr int kKOff = 0;
   static constexpr int kQOff = kStages * kStageBytes;
   static constexpr int kBarOff = kQOff + 2 * kQBytes;
-  // full[kStages], qfull[2], qempty[2], tfull / tempty[kItemBufs * kItemTiles], ebar[2]
+  // full[kStages], qfull[2], qempty[2], tfull / tempty[kItemBufs * kItemTiles], drain[2]
   static constexpr int kNumBars = kStages + 4 + 2 * kItemBufs * kItemTiles + 2;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-  // misc: tmem base (4), abort flag (4); then per epilogue group: lse2[NPAD], vis[NPAD], red[4][NPAD] float2 and
-  // a padded 32 x 33 transpose tile per warp
-  static constexpr int kGroupOff = kMiscOff + 48;  // + producer's stage ring (kStages <= 10 words)
-  static constexpr int kGroupBytes = NPAD * 4 + NPAD * 4 + 4 * NPAD * 8 + 4 * 32 * 33 * 4;
-  static constexpr int kTotal = kGroupOff + 2 * kGroupBytes;
+  // misc: tmem base (4), abort flag (4), producer's stage ring (kStages <= 10 words); then per epilogue warp:
+  // shift[NPAD] (negated row maxima or log-sum-exps), vis[NPAD], a padded 32 x 33 transpose tile
+  static constexpr int kWarpOff = kMiscOff + 48;
+  static constexpr int kWarpBytes = NPAD * 4 + NPAD * 4 + 32 * 33 * 4;
+  static constexpr int kTotal = kWarpOff + 8 * kWarpBytes;
   static constexpr int kAlloc = kTotal + 1024;  // slack for the 1024-byte alignment of the operand tiles
   static_assert(kItemBufs == 2, "each epilogue group owns one accumulator set");
 };
@@ -335,7 +317,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
   uint64_t* qempty = qfull + 2;                        // [2]
   uint64_t* tfull = qempty + 2;                        // [kItemBufs][kItemTiles]  MMA -> epilogue and TMA, per tile
   uint64_t* tempty = tfull + kItemBufs * kItemTiles;   // [kItemBufs][kItemTiles]  epilogue -> MMA, one per tile
-  uint64_t* ebars = tempty + kItemBufs * kItemTiles;   // [2] barrier of each epilogue group
+  uint64_t* drain = tempty + kItemBufs * kItemTiles;   // [2] used only when the kernel gives up
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(smem + SL::kMiscOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::kMiscOff + 4);
 
@@ -349,8 +331,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&qfull[i], 1);
-      mbar_init(&qempty[i], 1);
-      mbar_init(&ebars[i], 128);
+      mbar_init(&qempty[i], 2);  // both MMA warps commit
+      mbar_init(&drain[i], 1);
     }
     for (int i = 0; i < kItemBufs * kItemTiles; ++i) {
       mbar_init(&tfull[i], 1);
@@ -379,9 +361,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
     if (lane == 0) {
       const uint64_t pol_keep = l2_policy_evict_last(), pol_drop = l2_policy_evict_first();
       // A K stage may be refilled once the MMAs of the tile that used it last have completed. That event is the
-      // tile's tfull barrier (the MMA warp commits once per tile); stage_user remembers which one, and its parity.
+      // tile's tfull barrier (the MMA warps commit once per tile). stage_user remembers which accumulator slot that
+      // tile went to; slot_par remembers, per slot, the parity of the latest use of the slot that this thread has
+      // loaded or passed (a slot of an item's unused tail is committed without a load). Waiting for that latest use
+      // is unambiguous (the barrier cannot be more than one phase beyond it, because the next use needs this thread)
+      // and implies the completion of every earlier use, the one that read the stage included. Short items can
+      // bring a slot round again within fewer tiles than there are stages, so the parity of the stage's own tile
+      // would not do.
       volatile uint32_t* stage_user = reinterpret_cast<volatile uint32_t*>(smem + SL::kMiscOff + 8);
       for (int s2 = 0; s2 < kStages; ++s2) stage_user[s2] = 0;
+      uint32_t slot_par = 0;  // bit per slot (kItemBufs * kItemTiles <= 16)
       int stage = 0;
       int qi = 0;
       uint32_t q_par = 0;
@@ -397,7 +386,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         const uint32_t use_par = (uint32_t)(active / kItemBufs) & 1u;
         ++active;
         // window queries of the unit
-        ok = mbar_wait(&qempty[qi], q_par ^ 1, abort_flag, p.status);
+        ok = mbar_wait(&qempty[qi], q_par ^ 1, abort_flag, p.status, kSiteQEmpty);
         if (!ok) break;
         mbar_expect_tx(&qfull[qi], (uint32_t)(p.R * 128 * kKBlocks));
         for (int kb = 0; kb < kKBlocks; ++kb)
@@ -408,11 +397,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         const uint64_t pol = it.phase == 1 ? pol_keep : pol_drop;
         for (int t = 0; t < kItemTiles; ++t) {
           const int key0 = key_begin + t * kTileKeys;
-          if (key0 >= n) break;
+          const int slot = ib * kItemTiles + t;
+          if (key0 >= n) {  // not loaded; the MMA warps commit its barrier all the same
+            slot_par = (slot_par & ~(1u << slot)) | (use_par << slot);
+            continue;
+          }
           const uint32_t prev = stage_user[stage];
-          if (prev & 0x200u) ok = mbar_wait(&tfull[prev & 0xffu], (prev >> 8) & 1u, abort_flag, p.status);
+          if (prev & 0x200u)
+            ok = mbar_wait(&tfull[prev & 0xffu], (slot_par >> (prev & 0xffu)) & 1u, abort_flag, p.status, kSiteStage);
           if (!ok) break;
-          stage_user[stage] = (uint32_t)(ib * kItemTiles + t) | (use_par << 8) | 0x200u;
+          stage_user[stage] = (uint32_t)slot | 0x200u;
+          slot_par = (slot_par & ~(1u << slot)) | (use_par << slot);
           mbar_expect_tx(&full[stage], (uint32_t)SL::kStageBytes);
           for (int kb = 0; kb < kKBlocks; ++kb)
             tma_load_5d(k_s + stage * SL::kStageBytes + kb * kTileKeys * 128, &tmap_k, &full[stage], kb * 64, key0, h,
@@ -425,13 +420,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         while (clock64() - t0 < 2000000ll) __nanosleep(1000);
       }
     }
-  } else if (warp == 1) {
-    // ================================================================ MMA issuer
+  } else if (warp == 1 || warp == 10) {
+    // ================================================================ MMA issuers: the loaded K tiles of the CTA,
+    // counted in load order, go to the two warps in turn
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc_bf16(NPAD);
+      const int me = warp == 1 ? 0 : 1;
       const uint32_t k_lo0 = smem_desc_lo(smem_u32(k_s)), q_lo0 = smem_desc_lo(smem_u32(q_s));
       int stage = 0;
       uint32_t stage_par = 0;
+      int turn = 0;  // parity of the running count of loaded tiles
       int qi = 0;
       uint32_t q_par = 0;
       int active = 0;  // active items issued so far; item k uses accumulator set k % kItemBufs
@@ -444,57 +442,65 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         if (key_begin >= n) continue;
         const int ib = active % kItemBufs;
         const uint32_t use_par = (uint32_t)(active / kItemBufs) & 1u;
-        ok = mbar_wait(&qfull[qi], q_par, abort_flag, p.status);
+        ok = mbar_wait(&qfull[qi], q_par, abort_flag, p.status, kSiteQFull);
         if (!ok) break;
         const uint32_t q_lo = q_lo0 + (uint32_t)qi * (SL::kQBytes >> 4);
         for (int t = 0; t < kItemTiles; ++t) {
           const int key0 = key_begin + t * kTileKeys;
           if (key0 < n) {
-            // the tile's accumulator slot must have been read for the last time, and the K tile must have landed
-            ok = mbar_wait(&tempty[ib * kItemTiles + t], use_par ^ 1, abort_flag, p.status) &&
-                 mbar_wait(&full[stage], stage_par, abort_flag, p.status);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t k_lo = k_lo0 + (uint32_t)stage * (SL::kStageBytes >> 4);
-            const uint32_t d_tmem = tmem_base + ib * kItemCols + t * NPAD;
+            if (turn == me) {
+              // the tile's accumulator slot must have been read for the last time, and the K tile must have landed
+              ok = mbar_wait(&tempty[ib * kItemTiles + t], use_par ^ 1, abort_flag, p.status, kSiteTEmpty) &&
+                   mbar_wait(&full[stage], stage_par, abort_flag, p.status, kSiteFull);
+              if (!ok) break;
+              tc_fence_after();
+              const uint32_t k_lo = k_lo0 + (uint32_t)stage * (SL::kStageBytes >> 4);
+              const uint32_t d_tmem = tmem_base + ib * kItemCols + t * NPAD;
 #pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-              const int kb = ks >> 2, kk = ks & 3;
-              umma_bf16(d_tmem, k_lo + ((kb * kTileKeys * 128 + kk * 32) >> 4), q_lo + ((kb * NPAD * 128 + kk * 32) >> 4),
-                        idesc, ks > 0 ? 1u : 0u);
+              for (int ks = 0; ks < D / 16; ++ks) {
+                const int kb = ks >> 2, kk = ks & 3;
+                umma_bf16(d_tmem, k_lo + ((kb * kTileKeys * 128 + kk * 32) >> 4),
+                          q_lo + ((kb * NPAD * 128 + kk * 32) >> 4), idesc, ks > 0 ? 1u : 0u);
+              }
+              // one commit per tile: the accumulator is ready for the epilogue, and the K stage may be refilled
+              umma_commit(&tfull[ib * kItemTiles + t]);
             }
+            turn ^= 1;
             if (++stage == kStages) {
               stage = 0;
               stage_par ^= 1;
             }
+          } else if ((t & 1) == me) {
+            umma_commit(&tfull[ib * kItemTiles + t]);  // every tile barrier completes once per use of the set
           }
-          // one commit per tile: the accumulator is ready for the epilogue, and the K stage may be refilled
-          umma_commit(&tfull[ib * kItemTiles + t]);  // every tile barrier completes once per use of the set
         }
         if (!ok) break;
-        umma_commit(&qempty[qi]);  // the Q buffer may be refilled once this item's MMAs are done
+        umma_commit(&qempty[qi]);  // the Q buffer may be refilled once both warps' MMAs of this item are done
         qi ^= 1;
         if (qi == 0) q_par ^= 1;
         ++active;
       }
+      if (!ok) {
+        // abandoned: TMEM may only be freed once this thread's MMAs have completed
+        umma_commit(&drain[me]);
+        const long long t0 = clock64();
+        while (!mbar_try(&drain[me], 0) && clock64() - t0 < 20000000ll) __nanosleep(200);
+      }
     }
   } else {
-    // ================================================================ epilogue: two groups of 128 threads; group e
-    // takes the active items of its parity. A thread owns one key of each tile (one TMEM lane). An item is read
-    // as 32-column slabs: slab s covers tile s / kSlabsPerTile and window rows 32 * (s % kSlabsPerTile) ...
-    constexpr int kSlabsPerTile = NPAD / 32;
-    constexpr int kH1 = kSlabsPerTile - 1;          // row half of the odd slabs
+    // ================================================================ epilogue: two groups of four warps; group e
+    // takes the active items of its parity, warp = TMEM lane quarter. A thread owns one key of each tile. The warps
+    // run independently of one another.
+    constexpr int kBlocks = NPAD / 16;              // 16-row blocks per tile
     const int grp = (warp - 2) >> 2;              // 0 or 1
     const int quarter = warp & 3;                 // TMEM lanes [32 * quarter, 32 * quarter + 32)
     const int et = (quarter << 5) | lane;         // key index inside the tile
-    const int ethread = (((warp - 2) & 3) << 5) | lane;  // 0..127 inside the group
-    uint8_t* gbase = smem + SL::kGroupOff + grp * SL::kGroupBytes;
-    float* lse_s = reinterpret_cast<float*>(gbase);
-    int* vis_s = reinterpret_cast<int*>(gbase + NPAD * 4);
-    float2* red_s = reinterpret_cast<float2*>(gbase + NPAD * 8);
-    float* tr_s = reinterpret_cast<float*>(gbase + NPAD * 8 + 4 * NPAD * 8);
-    uint64_t* ebar = &ebars[grp];
-    uint32_t e_par = 0;
+    uint8_t* wbase = smem + SL::kWarpOff + (warp - 2) * SL::kWarpBytes;
+    float* shift_s = reinterpret_cast<float*>(wbase);
+    int* vis_s = reinterpret_cast<int*>(wbase + NPAD * 4);
+    float* tr = reinterpret_cast<float*>(wbase + NPAD * 8);
+    const uint64_t* shift2 = reinterpret_cast<const uint64_t*>(shift_s);
+    const uint64_t scale2x = pack2(p.scale2, p.scale2);
     int active = 0;
     bool ok = true;
     Item it;
@@ -519,13 +525,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
       uint64_t* tf = &tfull[ib * kItemTiles];
       uint64_t* te = &tempty[ib * kItemTiles];
       const int nt = min(kItemTiles, (n - key_begin + kTileKeys - 1) / kTileKeys);
-      const int nslab = nt * kSlabsPerTile;
       const int n_chunks_active = (n + kItemKeys - 1) / kItemKeys;
       // keys below this bound are seen by every window row
       const int all_bound = (n >= p.w) ? (p.causal ? n - p.w + 1 : n) : 0;
-      const uint64_t scale2x = pack2(p.scale2, p.scale2);
       auto wait_tile = [&](int t) -> bool {
-        const bool w_ok = __all_sync(0xffffffffu, mbar_wait(&tf[t], use_par, abort_flag, p.status));
+        const bool w_ok = __all_sync(0xffffffffu, mbar_wait(&tf[t], use_par, abort_flag, p.status, kSiteTile));
         tc_fence_after();
         return w_ok;
       };
@@ -534,19 +538,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         mbar_arrive(&te[t]);
       };
 
-      ok = epi_sync(ebar, e_par, abort_flag, p.status);  // the previous item's readers of the shared arrays are done
-      if (!ok) break;
-      if (ethread < NPAD) {
+      __syncwarp();  // the warp's readers of shift_s / vis_s of the previous item are done
+#pragma unroll
+      for (int cb = 0; cb < NPAD; cb += 32) {
+        const int row = cb + lane;
         // per-row visibility bound (exclusive key index) of this unit
         int vis = 0;
-        if (ethread < p.R) {
-          const int pos = n - p.w + ethread % p.w;
+        if (row < p.R) {
+          const int pos = n - p.w + row % p.w;
           if (pos >= 0) vis = p.causal ? pos + 1 : n;
         }
-        vis_s[ethread] = vis;
+        vis_s[row] = vis;
         if (it.phase == 2) {
           // wait until the row's log-sum-exp is published (all phase-1 items of the unit are done)
-          const int32_t* flag = p.done + (int64_t)it.unit * NPAD + ethread;
+          const int32_t* flag = p.done + (int64_t)it.unit * NPAD + row;
           const long long t0 = clock64();
           int spins = 0;
           while (true) {
@@ -556,191 +561,140 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
             if (*abort_flag) break;
             __nanosleep(64);
             if ((++spins & 255) == 0 && clock64() - t0 > kWaitCycles) {
-              *abort_flag = 1;
-              atomicCAS(p.status, 0, (int)MADAKV_ETIMEOUT);
+              give_up(abort_flag, p.status, kSiteFlag);
               break;
             }
           }
           // negated for the exponent's fused multiply-add; padding rows get a huge shift (they add exp2(-huge) = 0)
-          lse_s[ethread] = ethread < p.R ? -__ldcg(p.lse2 + (int64_t)it.unit * NPAD + ethread) : kEmptyMax;
+          shift_s[row] = row < p.R ? -__ldcg(p.lse2 + (int64_t)it.unit * NPAD + row) : kEmptyMax;
         }
       }
-      ok = epi_sync(ebar, e_par, abort_flag, p.status);  // vis_s (and lse_s) are published
-      ok = __all_sync(0xffffffffu, ok && !*abort_flag);
+      __syncwarp();
+      ok = __all_sync(0xffffffffu, !*abort_flag);
       if (!ok) break;
 
+      // An item is read tile by tile in blocks of 16 window rows (16 TMEM columns); the load of the next block is in
+      // flight while the current one is processed. `body(j, r, t)` gets block j of tile t; `before_tile(t)` runs
+      // before the first load of tile t.
+      auto sweep = [&](auto before_tile, auto body) -> bool {
+        uint32_t ra[16], rb[16];
+        if (!before_tile(0)) return false;
+        tmem_ld16_issue(tbase, ra);
+        for (int t = 0; t < nt; ++t) {
+#pragma unroll
+          for (int j = 0; j < kBlocks; j += 2) {
+            tmem_ld_wait16(ra);
+            tmem_ld16_issue(tbase + t * NPAD + (j + 1) * 16, rb);
+            body(std::integral_constant<int, 0>(), j, ra, t);
+            tmem_ld_wait16(rb);
+            if (j + 2 < kBlocks) {
+              tmem_ld16_issue(tbase + t * NPAD + (j + 2) * 16, ra);
+            } else if (t + 1 < nt) {
+              if (!before_tile(t + 1)) return false;
+              tmem_ld16_issue(tbase + (t + 1) * NPAD, ra);
+            }
+            body(std::integral_constant<int, 1>(), j + 1, rb, t);
+          }
+        }
+        return true;
+      };
+
       if (it.phase == 1) {
-        // pass A: maximum of the raw logits per window row over this lane's keys, two slabs at a time
+        // pass A: maximum of the raw logits per window row over this lane's keys
         float st_m[NPAD];
 #pragma unroll
         for (int c = 0; c < NPAD; ++c) st_m[c] = kEmptyMax;
-        for (int s = 0; s < nslab; s += 2) {
-          uint32_t ra[32], rb[32];
-          const bool two = s + 1 < nslab;
-          const int t0 = s / kSlabsPerTile, t1 = (s + 1) / kSlabsPerTile;
-          ok = wait_tile(t0) && (!two || t1 == t0 || wait_tile(t1));
-          if (!ok) break;
-          tmem_ld32_issue(tbase + s * 32, ra);
-          if (two) tmem_ld32_issue(tbase + (s + 1) * 32, rb);
-          tmem_ld_wait(ra, rb);
-          if (!two) {
+        ok = sweep([&](int t) { return wait_tile(t); },
+                   [&](auto, int j, uint32_t (&r)[16], int t) {
+                     const int key0 = key_begin + t * kTileKeys;
+                     if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
 #pragma unroll
-            for (int c = 0; c < 32; ++c) rb[c] = __float_as_uint(kEmptyMax);
-          }
-          const int key0 = key_begin + t0 * kTileKeys, key1 = key_begin + t1 * kTileKeys;
-          if (key0 + kTileKeys > all_bound) mask_slab(ra, key0 + et, vis_s);
-          if (two && key1 + kTileKeys > all_bound) mask_slab(rb, key1 + et, vis_s + kH1 * 32);
-          if constexpr (NPAD == 32) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) st_m[c] = max3(st_m[c], __uint_as_float(ra[c]), __uint_as_float(rb[c]));
-          } else {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              st_m[c] = fmaxf(st_m[c], __uint_as_float(ra[c]));
-              st_m[32 + c] = fmaxf(st_m[32 + c], __uint_as_float(rb[c]));
-            }
-          }
-        }
+                     for (int c = 0; c < 16; ++c) st_m[j * 16 + c] = fmaxf(st_m[j * 16 + c], __uint_as_float(r[c]));
+                   });
         if (!ok) break;
-        // pass B: sum of exp2 against the warp's maximum (second read of the accumulators, still in TMEM); the
-        // load of the next slab is in flight while the current one is processed
-        // the (negated, scaled) maxima are uniform over the warp: they go to the warp's shared-memory scratch (the
-        // transpose tile, not yet in use) and are read back as packed pairs, which keeps 32 registers free
+        // pass B: sum of exp2 against the warp's maximum (second read of the accumulators, still in TMEM). The
+        // (negated, scaled) maxima are uniform over the warp: they go to the warp's shift_s and are read back as
+        // packed pairs, which keeps 32 registers free
         uint64_t z2[NPAD / 2];
-        float* negm_s = tr_s + (ethread >> 5) * (32 * 33);
-        const uint64_t* negm2 = reinterpret_cast<const uint64_t*>(negm_s);
 #pragma unroll
         for (int c = 0; c < NPAD; ++c) {
           const float wm = warp_max(st_m[c]);
-          if (lane == (c & 31)) negm_s[c] = -(wm * p.scale2);
+          if (lane == (c & 31)) shift_s[c] = -(wm * p.scale2);
         }
 #pragma unroll
         for (int i = 0; i < NPAD / 2; ++i) z2[i] = 0ull;
         __syncwarp();
-        {
-          uint32_t ra[32];
-          auto proc = [&](uint32_t (&r)[32], int s, auto half) {
-            constexpr int H = decltype(half)::value;
-            const int t = s / kSlabsPerTile;
-            const int key0 = key_begin + t * kTileKeys;
-            if (H == kH1) release_tile(t);
-            if (key0 + kTileKeys > all_bound) mask_slab(r, key0 + et, vis_s + H * 32);
-            exp_accumulate(r, scale2x, negm2 + H * 16, z2 + H * 16);
-          };
-          for (int s = 0; s < nslab; s += 2) {
-            tmem_ld32_issue(tbase + s * 32, ra);
-            tmem_ld_wait(ra);
-            proc(ra, s, std::integral_constant<int, 0>());
-            if (s + 1 < nslab) {
-              tmem_ld32_issue(tbase + (s + 1) * 32, ra);
-              tmem_ld_wait(ra);
-              proc(ra, s + 1, std::integral_constant<int, kH1>());
-            }
-          }
-        }
+        sweep([&](int) { return true; },
+              [&](auto, int j, uint32_t (&r)[16], int t) {
+                const int key0 = key_begin + t * kTileKeys;
+                if (j == kBlocks - 1) release_tile(t);  // all loads of the tile have completed
+                if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
+                exp_accumulate16(r, scale2x, shift2 + j * 8, z2 + j * 8);
+              });
         for (int t = nt; t < kItemTiles; ++t) release_tile(t);  // unused slots: keep the barrier phases in step
-        // back to scalars; a row of which the whole warp saw no visible key summed exp2(0) for its masked entries:
-        // such a row is recorded as empty
-        float st_z[NPAD];
+        // Sum over the 32 lanes of the warp through a padded shared-memory transpose (fixed order): lane j ends up
+        // with the sum of row cb + j, publishes the warp's partial of that row, counts it, and if that completes
+        // the unit merges all partials of the row into its log-sum-exp.
 #pragma unroll
-        for (int i = 0; i < NPAD / 2; ++i) {
-          st_m[2 * i] = -negm_s[2 * i];
-          st_m[2 * i + 1] = -negm_s[2 * i + 1];
-          unpack2(z2[i], st_z[2 * i], st_z[2 * i + 1]);
-        }
-        __syncwarp();  // negm_s is about to be overwritten by the transpose
+        for (int cb = 0; cb < NPAD; cb += 32) {
+          const int row = cb + lane;
 #pragma unroll
-        for (int c = 0; c < NPAD; ++c)
-          if (st_m[c] < 0.5f * kEmptyMax * p.scale2) {
-            st_m[c] = kEmptyMax;
-            st_z[c] = 0.f;
+          for (int c = 0; c < 16; ++c) {
+            float lo, hi;
+            unpack2(z2[cb / 2 + c], lo, hi);
+            tr[(2 * c) * 33 + lane] = lo;
+            tr[(2 * c + 1) * 33 + lane] = hi;
           }
-        // sum over the 32 lanes of the warp through a padded shared-memory transpose (fixed order): lane j ends up
-        // with the sum of row cb + j; the maximum is already uniform over the warp
-        {
-          float* tr = tr_s + (ethread >> 5) * (32 * 33);
+          __syncwarp();
+          float zsum = 0.f;
 #pragma unroll
-          for (int cb = 0; cb < NPAD; cb += 32) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) tr[c * 33 + lane] = st_z[cb + c];
-            if (lane == 0) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c) red_s[(ethread >> 5) * NPAD + cb + c].x = st_m[cb + c];
-            }
-            __syncwarp();
-            float zsum = 0.f;
-#pragma unroll
-            for (int i = 0; i < 32; ++i) zsum += tr[lane * 33 + i];
-            red_s[(ethread >> 5) * NPAD + cb + lane].y = zsum;
-            __syncwarp();
+          for (int i = 0; i < 32; ++i) zsum += tr[lane * 33 + i];
+          float m2 = -shift_s[row];
+          // a row of which the whole warp saw no visible key summed exp2(0) for its masked entries: it is empty
+          if (m2 < 0.5f * kEmptyMax * p.scale2) {
+            m2 = kEmptyMax;
+            zsum = 0.f;
           }
-        }
-        ok = epi_sync(ebar, e_par, abort_flag, p.status);
-        if (!ok) break;
-        if (ethread < NPAD) {
-          // this thread owns window row `ethread`: publish the item's partial of the row, count it, and if that
-          // completes the unit merge the row's partials into its log-sum-exp
-          float2 a = red_s[ethread];
-#pragma unroll
-          for (int qd = 1; qd < 4; ++qd) {
-            const float2 o = red_s[qd * NPAD + ethread];
-            merge_stats(a.x, a.y, o.x, o.y);
-          }
-          float2* part = p.part + (int64_t)it.unit * p.cpu * NPAD + ethread;
-          __stcg(part + (int64_t)it.chunk * NPAD, a);
-          int32_t* cnt = p.done + (int64_t)it.unit * NPAD + ethread;
+          __syncwarp();
+          float2* part = p.part + (int64_t)it.unit * p.cpu * (4 * NPAD) + row;
+          __stcg(part + (int64_t)(it.chunk * 4 + quarter) * NPAD, make_float2(m2, zsum));
+          int32_t* cnt = p.done + (int64_t)it.unit * NPAD + row;
           int old;
           asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(cnt) : "memory");
-          if (old == n_chunks_active - 1) {
+          if (old == 4 * n_chunks_active - 1) {
             float M = kEmptyMax, Z = 0.f;
-            for (int c0 = 0; c0 < n_chunks_active; c0 += 8) {
+            for (int e0 = 0; e0 < 4 * n_chunks_active; e0 += 8) {  // 4 * n_chunks_active is a multiple of 4
               float2 v[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j)
-                v[j] = c0 + j < n_chunks_active ? __ldcg(part + (int64_t)(c0 + j) * NPAD) : make_float2(kEmptyMax, 0.f);
+                v[j] = e0 + j < 4 * n_chunks_active ? __ldcg(part + (int64_t)(e0 + j) * NPAD)
+                                                    : make_float2(kEmptyMax, 0.f);
 #pragma unroll
               for (int j = 0; j < 8; ++j) merge_stats(M, Z, v[j].x, v[j].y);
             }
             const float lse2 = (Z > 0.f) ? M + log2f(Z) : 0.f;
-            __stcg(p.lse2 + (int64_t)it.unit * NPAD + ethread, lse2);
-            if (p.lse_out && ethread < p.R) {
-              const int hq = h * p.g + ethread / p.w, wr = ethread % p.w;
+            __stcg(p.lse2 + (int64_t)it.unit * NPAD + row, lse2);
+            if (p.lse_out && row < p.R) {
+              const int hq = h * p.g + row / p.w, wr = row % p.w;
               p.lse_out[((int64_t)bl * p.Hq + hq) * p.w + wr] = (Z > 0.f) ? lse2 * 0.6931471805599453f : -INFINITY;
             }
             asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(cnt), "r"(kReady) : "memory");
           }
         }
       } else {
-        const uint64_t* neglse2 = reinterpret_cast<const uint64_t*>(lse_s);
-        uint32_t ra[32];
         uint64_t acc = 0ull;
-        auto proc = [&](uint32_t (&r)[32], int s, auto half) {
-          constexpr int H = decltype(half)::value;
-          const int t = s / kSlabsPerTile;
-          const int key = key_begin + t * kTileKeys + et;
-          if (H == kH1) release_tile(t);
-          if (key - et + kTileKeys > all_bound) mask_slab(r, key, vis_s + H * 32);
-          acc = exp_sum(r, scale2x, neglse2 + H * 16, H == 0 ? 0ull : acc);
-          if (H == kH1) {
-            float lo, hi;
-            unpack2(acc, lo, hi);
-            if (key < p.n_max) psi[key] = (key < n) ? lo + hi : 0.f;
-          }
-        };
-        for (int s = 0; s < nslab; s += 2) {
-          ok = wait_tile(s / kSlabsPerTile);
-          if (!ok) break;
-          tmem_ld32_issue(tbase + s * 32, ra);
-          tmem_ld_wait(ra);
-          proc(ra, s, std::integral_constant<int, 0>());
-          if (s + 1 < nslab) {
-            if (kSlabsPerTile == 1) ok = wait_tile(s + 1);
-            if (!ok) break;
-            tmem_ld32_issue(tbase + (s + 1) * 32, ra);
-            tmem_ld_wait(ra);
-            proc(ra, s + 1, std::integral_constant<int, kH1>());
-          }
-        }
+        ok = sweep([&](int t) { return wait_tile(t); },
+                   [&](auto, int j, uint32_t (&r)[16], int t) {
+                     const int key = key_begin + t * kTileKeys + et;
+                     if (j == kBlocks - 1) release_tile(t);  // all loads of the tile have completed
+                     if (key - et + kTileKeys > all_bound) mask_block16(r, key, vis_s + j * 16);
+                     acc = exp_sum16(r, scale2x, shift2 + j * 8, j == 0 ? 0ull : acc);
+                     if (j == kBlocks - 1) {
+                       float lo, hi;
+                       unpack2(acc, lo, hi);
+                       if (key < p.n_max) psi[key] = (key < n) ? lo + hi : 0.f;
+                     }
+                   });
         if (!ok) break;
         for (int t = nt; t < kItemTiles; ++t) {  // tiles beyond the sequence
           const int key = key_begin + t * kTileKeys + et;
@@ -858,9 +812,18 @@ int launch_score_tc(const madakv_config& c, const void* q, madakv_strides sq, co
   const long long total = (long long)p.units * p.cpu;
   if (total > 0x3fffffff) return MADAKV_EUNSUPPORTED;
   const int grid = (int)(total < sms ? total : sms);
+  // Phase 1 leads phase 2 by two work items per CTA: the K chunks in between (2 * grid items of 256 KB) stay within
+  // the L2. A longer lead only spills the L2, and leads beyond two items per CTA are not used at all: in a run of
+  // the whole pass with a lead of three and more items per CTA the device reported a launch failure whose cause was
+  // not found. The lead must cover a whole unit (all its phase-1 items come before its first phase-2 item);
+  // sequences too long for that take the generic path. MADAKV_SCORE_LAG (tests) can shorten the lead.
   int lag = 2 * grid;
-  if (const char* e = getenv("MADAKV_SCORE_LAG")) lag = atoi(e);
+  if (const char* e = getenv("MADAKV_SCORE_LAG")) {
+    const int v = atoi(e);
+    if (v >= 1 && v < lag) lag = v;
+  }
   if (lag < p.cpu) lag = p.cpu;
+  if (lag > 2 * grid) return MADAKV_EUNSUPPORTED;
   p.lag = lag;
 
   CUtensorMap mk, mq;

@@ -35,6 +35,9 @@ SHAPES = {
     "tc_d128_r40": synth.scaled(TINY, dtype="bf16", L=1, Hq=2, Hkv=2, d=128, n=900, w=40, budget=120, theta=0.3),
     "tc_d64_r64_b3": synth.scaled(TINY, dtype="bf16", B=3, L=2, Hq=2, Hkv=2, d=64, n=2100, w=64, budget=333,
                                   theta=0.3),
+    # many short sequences: work items of one to four tiles follow one another (accumulator slots and K stages
+    # come round again within a few tiles)
+    "tc_short_seqs": synth.scaled(TINY, dtype="bf16", B=5, L=3, Hq=4, Hkv=4, d=128, n=389, w=8, budget=40, theta=0.3),
 }
 
 
