@@ -239,9 +239,11 @@ def main():
     for i in range(args.warmup):
         step(i)
     sync_all()
+    site = int(buf.ws[4:8].view(torch.int32).item())  # diagnostic word beside the status (which wait gave up)
     status = mk.madakv_poll_status(buf.ws)
     if status != 0:
-        raise SystemExit(f"device status {mk.madakv_status_string(status)} after warm-up")
+        raise SystemExit(f"device status {mk.madakv_status_string(status)} after warm-up (wait site {site & 255}, "
+                         f"block {site >> 8})")
 
     sampler = ClockSampler(local) if rank == 0 else None
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
@@ -331,9 +333,11 @@ def main():
         torch.cuda.synchronize()
         decode_us["full"] = time_decode(full, steps=5)
         del full
+    site = int(buf.ws[4:8].view(torch.int32).item())
     status = mk.madakv_poll_status(buf.ws)
     if status != 0:
-        raise SystemExit(f"device status {mk.madakv_status_string(status)} after the timed region")
+        raise SystemExit(f"device status {mk.madakv_status_string(status)} after the timed region (wait site "
+                         f"{site & 255}, block {site >> 8})")
 
     if rank != 0:
         if world > 1:

@@ -160,7 +160,7 @@ int madakv_decode_attn(const madakv_config* cfg, int32_t layer, const void* q, c
  *
  * Arguments are those of madakv_decode_attn without k_new / v_new (no append, kept_len is only read), without the
  * workspace, and with read-only caches. Same layouts, same result bits as madakv_decode_attn on the same inputs.
- *   - Limit: B * L * H_q * ceil((n_max + max_new_tokens) / 512) * (d + 2) * 4 bytes must not exceed
+ *   - Limit: B * L * H_q * ceil((n_max + max_new_tokens) / 256) * (d + 2) * 4 bytes must not exceed
  *     MADAKV_STATIC_SCRATCH_BYTES; a larger problem returns MADAKV_ESTATIC before anything is launched.
  *   - The first call on each device looks up the device address of the built-in array (a host-side query, no
  *     allocation) with that device current; make that first call outside any stream capture.

@@ -24,7 +24,7 @@ namespace madakv {
 constexpr size_t kHeaderBytes = 256;
 constexpr int kScoreChunk = 1024;   // keys per (max, sum) partial of the generic scoring path
 constexpr int kScoreTcChunk = 512;  // keys per work item (and per partial) of the tensor-core scoring path
-constexpr int kDecodeChunk = 512;   // cache rows per split of decode attention
+constexpr int kDecodeChunk = 256;   // cache rows per split of decode attention
 
 struct WsHeader {
   int32_t status;        // madakv_status set by device code

@@ -70,12 +70,19 @@ struct Vec16<float> {
     const float4 v = *reinterpret_cast<const float4*>(p);
     f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
   }
+  __device__ static void cvt(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+  }
 };
 template <>
 struct Vec16<__nv_bfloat16> {
   static constexpr int N = 8;
   __device__ static void load(const void* p, float* f) {
     const uint4 v = *reinterpret_cast<const uint4*>(p);
+    f[0] = bf16_lo(v.x); f[1] = bf16_hi(v.x); f[2] = bf16_lo(v.y); f[3] = bf16_hi(v.y);
+    f[4] = bf16_lo(v.z); f[5] = bf16_hi(v.z); f[6] = bf16_lo(v.w); f[7] = bf16_hi(v.w);
+  }
+  __device__ static void cvt(const uint4& v, float* f) {
     f[0] = bf16_lo(v.x); f[1] = bf16_hi(v.x); f[2] = bf16_lo(v.y); f[3] = bf16_hi(v.y);
     f[4] = bf16_lo(v.z); f[5] = bf16_hi(v.z); f[6] = bf16_lo(v.w); f[7] = bf16_hi(v.w);
   }
@@ -121,38 +128,49 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
   }
   const char* kc = (const char*)p.k_c + off * ROW_BYTES + lane * 16;
   const char* vc = (const char*)p.v_c + off * ROW_BYTES + lane * 16;
-  for (int r0 = row_begin; r0 < row_end; r0 += GROUPS) {  // uniform trip count: the shuffles below need full warps
-    const int r = r0 + grp;
-    const bool valid = r < row_end;
-    float kf[EPL], vf[EPL];
-    if (valid) {
-      Vec16<T>::load(kc + (int64_t)r * ROW_BYTES, kf);
-      Vec16<T>::load(vc + (int64_t)r * ROW_BYTES, vf);
-    } else {
+  // U rows per thread are in flight at a time: all their 16-byte K and V loads are issued before the first use, so a
+  // block keeps GROUPS * U * 2 * ROW_BYTES bytes on the wire (the online-softmax chain below is short next to the
+  // memory latency). Uniform trip count: the shuffles need full warps.
+  constexpr int U = G <= 2 ? 4 : 2;
+  for (int r0 = row_begin; r0 < row_end; r0 += GROUPS * U) {
+    uint4 kraw[U], vraw[U];
 #pragma unroll
-      for (int c = 0; c < EPL; ++c) kf[c] = vf[c] = 0.f;
+    for (int j = 0; j < U; ++j) {
+      const int r = r0 + grp + GROUPS * j;
+      kraw[j] = vraw[j] = make_uint4(0u, 0u, 0u, 0u);
+      if (r < row_end) {
+        kraw[j] = __ldcs(reinterpret_cast<const uint4*>(kc + (int64_t)r * ROW_BYTES));
+        vraw[j] = __ldcs(reinterpret_cast<const uint4*>(vc + (int64_t)r * ROW_BYTES));
+      }
     }
 #pragma unroll
-    for (int i = 0; i < G; ++i) {
-      if (i >= p.g) break;
-      float s = 0.f;
+    for (int j = 0; j < U; ++j) {
+      const bool valid = r0 + grp + GROUPS * j < row_end;
+      float kf[EPL], vf[EPL];
+      Vec16<T>::cvt(kraw[j], kf);
+      Vec16<T>::cvt(vraw[j], vf);
 #pragma unroll
-      for (int c = 0; c < EPL; ++c) s = fmaf(qr[i][c], kf[c], s);
+      for (int i = 0; i < G; ++i) {
+        if (i >= p.g) break;
+        float s = 0.f;
 #pragma unroll
-      for (int sh = LPR / 2; sh >= 1; sh >>= 1) s += __shfl_xor_sync(0xffffffffu, s, sh);
-      s *= p.scale2;
-      if (valid) {
-        if (s > m[i]) {
-          const float f = exp2f(m[i] - s);
-          l[i] *= f;
+        for (int c = 0; c < EPL; ++c) s = fmaf(qr[i][c], kf[c], s);
 #pragma unroll
-          for (int c = 0; c < EPL; ++c) o[i][c] *= f;
-          m[i] = s;
+        for (int sh = LPR / 2; sh >= 1; sh >>= 1) s += __shfl_xor_sync(0xffffffffu, s, sh);
+        s *= p.scale2;
+        if (valid) {
+          if (s > m[i]) {
+            const float f = exp2f(m[i] - s);
+            l[i] *= f;
+#pragma unroll
+            for (int c = 0; c < EPL; ++c) o[i][c] *= f;
+            m[i] = s;
+          }
+          const float pw = exp2f(s - m[i]);
+          l[i] += pw;
+#pragma unroll
+          for (int c = 0; c < EPL; ++c) o[i][c] = fmaf(pw, vf[c], o[i][c]);
         }
-        const float pw = exp2f(s - m[i]);
-        l[i] += pw;
-#pragma unroll
-        for (int c = 0; c < EPL; ++c) o[i][c] = fmaf(pw, vf[c], o[i][c]);
       }
     }
   }

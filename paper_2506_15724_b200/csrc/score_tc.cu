@@ -14,14 +14,21 @@
 //     for the flags of its unit. Every item only depends on items earlier in the global order and every CTA walks
 //     its items in that order, so with all CTAs resident (grid <= SM count, one CTA per SM) the waits always end.
 // Warp roles: warp 0 TMA producer; warps 1 and 10 MMA issuers that take alternate K tiles (an MMA of N <= 64 keeps
-// the tensor pipe busy for ~45 cycles, about as long as one thread needs to poll the two barriers of the next tile,
-// so two issuers keep the pipe fed); warps 2-9 epilogue: two groups of four warps that take alternate work items,
-// the four warps of a group being the four TMEM lane quarters. A thread owns one key of a tile and all window rows
+// the tensor pipe busy for ~45 cycles, about as long as one thread needs to poll the barriers of the next tile, so
+// two issuers keep the pipe fed). Both issuers wait on the "landed" barrier of EVERY K tile, in load order, also of
+// the tiles the other one issues, and a stage is only refilled once the tile's MMAs have completed AND the other
+// issuer has reported that it saw the tile land: a barrier that is tested by parity must be taken phase by phase
+// by each of its waiters, and none of them may fall two phases behind. (An issuer that only looked at its own
+// tiles could test a stage's barrier one phase early when loads complete out of order, e.g. an L2 hit overtaking
+// an HBM miss, and run ahead of the data; the producer then armed that barrier twice in one phase, which ended in
+// a launch failure. An issuer that took every phase but did not gate the refill could fall two phases behind and
+// wait for ever.) Warps 2-9 epilogue: two groups of four warps
+// that take alternate work items, the four warps of a group being the four TMEM lane quarters. A thread owns one key of a tile and all window rows
 // of it, so psi(i) is an in-thread sum over N. The epilogue warps never synchronise with one another: every warp
 // keeps its own copy of the row shifts and visibility bounds, publishes its own (max, sum) partial per row and
 // item, and counts it on the row's counter. The accumulators of a whole item stay in TMEM, so phase 1 reads them
 // twice (row maximum, then one exp2 per logit) instead of rescaling a running sum; every tile's accumulator is
-// handed back to the MMA warps right after its last read.
+// handed back to the MMA warp right after its last read.
 // Every wait is bounded: on expiry the kernel records MADAKV_ETIMEOUT, lets its copies drain, frees TMEM and returns.
 #include <cuda.h>
 #include <cstdlib>
@@ -286,8 +293,8 @@ struct SmemLayout {
   static constexpr int kKOff = 0;
   static constexpr int kQOff = kStages * kStageBytes;
   static constexpr int kBarOff = kQOff + 2 * kQBytes;
-  // full[kStages], qfull[2], qempty[2], tfull / tempty[kItemBufs * kItemTiles], drain[2]
-  static constexpr int kNumBars = kStages + 4 + 2 * kItemBufs * kItemTiles + 2;
+  // full[kStages], seen[kStages], qfull[2], qempty[2], tfull / tempty[kItemBufs * kItemTiles], drain[2]
+  static constexpr int kNumBars = 2 * kStages + 4 + 2 * kItemBufs * kItemTiles + 2;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   // misc: tmem base (4), abort flag (4), producer's stage ring (kStages <= 10 words); then per epilogue warp:
   // shift[NPAD] (negated row maxima or log-sum-exps), vis[NPAD], a padded 32 x 33 transpose tile
@@ -313,7 +320,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
   uint8_t* q_s = smem + SL::kQOff;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kBarOff);
   uint64_t* full = bars;                               // [kStages]                TMA -> MMA
-  uint64_t* qfull = bars + kStages;                    // [2]
+  uint64_t* seen = bars + kStages;                     // [kStages]  the MMA warp that does not issue a tile -> TMA
+  uint64_t* qfull = bars + 2 * kStages;                // [2]
   uint64_t* qempty = qfull + 2;                        // [2]
   uint64_t* tfull = qempty + 2;                        // [kItemBufs][kItemTiles]  MMA -> epilogue and TMA, per tile
   uint64_t* tempty = tfull + kItemBufs * kItemTiles;   // [kItemBufs][kItemTiles]  epilogue -> MMA, one per tile
@@ -328,6 +336,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&full[s], 1);
+      mbar_init(&seen[s], 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&qfull[i], 1);
@@ -361,7 +370,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
     if (lane == 0) {
       const uint64_t pol_keep = l2_policy_evict_last(), pol_drop = l2_policy_evict_first();
       // A K stage may be refilled once the MMAs of the tile that used it last have completed. That event is the
-      // tile's tfull barrier (the MMA warps commit once per tile). stage_user remembers which accumulator slot that
+      // tile's tfull barrier (the MMA warp commits once per tile). stage_user remembers which accumulator slot that
       // tile went to; slot_par remembers, per slot, the parity of the latest use of the slot that this thread has
       // loaded or passed (a slot of an item's unused tail is committed without a load). Waiting for that latest use
       // is unambiguous (the barrier cannot be more than one phase beyond it, because the next use needs this thread)
@@ -372,6 +381,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
       for (int s2 = 0; s2 < kStages; ++s2) stage_user[s2] = 0;
       uint32_t slot_par = 0;  // bit per slot (kItemBufs * kItemTiles <= 16)
       int stage = 0;
+      uint32_t lap_par = 0;  // parity of the number of times the stage ring has been gone round
       int qi = 0;
       uint32_t q_par = 0;
       int active = 0;
@@ -398,13 +408,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         for (int t = 0; t < kItemTiles; ++t) {
           const int key0 = key_begin + t * kTileKeys;
           const int slot = ib * kItemTiles + t;
-          if (key0 >= n) {  // not loaded; the MMA warps commit its barrier all the same
+          if (key0 >= n) {  // not loaded; the MMA warp commits its barrier all the same
             slot_par = (slot_par & ~(1u << slot)) | (use_par << slot);
             continue;
           }
           const uint32_t prev = stage_user[stage];
-          if (prev & 0x200u)
-            ok = mbar_wait(&tfull[prev & 0xffu], (slot_par >> (prev & 0xffu)) & 1u, abort_flag, p.status, kSiteStage);
+          if (prev & 0x200u)  // the stage's last tile: its MMAs are done, and the other MMA warp has seen it land
+            ok = mbar_wait(&tfull[prev & 0xffu], (slot_par >> (prev & 0xffu)) & 1u, abort_flag, p.status, kSiteStage) &&
+                 mbar_wait(&seen[stage], lap_par ^ 1u, abort_flag, p.status, kSiteStage);
           if (!ok) break;
           stage_user[stage] = (uint32_t)slot | 0x200u;
           slot_par = (slot_par & ~(1u << slot)) | (use_par << slot);
@@ -412,7 +423,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
           for (int kb = 0; kb < kKBlocks; ++kb)
             tma_load_5d(k_s + stage * SL::kStageBytes + kb * kTileKeys * 128, &tmap_k, &full[stage], kb * 64, key0, h,
                         l, b, pol);
-          if (++stage == kStages) stage = 0;
+          if (++stage == kStages) {
+            stage = 0;
+            lap_par ^= 1u;
+          }
         }
       }
       if (!ok) {  // abandoned: give copies in flight time to land before the CTA's shared memory goes away
@@ -426,10 +440,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc_bf16(NPAD);
       const int me = warp == 1 ? 0 : 1;
+      int turn = 0;  // parity of the running count of loaded tiles
       const uint32_t k_lo0 = smem_desc_lo(smem_u32(k_s)), q_lo0 = smem_desc_lo(smem_u32(q_s));
       int stage = 0;
       uint32_t stage_par = 0;
-      int turn = 0;  // parity of the running count of loaded tiles
       int qi = 0;
       uint32_t q_par = 0;
       int active = 0;  // active items issued so far; item k uses accumulator set k % kItemBufs
@@ -448,10 +462,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
         for (int t = 0; t < kItemTiles; ++t) {
           const int key0 = key_begin + t * kTileKeys;
           if (key0 < n) {
+            // the K tile must have landed (both warps take every stage barrier, phase by phase) ...
+            ok = mbar_wait(&full[stage], stage_par, abort_flag, p.status, kSiteFull);
+            if (!ok) break;
             if (turn == me) {
-              // the tile's accumulator slot must have been read for the last time, and the K tile must have landed
-              ok = mbar_wait(&tempty[ib * kItemTiles + t], use_par ^ 1, abort_flag, p.status, kSiteTEmpty) &&
-                   mbar_wait(&full[stage], stage_par, abort_flag, p.status, kSiteFull);
+              // ... and the tile's accumulator slot must have been read for the last time
+              ok = mbar_wait(&tempty[ib * kItemTiles + t], use_par ^ 1, abort_flag, p.status, kSiteTEmpty);
               if (!ok) break;
               tc_fence_after();
               const uint32_t k_lo = k_lo0 + (uint32_t)stage * (SL::kStageBytes >> 4);
@@ -464,6 +480,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
               }
               // one commit per tile: the accumulator is ready for the epilogue, and the K stage may be refilled
               umma_commit(&tfull[ib * kItemTiles + t]);
+            } else {
+              mbar_arrive(&seen[stage]);  // this warp has taken the stage's phase; it may be refilled
             }
             turn ^= 1;
             if (++stage == kStages) {
@@ -814,8 +832,8 @@ int launch_score_tc(const madakv_config& c, const void* q, madakv_strides sq, co
   const int grid = (int)(total < sms ? total : sms);
   // Phase 1 leads phase 2 by two work items per CTA: the K chunks in between (2 * grid items of 256 KB) stay within
   // the L2. A longer lead only spills the L2, and leads beyond two items per CTA are not used at all: in a run of
-  // the whole pass with a lead of three and more items per CTA the device reported a launch failure whose cause was
-  // not found. The lead must cover a whole unit (all its phase-1 items come before its first phase-2 item);
+  // the whole pass with a lead of three and more items per CTA (and MMA warps that did not yet take every stage
+  // barrier in order) the device reported a launch failure. The lead must cover a whole unit (all its phase-1 items come before its first phase-2 item);
   // sequences too long for that take the generic path. MADAKV_SCORE_LAG (tests) can shorten the lead.
   int lag = 2 * grid;
   if (const char* e = getenv("MADAKV_SCORE_LAG")) {

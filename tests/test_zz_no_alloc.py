@@ -32,7 +32,7 @@ def test_static_scratch_decode_matches_workspace_decode(name):
     buf = mk.EvictionBuffers(cfg, capacity_of(wl))
     buf.run_eviction(inp["q_win"], inp["k"], inp["v"], inp["mask"], inp["seq_len"], inp["budget"])
     assert mk.madakv_poll_status(buf.ws) == 0
-    assert int(buf.kept_len.max()) > 512, "the case must span several splits"
+    assert int(buf.kept_len.max()) > 256, "the case must span several splits"
     for step, layer in ((0, -1), (1, -1), (2, wl.L - 1)):  # calls in a row on the shared scratch
         q = synth.make_decode_step(wl, step)[0].cuda()
         want, want_lse = torch.zeros_like(buf.out), torch.zeros_like(buf.lse_dec)
@@ -47,7 +47,7 @@ def test_static_scratch_decode_matches_workspace_decode(name):
 
 
 def test_static_scratch_limit_is_reported():
-    # 64 layers * 64 query heads * 17 splits * 130 floats * 4 B > 16 MiB: refused on the host, nothing is launched
+    # 64 layers * 64 query heads * 33 splits * 130 floats * 4 B > 16 MiB: refused on the host, nothing is launched
     wl = synth.scaled(TINY, dtype="bf16", L=64, Hq=64, Hkv=64, d=128, n=8192)
     cfg = config_of(wl)
     dummy = torch.zeros(4096, dtype=torch.bfloat16, device="cuda").view(-1, 128)
