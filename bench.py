@@ -26,8 +26,6 @@ from paper_2506_15724_b200 import synth  # noqa: E402
 
 METRIC = "prompt tokens evicted/sec"
 UNIT = "tokens/s"
-# kernels launched per step: score 3 (stats, reduce, psi) or 1 (fused), allocate 2, select 3, compact 1,
-# decode 3 (append, partial, merge)
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -40,54 +38,94 @@ def measured_peaks():
 
 
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    """Samples SM clock, power and throttle reasons of one GPU while the timed region runs (read-only NVML queries
+    from a thread, every ~2 ms; nvidia-smi polling as a fallback when NVML cannot be loaded)."""
+    SMI_FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+                  "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+                  "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index):
-        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        import threading
+
+        self.samples, self.reasons, self.max_mhz, self.proc, self.thread = [], set(), None, None, None
+        self._stop = threading.Event()
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms",
-                 "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+            import pynvml
+
+            pynvml.nvmlInit()
+            h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            bits = {
+                "hw_slowdown": getattr(pynvml, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+                "hw_thermal_slowdown": getattr(pynvml, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+                "sw_thermal_slowdown": getattr(pynvml, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+                "sw_power_cap": getattr(pynvml, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+            }
+
+            def loop():
+                while not self._stop.is_set():
+                    try:
+                        self.samples.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                        r = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                        for name, bit in bits.items():
+                            if r & bit:
+                                self.reasons.add(name)
+                    except Exception:
+                        pass
+                    time.sleep(0.002)
+
+            self.thread = threading.Thread(target=loop, daemon=True)
+            self.thread.start()
         except Exception:
-            self.proc = None
+            self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            try:
+                self.proc = subprocess.Popen(
+                    ["nvidia-smi", "-i", str(index), f"--query-gpu={self.SMI_FIELDS}", "--format=csv,noheader,nounits",
+                     "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+            except Exception:
+                self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
-            return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        self.tmp.flush()
-        self.tmp.seek(0)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.tmp.read().splitlines():
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 7:
-                continue
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "source": "nvml"}
+        if self.thread is not None:
+            self._stop.set()
+            self.thread.join(timeout=2)
+        elif self.proc is not None:
+            out["source"] = "nvidia-smi"
+            self.proc.terminate()
             try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
-            except ValueError:
-                continue
-            for nm, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        self.tmp.close()
-        os.unlink(self.tmp.name)
-        if sm:
-            sm.sort()
-            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+            self.tmp.flush()
+            self.tmp.seek(0)
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            mx = []
+            for line in self.tmp.read().splitlines():
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    self.samples.append(float(parts[0]))
+                    mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for nm, val in zip(names, parts[3:7]):
+                    if val.lower().startswith("active"):
+                        self.reasons.add(nm)
+            self.tmp.close()
+            os.unlink(self.tmp.name)
+            if mx:
+                out["sm_max_mhz"] = max(mx)
+        if self.samples:
+            sm = sorted(self.samples)
+            out.update(sm_mhz=sm[len(sm) // 2], reasons=sorted(self.reasons), samples=len(sm))
         return out
 
 
 def cpu_oracle_leg(wl, seconds_target=15.0):
-    """The oracle, as it stands, on a bounded sample of the workload: the first layers of the same inputs."""
+    """The oracle, as it stands, on a bounded sample of the workload: the first layers of the same inputs (all of
+    them when the whole workload fits the time target), repeated until about `seconds_target` of CPU work is done."""
     import numpy as np
 
     import oracle
@@ -96,35 +134,38 @@ def cpu_oracle_leg(wl, seconds_target=15.0):
         t = t.detach().cpu().contiguous()
         return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
 
-    layers = 1
-    sub = synth.scaled(wl, L=layers)
     code = 0 if wl.dtype == "f32" else 1
-    inp = synth.make_inputs(sub)
-    q, k, v = to_np(inp["q_win"]), to_np(inp["k"]), to_np(inp["v"])
-    mask, sl, bud = to_np(inp["mask"]), to_np(inp["seq_len"]), to_np(inp["budget"])
-    dq, kn, vn = [to_np(t) for t in synth.make_decode_step(sub, 0)]
-    cap = sub.units * (sub.n + sub.max_new_tokens)
 
-    def one_pass():
-        psi = oracle.score(code, q, k, sl).astype(np.float32)
-        al = oracle.allocate(psi, mask, sl, bud, wl.theta)
-        rc, kept_len, seg_off, kept_idx = oracle.select(psi, mask, sl, al["budgets"], headroom=sub.max_new_tokens,
-                                                        capacity=cap)
-        k_c, v_c = oracle.compact(code, k, v, kept_idx, seg_off, kept_len, cap)
-        oracle.decode(code, dq, kn, vn, k_c, v_c, seg_off, kept_len, Hkv=sub.Hkv)
+    def prepare(layers):
+        sub = synth.scaled(wl, L=layers)
+        inp = synth.make_inputs(sub)
+        q, k, v = to_np(inp["q_win"]), to_np(inp["k"]), to_np(inp["v"])
+        mask, sl, bud = to_np(inp["mask"]), to_np(inp["seq_len"]), to_np(inp["budget"])
+        dq, kn, vn = [to_np(t) for t in synth.make_decode_step(sub, 0)]
+        cap = sub.units * (sub.n + sub.max_new_tokens)
 
+        def one_pass():
+            psi = oracle.score(code, q, k, sl).astype(np.float32)
+            al = oracle.allocate(psi, mask, sl, bud, wl.theta)
+            rc, kept_len, seg_off, kept_idx = oracle.select(psi, mask, sl, al["budgets"], headroom=sub.max_new_tokens,
+                                                            capacity=cap)
+            k_c, v_c = oracle.compact(code, k, v, kept_idx, seg_off, kept_len, cap)
+            oracle.decode(code, dq, kn, vn, k_c, v_c, seg_off, kept_len, Hkv=sub.Hkv)
+
+        return sub, one_pass, int(sl.sum())
+
+    sub, one_pass, tokens = prepare(1)
     t0 = time.perf_counter()
     one_pass()
-    dt = time.perf_counter() - t0
-    reps = 1
-    if dt < seconds_target / 4:
-        extra = max(1, min(8, int(seconds_target / max(dt, 1e-3)) - 1))
-        t0 = time.perf_counter()
-        for _ in range(extra):
-            one_pass()
-        dt = (time.perf_counter() - t0) / extra
-        reps = extra
-    tokens = int(sl.sum())
+    t1 = time.perf_counter() - t0
+    layers = int(max(1, min(wl.L, seconds_target / 2 / max(t1, 1e-3))))
+    if layers > 1:
+        sub, one_pass, tokens = prepare(layers)
+    reps = int(max(1, min(16, seconds_target / max(t1 * layers, 1e-3))))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        one_pass()
+    dt = (time.perf_counter() - t0) / reps
     value = tokens * (layers / wl.L) / dt  # tokens/s of the full-depth pass at the sampled layers' rate
     return {
         "value": value, "unit": UNIT, "cores": oracle.hardware_threads(), "kind": "oracle",
@@ -159,7 +200,7 @@ def run_reference(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="llava", choices=list(synth.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -357,7 +398,7 @@ def main():
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms},
-        "gpu_launches": args.steps * LAUNCHES_PER_STEP,
+        "gpu_launches": args.steps * launches_per_step(wl),
         "roofline": {"bound": "hbm", "kernel": "score stage (stage 1)", "achieved": score_gbs, "peak": peak,
                      "unit": "GB/s", "frac": score_gbs / peak, "traffic": TRAFFIC.get(wl.name), "peak_kind": peak_kind,
                      "algorithmic_bytes": k_bytes},
@@ -375,9 +416,17 @@ def main():
         dist.destroy_process_group()
 
 
-LAUNCHES_PER_STEP = 12
-# dram bytes (read + write) per launch of the dominant kernel from an ncu capture, per workload; None = not captured
-TRAFFIC = {}
+def launches_per_step(wl):
+    """Kernels of this library launched by one step: score 1 (tensor-core path) or 3 (generic path), allocate 2,
+    select 2, compact 1, decode 3 (append, partial, merge)."""
+    tc = wl.dtype == "bf16" and wl.g * wl.w <= 64
+    return (1 if tc else 3) + 2 + 2 + 1 + 3
+
+
+# dram bytes (read + write) per launch of the dominant kernel (score_tc), per workload, from the ncu capture summarised
+# in profiles/all_kernels_llava.md: 362.7 MB measured on the 4-layer case, times 8 for the 32 layers (traffic grows
+# with the number of units); None = not captured
+TRAFFIC = {"llava": 8 * 362.7e6}
 
 if __name__ == "__main__":
     main()
