@@ -141,6 +141,8 @@ int launch_score(const madakv_config& c, const void* q, madakv_strides sq, const
 bool score_tc_supported(const madakv_config& c, madakv_strides sq, madakv_strides sk);
 int launch_score_tc(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
                     const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st);
+int launch_score_cluster(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                         const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st);
 int launch_score_generic(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
                          const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st);
 int launch_allocate(const madakv_config& c, const float* psi, const uint8_t* mask, const int32_t* seq_len,

@@ -289,8 +289,12 @@ int launch_score_generic(const madakv_config& c, const void* q, madakv_strides s
 int launch_score(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
                  const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st) {
   if (score_tc_supported(c, sq, sk)) {
-    const int rc = launch_score_tc(c, q, sq, k, sk, seq_len, lse, psi, ws, st);
-    if (rc != MADAKV_EUNSUPPORTED) return rc;  // shapes the tensor-core path declines go the generic way
+    // tensor-core paths: logits resident in a cluster's TMEM when a unit fits, else the two-phase kernel; shapes
+    // they decline go the generic way
+    int rc = launch_score_cluster(c, q, sq, k, sk, seq_len, lse, psi, ws, st);
+    if (rc != MADAKV_EUNSUPPORTED) return rc;
+    rc = launch_score_tc(c, q, sq, k, sk, seq_len, lse, psi, ws, st);
+    if (rc != MADAKV_EUNSUPPORTED) return rc;
   }
   return launch_score_generic(c, q, sq, k, sk, seq_len, lse, psi, ws, st);
 }

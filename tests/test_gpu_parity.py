@@ -37,6 +37,9 @@ SHAPES = {
                                   theta=0.3),
     # many short sequences: work items of one to four tiles follow one another (accumulator slots and K stages
     # come round again within a few tiles)
+    # 8192 keys x 32 rows: a unit needs the TMEM of a 4-CTA cluster (ragged batch: shorter sequences use fewer tiles)
+    "tc_cluster4": synth.scaled(TINY, dtype="bf16", B=2, L=2, Hq=3, Hkv=3, d=128, n=8192, w=32, budget=900, theta=0.3,
+                                n_needles=8),
     "tc_short_seqs": synth.scaled(TINY, dtype="bf16", B=5, L=3, Hq=4, Hkv=4, d=128, n=389, w=8, budget=40, theta=0.3),
 }
 
@@ -57,7 +60,14 @@ def dev(inp):
 
 @pytest.mark.parametrize("name", list(SHAPES))
 @pytest.mark.parametrize("causal", [1, 0])
-def test_score_matches_oracle(name, causal):
+@pytest.mark.parametrize("path", ["auto", "twophase"])
+def test_score_matches_oracle(name, causal, path, monkeypatch):
+    # "auto": the library's own choice (for bf16 shapes with g * w <= 64 the TMEM-resident cluster kernel when a unit
+    # fits); "twophase": the two-phase tensor-core kernel is forced where a tensor-core path applies
+    if path == "twophase":
+        if not name.startswith("tc_"):
+            pytest.skip("no tensor-core path for this shape")
+        monkeypatch.setenv("MADAKV_SCORE_PATH", "twophase")
     wl = SHAPES[name]
     inp = make_case(wl)
     cfg = config_of(wl, causal=causal)
@@ -92,6 +102,7 @@ def test_tensor_core_score_item_interleaving(lag, monkeypatch):
     cfg = config_of(wl)
     g = dev(inp)
     buf = mk.EvictionBuffers(cfg, capacity_of(wl), want_lse=True)
+    monkeypatch.setenv("MADAKV_SCORE_PATH", "twophase")  # the kernel with the item schedule
     mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], buf.lse, buf.psi, buf.ws)
     assert mk.madakv_poll_status(buf.ws) == 0
     base = buf.psi.clone()
@@ -104,6 +115,12 @@ def test_tensor_core_score_item_interleaving(lag, monkeypatch):
     assert psi_close(buf.psi.cpu().numpy(), want, PSI_RTOL) < PSI_RTOL_SEEN
     monkeypatch.setenv("MADAKV_SCORE_PATH", "generic")
     mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], buf.lse, buf.psi, buf.ws)
+    assert psi_close(buf.psi.cpu().numpy(), want, PSI_RTOL) < PSI_RTOL_SEEN
+    monkeypatch.delenv("MADAKV_SCORE_PATH")  # the cluster kernel (8 units of 4096 keys: clusters of 2)
+    monkeypatch.delenv("MADAKV_SCORE_LAG")
+    buf.psi.fill_(-1.0)
+    mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], buf.lse, buf.psi, buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
     assert psi_close(buf.psi.cpu().numpy(), want, PSI_RTOL) < PSI_RTOL_SEEN
 
 
