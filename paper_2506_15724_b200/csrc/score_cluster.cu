@@ -6,13 +6,14 @@
 // (sequence, layer, KV head) at a time, CTA r computes the window-QK^T tiles of its share of the keys with tcgen05.mma
 // (128 keys of a tile on M, the g*w window rows on N, head_dim on K; operands by TMA, 128-byte swizzle) and KEEPS all
 // its fp32 accumulators in TMEM (512 columns = 16 tiles of 32 rows or 8 tiles of 64 rows). The epilogue warps read
-// them three times from TMEM: row maxima, sum of exp2 against the maxima, and, once the (max, sum) pairs of all warps
-// of the cluster have been exchanged through distributed shared memory and merged into the rows' log-sum-exps, the
+// them from TMEM as they arrive for the rows' (max, sum of exp2) statistics (one sweep with a running maximum for up
+// to 32 rows, a maximum sweep and a sum sweep for 64), and once more when the (max, sum) pairs of all warps of the
+// cluster have been exchanged through distributed shared memory and merged into the rows' log-sum-exps, for the
 // weights exp2(s - lse) whose sum over rows is psi. So K is read from HBM exactly once and each tile takes one MMA pass.
 //
 // Warp roles per CTA: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 epilogue (two groups of four
 // warps = the four TMEM lane quarters; group e takes the CTA's tiles of parity e; a thread owns one key of a tile and
-// all window rows of it). A tile's TMEM slot is handed back to the MMA warp after its third read, so the MMAs of the
+// all window rows of it). A tile's TMEM slot is handed back to the MMA warp after its last read, so the MMAs of the
 // next unit start while the last sweep of this one is still running; the TMA ring runs ahead across units.
 // Synchronisation between CTAs exists only inside a cluster (whose CTAs are co-scheduled by the hardware): every lane
 // of every epilogue warp stores its rows' pairs into each peer's shared memory and arrives on that peer's mbarrier.
@@ -32,6 +33,7 @@ struct ClParams {
   float* lse_out;   // natural log [B,L,Hq,w] or null
   int32_t* status;  // ws header
   int units, L, Hq, Hkv, g, w, R, n_max, causal, C;
+  int per_max, sets;  // most tiles a CTA gets of one unit; how many such tile sets fit its TMEM (units alternate sets)
   float scale2;
 };
 
@@ -59,9 +61,12 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
 __device__ __forceinline__ void st_remote_f2(uint32_t raddr, float a, float b) {
   asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(raddr), "f"(a), "f"(b) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t raddr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(raddr) : "memory");
+// Arrive on a peer's barrier without ordering of its own: the caller has fenced its stores at cluster scope once for
+// all peers (a releasing arrive per peer would wait for the remote stores one round trip at a time).
+__device__ __forceinline__ void mbar_arrive_remote_relaxed(uint32_t raddr) {
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(raddr) : "memory");
 }
+__device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_try_cluster(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -166,6 +171,9 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
     tile0 = rank * per;
     my_tiles = max(0, min(per, tiles - tile0));
   };
+  // first TMEM slot of the unit: consecutive units of the cluster take alternate sets of slots when two sets fit, so
+  // that the MMAs of the next unit do not have to wait for this unit's last sweep
+  auto slot_base_of = [&](int u) { return (((u - cluster) / n_clusters) % p.sets) * p.per_max; };
 
   if (warp == 0) {
     // ================================================================ TMA producer
@@ -188,6 +196,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
         int tile0, my_tiles;
         my_share(n, tile0, my_tiles);
         if (my_tiles == 0) continue;
+        const int sb = slot_base_of(u);
         ok = mbar_wait(&qempty[qi], q_par ^ 1, abort_flag, p.status, kSiteQEmpty);
         if (!ok) break;
         mbar_expect_tx(&qfull[qi], (uint32_t)(p.R * 128 * kKBlocks));
@@ -195,7 +204,8 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
           tma_load_5d(q_s + qi * SL::kQBytes + kb * NPAD * 128, &tmap_q, &qfull[qi], kb * 64, 0, h * p.g, l, b, pol_q);
         qi ^= 1;
         if (qi == 0) q_par ^= 1;
-        for (int j = 0; j < my_tiles; ++j) {
+        for (int jj = 0; jj < my_tiles; ++jj) {
+          const int j = sb + jj;  // slot
           const uint32_t prev = stage_user[stage];
           if (prev & 0x200u)
             ok = mbar_wait(&tfull[prev & 0xffu], (slot_par >> (prev & 0xffu)) & 1u, abort_flag, p.status, kSiteStage);
@@ -207,7 +217,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
           mbar_expect_tx(&full[stage], (uint32_t)SL::kStageBytes);
           for (int kb = 0; kb < kKBlocks; ++kb)
             tma_load_5d(k_s + stage * SL::kStageBytes + kb * kTileKeys * 128, &tmap_k, &full[stage], kb * 64,
-                        (tile0 + j) * kTileKeys, h, l, b, pol);
+                        (tile0 + jj) * kTileKeys, h, l, b, pol);
           if (++stage == kStages) stage = 0;
         }
       }
@@ -231,10 +241,12 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
         int tile0, my_tiles;
         my_share(n, tile0, my_tiles);
         if (my_tiles == 0) continue;
+        const int sb = slot_base_of(u);
         ok = mbar_wait(&qfull[qi], q_par, abort_flag, p.status, kSiteQFull);
         if (!ok) break;
         const uint32_t q_lo = q_lo0 + (uint32_t)qi * (SL::kQBytes >> 4);
-        for (int j = 0; j < my_tiles; ++j) {
+        for (int jj = 0; jj < my_tiles; ++jj) {
+          const int j = sb + jj;  // slot
           if (slot_used & (1u << j)) slot_par ^= 1u << j;
           slot_used |= 1u << j;
           const uint32_t use_par = (slot_par >> j) & 1u;
@@ -291,19 +303,20 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
       float* psi = p.psi + (int64_t)u * p.n_max;
       int tile0, my_tiles;
       my_share(n, tile0, my_tiles);
-      const int cnt = my_tiles > grp ? (my_tiles - grp + 1) / 2 : 0;  // this group's tiles: slots grp, grp + 2, ...
+      const int cnt = my_tiles > grp ? (my_tiles - grp + 1) / 2 : 0;  // this group's tiles: grp, grp + 2, ...
+      const int sb = slot_base_of(u);
       const int all_bound = (n >= p.w) ? (p.causal ? n - p.w + 1 : n) : 0;  // keys below are seen by every row
       if (rank == 0) {  // positions beyond the unit's last tile
         for (int key = ((n + kTileKeys - 1) / kTileKeys) * kTileKeys + ew * 32 + lane; key < p.n_max; key += 256)
           psi[key] = 0.f;
       }
       for (int i = 0; i < cnt; ++i) {  // parity of this use of the group's slots
-        const int j = grp + 2 * i;
+        const int j = sb + grp + 2 * i;
         if (slot_used & (1u << j)) slot_par ^= 1u << j;
         slot_used |= 1u << j;
       }
       auto wait_tile = [&](int i) -> bool {
-        const int j = grp + 2 * i;
+        const int j = sb + grp + 2 * i;
         const bool w_ok =
             __all_sync(0xffffffffu, mbar_wait(&tfull[j], (slot_par >> j) & 1u, abort_flag, p.status, kSiteTile));
         tc_fence_after();
@@ -311,7 +324,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
       };
       auto release_tile = [&](int i) {
         tc_fence_before();
-        mbar_arrive(&tempty[grp + 2 * i]);
+        mbar_arrive(&tempty[sb + grp + 2 * i]);
       };
       // The group's tiles are read in blocks of 16 window rows (16 TMEM columns); the load of the next block is in
       // flight while the current one is processed. `body(j, r, i)` gets block j of the group's i-th tile.
@@ -319,9 +332,9 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
         if (cnt == 0) return true;
         uint32_t ra[16], rb[16];
         if (!before_tile(0)) return false;
-        tmem_ld16_issue(tlane + grp * NPAD, ra);
+        tmem_ld16_issue(tlane + (sb + grp) * NPAD, ra);
         for (int i = 0; i < cnt; ++i) {
-          const uint32_t taddr = tlane + (grp + 2 * i) * NPAD;
+          const uint32_t taddr = tlane + (sb + grp + 2 * i) * NPAD;
 #pragma unroll
           for (int j = 0; j < kBlocks; j += 2) {
             tmem_ld_wait16(ra);
@@ -353,35 +366,74 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
       }
       __syncwarp();
 
-      // sweep 1: maximum of the raw logits per window row over this lane's keys
-      float st_m[NPAD];
-#pragma unroll
-      for (int c = 0; c < NPAD; ++c) st_m[c] = kEmptyMax;
-      ok = sweep([&](int i) { return wait_tile(i); },
-                 [&](int j, uint32_t (&r)[16], int i) {
-                   const int key0 = (tile0 + grp + 2 * i) * kTileKeys;
-                   if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
-#pragma unroll
-                   for (int c = 0; c < 16; ++c) st_m[j * 16 + c] = fmaxf(st_m[j * 16 + c], __uint_as_float(r[c]));
-                 });
-      if (!ok) break;
-      // sweep 2: sum of exp2 against the warp's maximum. The (negated, scaled) maxima are uniform over the warp: they
-      // go to the warp's shift_s and are read back as packed pairs, which keeps 32 registers free
       uint64_t z2[NPAD / 2];
+      if constexpr (NPAD == 32) {
+        // sweep 1 (as the tiles arrive): every lane keeps, per window row, a running maximum m and the sum z of
+        // exp2(s - m) over its keys. A new logit costs one exponential: e = exp2(-|s - m|), then z = z * e + 1 and
+        // m = s if s is the new maximum, else z += e. Afterwards the lanes' maxima are replaced by the warp's.
+        float st_m[NPAD], st_z[NPAD];
 #pragma unroll
-      for (int c = 0; c < NPAD; ++c) {
-        const float wm = warp_max(st_m[c]);
-        if (lane == (c & 31)) shift_s[c] = -(wm * p.scale2);
+        for (int c = 0; c < NPAD; ++c) {
+          st_m[c] = 4.f * kEmptyMax;  // below any (scaled) masked logit
+          st_z[c] = 0.f;
+        }
+        ok = sweep([&](int i) { return wait_tile(i); },
+                   [&](int j, uint32_t (&r)[16], int i) {
+                     const int key0 = (tile0 + grp + 2 * i) * kTileKeys;
+                     if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
+#pragma unroll
+                     for (int c = 0; c < 16; ++c) {
+                       const float t = __uint_as_float(r[c]) * p.scale2;
+                       const float d = t - st_m[j * 16 + c];
+                       const float e = ex2(-fabsf(d));
+                       if (d > 0.f) {
+                         st_z[j * 16 + c] = fmaf(st_z[j * 16 + c], e, 1.f);
+                         st_m[j * 16 + c] = t;
+                       } else {
+                         st_z[j * 16 + c] += e;
+                       }
+                     }
+                   });
+        if (!ok) break;
+#pragma unroll
+        for (int c = 0; c < NPAD; ++c) {
+          const float wm = warp_max(st_m[c]);
+          st_z[c] *= ex2(st_m[c] - wm);
+          if (lane == (c & 31)) shift_s[c] = -wm;
+        }
+#pragma unroll
+        for (int i = 0; i < NPAD / 2; ++i) z2[i] = pack2(st_z[2 * i], st_z[2 * i + 1]);
+        __syncwarp();
+      } else {
+        // sweep 1: maximum of the raw logits per window row over this lane's keys
+        float st_m[NPAD];
+#pragma unroll
+        for (int c = 0; c < NPAD; ++c) st_m[c] = kEmptyMax;
+        ok = sweep([&](int i) { return wait_tile(i); },
+                   [&](int j, uint32_t (&r)[16], int i) {
+                     const int key0 = (tile0 + grp + 2 * i) * kTileKeys;
+                     if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
+#pragma unroll
+                     for (int c = 0; c < 16; ++c) st_m[j * 16 + c] = fmaxf(st_m[j * 16 + c], __uint_as_float(r[c]));
+                   });
+        if (!ok) break;
+        // sweep 2: sum of exp2 against the warp's maximum. The (negated, scaled) maxima are uniform over the warp:
+        // they go to the warp's shift_s and are read back as packed pairs, which keeps registers free
+#pragma unroll
+        for (int c = 0; c < NPAD; ++c) {
+          const float wm = warp_max(st_m[c]);
+          if (lane == (c & 31)) shift_s[c] = -(wm * p.scale2);
+        }
+#pragma unroll
+        for (int i = 0; i < NPAD / 2; ++i) z2[i] = 0ull;
+        __syncwarp();
+        sweep([&](int) { return true; },
+              [&](int j, uint32_t (&r)[16], int i) {
+                const int key0 = (tile0 + grp + 2 * i) * kTileKeys;
+                if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
+                exp_accumulate16(r, scale2x, shift2 + j * 8, z2 + j * 8);
+              });
       }
-#pragma unroll
-      for (int i = 0; i < NPAD / 2; ++i) z2[i] = 0ull;
-      __syncwarp();
-      sweep([&](int) { return true; },
-            [&](int j, uint32_t (&r)[16], int i) {
-              const int key0 = (tile0 + grp + 2 * i) * kTileKeys;
-              if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
-              exp_accumulate16(r, scale2x, shift2 + j * 8, z2 + j * 8);
-            });
       // Sum over the 32 lanes through a padded shared-memory transpose (fixed order): lane j ends up with the sum of
       // row cb + j. It then stores the warp's (max, sum) of that row into every CTA of the cluster and arrives on
       // that CTA's barrier.
@@ -413,8 +465,10 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
 #pragma unroll
         for (int cb = 0; cb < NPAD; cb += 32)
           st_remote_f2(map_to_rank(smem_u32(my_stats + cb + lane), (uint32_t)peer), mine[cb / 32].x, mine[cb / 32].y);
-        mbar_arrive_remote(map_to_rank(smem_u32(&stats_bar[unit_par]), (uint32_t)peer));
       }
+      fence_cluster();  // this lane's stores to all peers come before its arrivals
+      for (int peer = 0; peer < C; ++peer)
+        mbar_arrive_remote_relaxed(map_to_rank(smem_u32(&stats_bar[unit_par]), (uint32_t)peer));
       // wait for the pairs of every warp of the cluster (bounded)
       {
         // the barrier completes once per two units: its phase parity for this unit is the parity of (units taken / 2)
@@ -440,14 +494,21 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
 #pragma unroll
       for (int cb = 0; cb < NPAD; cb += 32) {
         const int row = cb + lane;
+        // maximum first, then the sums rescaled to it, eight independent terms at a time (fixed order)
         const float2* src = stats + (size_t)unit_par * C * 8 * NPAD + row;
         float M = kEmptyMax, Z = 0.f;
         for (int e0 = 0; e0 < C * 8; e0 += 8) {
-          float2 v[8];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) v[j] = src[(size_t)(e0 + j) * NPAD];
+          for (int j = 0; j < 8; ++j) M = fmaxf(M, src[(size_t)(e0 + j) * NPAD].x);
+        }
+        for (int e0 = 0; e0 < C * 8; e0 += 8) {
+          float t[8];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) merge_stats(M, Z, v[j].x, v[j].y);
+          for (int j = 0; j < 8; ++j) {
+            const float2 v = src[(size_t)(e0 + j) * NPAD];
+            t[j] = v.y * ex2(v.x - M);  // an empty entry has sum 0
+          }
+          Z += ((t[0] + t[1]) + (t[2] + t[3])) + ((t[4] + t[5]) + (t[6] + t[7]));
         }
         const float lse2 = (Z > 0.f) ? M + log2f(Z) : 0.f;
         // negated for the exponent's fused multiply-add; padding rows get a huge shift (they add exp2(-huge) = 0)
@@ -514,6 +575,9 @@ int run_cluster(const CUtensorMap& mk, const CUtensorMap& mq, const ClParams& p,
     return MADAKV_EUNSUPPORTED;
   }
   const int clusters = min(min(max_clusters, sms / p.C), p.units);
+  if (getenv("MADAKV_DEBUG"))
+    fprintf(stderr, "madakv: score cluster kernel: cluster size %d, %d of at most %d clusters, %d B shared memory\n", p.C,
+            clusters, max_clusters, smem);
   cfg.gridDim = dim3((unsigned)(clusters * p.C));
   if (cudaLaunchKernelEx(&cfg, kern, mk, mq, p) != cudaSuccess) {
     cudaGetLastError();
@@ -524,14 +588,28 @@ int run_cluster(const CUtensorMap& mk, const CUtensorMap& mq, const ClParams& p,
 
 }  // namespace
 
-// The cluster size that makes the logits of the longest sequence fit, or 0 if none up to kMaxCluster does.
-static int cluster_size_for(const madakv_config& c) {
+// The cluster size for a shape, or 0 if the logits of the longest sequence do not fit the TMEM of kMaxCluster CTAs:
+// the smallest size whose per-CTA share of tiles fits. When that share fits twice, consecutive units use alternate
+// halves of the TMEM.
+static int cluster_size_for(const madakv_config& c, int* per_max, int* sets) {
   const int R = (c.n_q_heads / c.n_kv_heads) * c.window;
   const int npad = R <= 32 ? 32 : 64;
   const int slots = kTmemCols / npad;
   const int tiles = (c.max_seq_len + kTileKeys - 1) / kTileKeys;
-  for (int C = 1; C <= kMaxCluster; C *= 2)
-    if ((tiles + C - 1) / C <= slots) return C;
+  // Measured on the 8192-token workload: clusters of 8 (two sets) leave 28 of 148 SMs without a cluster and lose to
+  // clusters of 4 (one set), so the smallest cluster that fits is the default.
+  int first = 1;
+  if (const char* e = getenv("MADAKV_CLUSTER_SETS"))  // tests: 2 = prefer a cluster size where two sets fit
+    if (e[0] == '2') first = 2;
+  for (int want = first; want >= 1; --want)
+    for (int C = 1; C <= kMaxCluster; C *= 2) {
+      const int per = (tiles + C - 1) / C;
+      if (per * want <= slots) {
+        *per_max = per;
+        *sets = slots / per < 2 ? 1 : 2;
+        return C;
+      }
+    }
   return 0;
 }
 
@@ -539,7 +617,8 @@ int launch_score_cluster(const madakv_config& c, const void* q, madakv_strides s
                          const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st) {
   const int g = c.n_q_heads / c.n_kv_heads;
   if (c.dtype != MADAKV_BF16 || g * c.window > 64) return MADAKV_EUNSUPPORTED;
-  const int C = cluster_size_for(c);
+  int per_max = 0, sets = 0;
+  const int C = cluster_size_for(c, &per_max, &sets);
   if (C == 0) return MADAKV_EUNSUPPORTED;
   if (const char* e = getenv("MADAKV_SCORE_PATH"))
     if (e[0] == 't') return MADAKV_EUNSUPPORTED;  // tests: force the two-phase kernel
@@ -558,6 +637,8 @@ int launch_score_cluster(const madakv_config& c, const void* q, madakv_strides s
   p.n_max = c.max_seq_len;
   p.causal = c.causal;
   p.C = C;
+  p.per_max = per_max;
+  p.sets = sets;
   p.scale2 = scale_of(c) * kLog2e;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
