@@ -305,3 +305,60 @@ def test_strided_kv_layout():
     b.run_eviction(g["q_win"], kv, vv, g["mask"], g["seq_len"], g["budget"])
     assert torch.equal(a.psi, b.psi) and torch.equal(a.kept_idx, b.kept_idx)
     assert torch.equal(a.k_c, b.k_c) and torch.equal(a.v_c, b.v_c)
+
+
+def test_full_size_llava_workload_sampled():
+    """The benchmark workload at full size (32 layers x 32 heads x 8192 tokens, the launch configuration bench.py
+    times): scores of sampled units against the oracle, everything downstream of the scores exactly (the oracle's
+    allocation and selection re-run on all 1024 units of the CUDA path's scores; compacted rows and the decode
+    output on sampled units)."""
+    wl = synth.CONFIGS["llava"]
+    inp = synth.make_inputs(wl, device="cuda")
+    cfg = config_of(wl)
+    cap = wl.units * (min(wl.n, 2 * wl.budget) + wl.max_new_tokens)
+    buf = mk.EvictionBuffers(cfg, cap, want_lse=True)
+    mk.madakv_score(cfg, inp["q_win"], inp["k"], inp["seq_len"], buf.lse, buf.psi, buf.ws)
+    mk.madakv_allocate(cfg, buf.psi, inp["mask"], inp["seq_len"], inp["budget"], buf.mass, buf.pref, buf.demand, buf.phi,
+                       buf.budgets, buf.ws)
+    mk.madakv_select(cfg, buf.psi, inp["mask"], inp["seq_len"], buf.budgets, buf.kept_len, buf.seg_off, buf.kept_idx,
+                     buf.ws)
+    mk.madakv_compact(cfg, inp["k"], inp["v"], buf.kept_idx, buf.seg_off, buf.kept_len, buf.k_c, buf.v_c, buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    psi = buf.psi.cpu().numpy()
+    mask, sl, bud = to_np(inp["mask"]), to_np(inp["seq_len"]), to_np(inp["budget"])
+    # scores and log-sum-exps of sampled units (first, middle, last layers; a few heads each)
+    rng = np.random.RandomState(7)
+    for l in (0, 13, wl.L - 1):
+        hs = sorted(rng.choice(wl.Hkv, size=3, replace=False).tolist())
+        q_sub = to_np(inp["q_win"][:, l:l + 1, hs])
+        k_sub = to_np(inp["k"][:, l:l + 1, hs])
+        want, want_lse = oracle.score(1, q_sub, k_sub, sl, want_lse=True)
+        worst = psi_close(psi[:, l:l + 1, hs], want, PSI_RTOL)
+        assert worst < PSI_RTOL_SEEN, worst
+        np.testing.assert_allclose(buf.lse.cpu().numpy()[:, l:l + 1, hs], want_lse, rtol=0, atol=2e-5)
+    np.testing.assert_allclose(psi.sum(-1), wl.g * wl.w, rtol=1e-5)  # every softmax row sums to 1
+    # stages 2-4a on all units: bit-exact functions of the fp32 scores
+    al = oracle.allocate(psi, mask, sl, bud, float(np.float32(cfg.theta)))
+    for key in ("mass", "pref", "demand", "phi", "budgets"):
+        assert np.array_equal(getattr(buf, key).cpu().numpy(), al[key]), key
+    rc, kept_len, seg_off, kept_idx = oracle.select(psi, mask, sl, al["budgets"], headroom=wl.max_new_tokens,
+                                                    capacity=cap)
+    assert rc == 0
+    assert np.array_equal(buf.kept_len.cpu().numpy(), kept_len)
+    assert np.array_equal(buf.seg_off.cpu().numpy(), seg_off)
+    assert_segments_equal(kept_len, seg_off, buf.kept_idx.cpu().numpy(), kept_idx, "kept_idx")
+    # stage 4b and decode on sampled units: gathered rows are the kept rows; attention against the oracle
+    q, kn, vn = synth.make_decode_step(wl, 0, device="cuda")
+    buf.run_decode(q, None, None)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    k5 = inp["k"].view(wl.units, wl.n, wl.d)
+    v5 = inp["v"].view(wl.units, wl.n, wl.d)
+    out = buf.out.float().cpu().numpy().reshape(wl.units, wl.d)
+    for u in rng.choice(wl.units, size=6, replace=False).tolist() + [0, wl.units - 1]:
+        a, b = int(seg_off[u]), int(seg_off[u] + kept_len[u])
+        idx = torch.from_numpy(kept_idx[a:b].astype(np.int64)).cuda()
+        assert torch.equal(buf.k_c[a:b], k5[u][idx]) and torch.equal(buf.v_c[a:b], v5[u][idx]), u
+        kc, vc = to_np(buf.k_c[a:b]), to_np(buf.v_c[a:b])
+        rc, want, _ = oracle.decode(1, to_np(q.view(wl.units, 1, 1, wl.d)[u:u + 1]), None, None, kc, vc,
+                                    np.array([0, b - a], np.int64), np.array([b - a], np.int32), Hkv=1)
+        assert np.abs(out[u] - want.reshape(-1)).max() <= DEC_ATOL["bf16"], u
