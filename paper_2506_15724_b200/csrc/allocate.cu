@@ -41,7 +41,8 @@ __device__ __forceinline__ void hist_add(Hist& h, int bucket, u64 m) {
   atomicAdd(&h.cnt[bucket], 1u);
   const unsigned int add = (unsigned int)m;
   const unsigned int old = atomicAdd(&h.mlo[bucket], add);
-  atomicAdd(&h.mhi[bucket], (unsigned int)(m >> 32) + ((unsigned int)(old + add) < old ? 1u : 0u));
+  const unsigned int hi = (unsigned int)(m >> 32) + ((unsigned int)(old + add) < old ? 1u : 0u);
+  if (hi) atomicAdd(&h.mhi[bucket], hi);  // rare: importance values are mostly below 1, carries are few
 }
 __device__ __forceinline__ u64 hist_mass(const Hist& h, int bucket) {
   return ((u64)h.mhi[bucket] << 32) | h.mlo[bucket];
@@ -261,7 +262,23 @@ __global__ void alloc_seq_kernel(AllocParams p) {
   if (threadIdx.x == 0) s_nv = 0;
   __syncthreads();
   int c = 0;
-  for (int i = threadIdx.x; i < n; i += blockDim.x) c += p.mask[(int64_t)b * p.n_max + i] ? 1 : 0;
+  {
+    const uint8_t* mask = p.mask + (int64_t)b * p.n_max;
+    if ((reinterpret_cast<uintptr_t>(mask) & 15) == 0) {  // 16 tokens per load
+      const int n16 = n >> 4;
+      for (int i = threadIdx.x; i < n16; i += blockDim.x) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(mask) + i);
+        const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k)  // a byte counts if it is not zero
+          c += __popc(((w4[k] | (w4[k] >> 1) | (w4[k] >> 2) | (w4[k] >> 3) | (w4[k] >> 4) | (w4[k] >> 5) | (w4[k] >> 6) |
+                        (w4[k] >> 7)) & 0x01010101u));
+      }
+      for (int i = (n16 << 4) + threadIdx.x; i < n; i += blockDim.x) c += mask[i] ? 1 : 0;
+    } else {
+      for (int i = threadIdx.x; i < n; i += blockDim.x) c += mask[i] ? 1 : 0;
+    }
+  }
 #pragma unroll
   for (int off = 16; off >= 1; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
   if ((threadIdx.x & 31) == 0 && c) atomicAdd(&s_nv, c);
@@ -338,7 +355,7 @@ int launch_allocate(const madakv_config& c, const float* psi, const uint8_t* mas
   p.theta_fix = (u64)((double)c.theta * 4294967296.0);
   const int units = c.batch * c.n_layers * c.n_kv_heads;
   alloc_unit_kernel<<<units, NT, 0, st>>>(p);
-  alloc_seq_kernel<<<c.batch, 256, c.n_layers * (sizeof(double) + sizeof(long long)), st>>>(p);
+  alloc_seq_kernel<<<c.batch, 1024, c.n_layers * (sizeof(double) + sizeof(long long)), st>>>(p);
   return launch_status();
 }
 
