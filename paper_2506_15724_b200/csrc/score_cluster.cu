@@ -82,7 +82,7 @@ __device__ __forceinline__ void cluster_sync_all() {
 
 template <int D, int NPAD>
 struct ClSmem {
-  static constexpr int kStages = NPAD == 32 ? (D == 128 ? 4 : 8) : (D == 128 ? 2 : 4);  // 128 KB or 64 KB of K in flight
+  static constexpr int kStages = NPAD == 32 ? (D == 128 ? 5 : 10) : (D == 128 ? 3 : 6);  // 160 KB or 96 KB of K in flight
   static constexpr int kKBlocks = D / 64;
   static constexpr int kStageBytes = kTileKeys * D * 2;
   static constexpr int kQBytes = NPAD * D * 2;
@@ -95,8 +95,8 @@ struct ClSmem {
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   // misc: tmem base (4), abort flag (4), producer's stage ring (kStages <= 10 words)
   static constexpr int kWarpOff = kMiscOff + 48;
-  // per epilogue warp: shift[NPAD], vis[NPAD], a padded 32 x 33 transpose tile
-  static constexpr int kWarpBytes = NPAD * 4 + NPAD * 4 + 32 * 33 * 4;
+  // per epilogue warp: shift[NPAD], vis[NPAD]
+  static constexpr int kWarpBytes = NPAD * 4 + NPAD * 4;
   static constexpr int kStatsOff = kWarpOff + 8 * kWarpBytes;
   // exchanged (max, sum) pairs: [2 unit parities][C CTAs][8 warps][NPAD rows]
   static constexpr int stats_bytes(int C) { return 2 * C * 8 * NPAD * 8; }
@@ -290,7 +290,6 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
     uint8_t* wbase = smem + SL::kWarpOff + ew * SL::kWarpBytes;
     float* shift_s = reinterpret_cast<float*>(wbase);
     int* vis_s = reinterpret_cast<int*>(wbase + NPAD * 4);
-    float* tr = reinterpret_cast<float*>(wbase + NPAD * 8);
     const uint64_t* shift2 = reinterpret_cast<const uint64_t*>(shift_s);
     const uint64_t scale2x = pack2(p.scale2, p.scale2);
     const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16);
@@ -434,24 +433,17 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
                 exp_accumulate16(r, scale2x, shift2 + j * 8, z2 + j * 8);
               });
       }
-      // Sum over the 32 lanes through a padded shared-memory transpose (fixed order): lane j ends up with the sum of
+      // Sum over the 32 lanes by a transposing shuffle reduction (fixed order): lane j ends up with the sum of
       // row cb + j. It then stores the warp's (max, sum) of that row into every CTA of the cluster and arrives on
       // that CTA's barrier.
       float2* my_stats = stats + ((size_t)(unit_par * C + rank) * 8 + ew) * NPAD;
       float2 mine[NPAD / 32];
 #pragma unroll
       for (int cb = 0; cb < NPAD; cb += 32) {
+        float zv[32];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          float lo, hi;
-          unpack2(z2[cb / 2 + c], lo, hi);
-          tr[(2 * c) * 33 + lane] = lo;
-          tr[(2 * c + 1) * 33 + lane] = hi;
-        }
-        __syncwarp();
-        float zsum = 0.f;
-#pragma unroll
-        for (int i = 0; i < 32; ++i) zsum += tr[lane * 33 + i];
+        for (int c = 0; c < 16; ++c) unpack2(z2[cb / 2 + c], zv[2 * c], zv[2 * c + 1]);
+        float zsum = warp_rowsum32(zv);
         float m2 = -shift_s[cb + lane];
         // a row of which the whole warp saw no visible key summed exp2(0) for its masked entries: it is empty
         if (cnt == 0 || m2 < 0.5f * kEmptyMax * p.scale2) {
@@ -459,7 +451,6 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
           zsum = 0.f;
         }
         mine[cb / 32] = make_float2(m2, zsum);
-        __syncwarp();
       }
       for (int peer = 0; peer < C; ++peer) {
 #pragma unroll

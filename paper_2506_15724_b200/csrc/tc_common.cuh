@@ -162,6 +162,22 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Sum over the 32 lanes of 32 per-lane values, transposed: lane j returns the sum over all lanes of their v[j]. Five
+// exchange rounds (31 shuffles) in registers; the order of the additions is fixed (a tree over lane pairs).
+__device__ __forceinline__ float warp_rowsum32(float (&v)[32]) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) {
+    const bool up = (lane & m) != 0;
+#pragma unroll
+    for (int i = 0; i < m; ++i) {
+      const float keep = up ? v[i + m] : v[i];
+      const float send = up ? v[i] : v[i + m];
+      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, m);
+    }
+  }
+  return v[0];
+}
 // (max, sum) merge of two partial softmax statistics in the log2 domain.
 __device__ __forceinline__ void merge_stats(float& m, float& z, float mo, float zo) {
   const float mn = fmaxf(m, mo);
