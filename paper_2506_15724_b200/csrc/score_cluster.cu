@@ -6,8 +6,8 @@
 // (sequence, layer, KV head) at a time, CTA r computes the window-QK^T tiles of its share of the keys with tcgen05.mma
 // (128 keys of a tile on M, the g*w window rows on N, head_dim on K; operands by TMA, 128-byte swizzle) and KEEPS all
 // its fp32 accumulators in TMEM (512 columns = 16 tiles of 32 rows or 8 tiles of 64 rows). The epilogue warps read
-// them from TMEM as they arrive for the rows' (max, sum of exp2) statistics (one sweep with a running maximum for up
-// to 32 rows, a maximum sweep and a sum sweep for 64), and once more when the (max, sum) pairs of all warps of the
+// them from TMEM as they arrive for the rows' (max, sum of exp2) statistics (one sweep against a per-lane reference
+// logit for up to 32 rows, with an exact fallback; a maximum sweep and a sum sweep for 64), and once more when the (max, sum) pairs of all warps of the
 // cluster have been exchanged through distributed shared memory and merged into the rows' log-sum-exps, for the
 // weights exp2(s - lse) whose sum over rows is psi. So K is read from HBM exactly once and each tile takes one MMA pass.
 //
@@ -366,58 +366,22 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
       __syncwarp();
 
       uint64_t z2[NPAD / 2];
-      if constexpr (NPAD == 32) {
-        // sweep 1 (as the tiles arrive): every lane keeps, per window row, a running maximum m and the sum z of
-        // exp2(s - m) over its keys. A new logit costs one exponential: e = exp2(-|s - m|), then z = z * e + 1 and
-        // m = s if s is the new maximum, else z += e. Afterwards the lanes' maxima are replaced by the warp's.
-        float st_m[NPAD], st_z[NPAD];
-#pragma unroll
-        for (int c = 0; c < NPAD; ++c) {
-          st_m[c] = 4.f * kEmptyMax;  // below any (scaled) masked logit
-          st_z[c] = 0.f;
-        }
-        ok = sweep([&](int i) { return wait_tile(i); },
-                   [&](int j, uint32_t (&r)[16], int i) {
-                     const int key0 = (tile0 + grp + 2 * i) * kTileKeys;
-                     if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
-#pragma unroll
-                     for (int c = 0; c < 16; ++c) {
-                       const float t = __uint_as_float(r[c]) * p.scale2;
-                       const float d = t - st_m[j * 16 + c];
-                       const float e = ex2(-fabsf(d));
-                       if (d > 0.f) {
-                         st_z[j * 16 + c] = fmaf(st_z[j * 16 + c], e, 1.f);
-                         st_m[j * 16 + c] = t;
-                       } else {
-                         st_z[j * 16 + c] += e;
-                       }
-                     }
-                   });
-        if (!ok) break;
-#pragma unroll
-        for (int c = 0; c < NPAD; ++c) {
-          const float wm = warp_max(st_m[c]);
-          st_z[c] *= ex2(st_m[c] - wm);
-          if (lane == (c & 31)) shift_s[c] = -wm;
-        }
-#pragma unroll
-        for (int i = 0; i < NPAD / 2; ++i) z2[i] = pack2(st_z[2 * i], st_z[2 * i + 1]);
-        __syncwarp();
-      } else {
-        // sweep 1: maximum of the raw logits per window row over this lane's keys
+      // Exact statistics in two sweeps: the warp's maximum per row, then the sum of exp2 against it. The (negated,
+      // scaled) maxima are uniform over the warp: they go to the warp's shift_s and are read back as packed pairs.
+      auto exact_stats = [&]() -> bool {
         float st_m[NPAD];
 #pragma unroll
         for (int c = 0; c < NPAD; ++c) st_m[c] = kEmptyMax;
-        ok = sweep([&](int i) { return wait_tile(i); },
-                   [&](int j, uint32_t (&r)[16], int i) {
-                     const int key0 = (tile0 + grp + 2 * i) * kTileKeys;
-                     if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
+        const bool s_ok = sweep([&](int i) { return wait_tile(i); },
+                                [&](int j, uint32_t (&r)[16], int i) {
+                                  const int key0 = (tile0 + grp + 2 * i) * kTileKeys;
+                                  if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
 #pragma unroll
-                     for (int c = 0; c < 16; ++c) st_m[j * 16 + c] = fmaxf(st_m[j * 16 + c], __uint_as_float(r[c]));
-                   });
-        if (!ok) break;
-        // sweep 2: sum of exp2 against the warp's maximum. The (negated, scaled) maxima are uniform over the warp:
-        // they go to the warp's shift_s and are read back as packed pairs, which keeps registers free
+                                  for (int c = 0; c < 16; ++c)
+                                    st_m[j * 16 + c] = fmaxf(st_m[j * 16 + c], __uint_as_float(r[c]));
+                                });
+        if (!s_ok) return false;
+        __syncwarp();
 #pragma unroll
         for (int c = 0; c < NPAD; ++c) {
           const float wm = warp_max(st_m[c]);
@@ -432,6 +396,62 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
                 if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
                 exp_accumulate16(r, scale2x, shift2 + j * 8, z2 + j * 8);
               });
+        return true;
+      };
+      if constexpr (NPAD == 32) {
+        // One sweep as the tiles arrive: every lane takes, per window row, its logit of the group's first tile as the
+        // reference and sums exp2(s - reference) over its keys (the reference's own term is 1). No maximum is needed
+        // as long as no later logit lies ~100 binades above the reference; if a sum leaves that range (or a
+        // reference was a masked logit), the warp redoes the unit's statistics exactly. Afterwards the lanes'
+        // references are replaced by the warp's maximum of them.
+        uint64_t negm2[NPAD / 2];
+#pragma unroll
+        for (int i = 0; i < NPAD / 2; ++i) {
+          negm2[i] = pack2(-4.f * kEmptyMax, -4.f * kEmptyMax);  // no tile: reference below any masked logit
+          z2[i] = 0ull;
+        }
+        ok = sweep([&](int i) { return wait_tile(i); },
+                   [&](int j, uint32_t (&r)[16], int i) {
+                     const int key0 = (tile0 + grp + 2 * i) * kTileKeys;
+                     if (key0 + kTileKeys > all_bound) mask_block16(r, key0 + et, vis_s + j * 16);
+                     if (i == 0) {
+#pragma unroll
+                       for (int c = 0; c < 8; ++c)
+                         negm2[j * 8 + c] = pack2(-(__uint_as_float(r[2 * c]) * p.scale2),
+                                                  -(__uint_as_float(r[2 * c + 1]) * p.scale2));
+                     }
+                     exp_accumulate16(r, scale2x, negm2 + j * 8, z2 + j * 8);
+                   });
+        if (!ok) break;
+        float st_m[NPAD], st_z[NPAD];
+        bool bad = false;
+#pragma unroll
+        for (int i = 0; i < NPAD / 2; ++i) {
+          float a, b2;
+          unpack2(negm2[i], a, b2);
+          st_m[2 * i] = -a;
+          st_m[2 * i + 1] = -b2;
+          unpack2(z2[i], st_z[2 * i], st_z[2 * i + 1]);
+          bad = bad || !(st_z[2 * i] < 1.0e30f) || !(st_z[2 * i + 1] < 1.0e30f);  // also catches inf and NaN
+        }
+        if (__any_sync(0xffffffffu, bad)) {
+          ok = exact_stats();
+          if (!ok) break;
+        } else {
+          __syncwarp();
+#pragma unroll
+          for (int c = 0; c < NPAD; ++c) {
+            const float wm = warp_max(st_m[c]);
+            st_z[c] *= ex2(st_m[c] - wm);
+            if (lane == (c & 31)) shift_s[c] = -wm;
+          }
+#pragma unroll
+          for (int i = 0; i < NPAD / 2; ++i) z2[i] = pack2(st_z[2 * i], st_z[2 * i + 1]);
+          __syncwarp();
+        }
+      } else {
+        ok = exact_stats();
+        if (!ok) break;
       }
       // Sum over the 32 lanes by a transposing shuffle reduction (fixed order): lane j ends up with the sum of
       // row cb + j. It then stores the warp's (max, sum) of that row into every CTA of the cluster and arrives on

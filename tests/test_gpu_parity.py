@@ -362,3 +362,27 @@ def test_full_size_llava_workload_sampled():
         rc, want, _ = oracle.decode(1, to_np(q.view(wl.units, 1, 1, wl.d)[u:u + 1]), None, None, kc, vc,
                                     np.array([0, b - a], np.int64), np.array([b - a], np.int32), Hkv=1)
         assert np.abs(out[u] - want.reshape(-1)).max() <= DEC_ATOL["bf16"], u
+
+
+@pytest.mark.parametrize("path", ["auto", "twophase"])
+def test_score_with_logits_far_apart(path, monkeypatch):
+    # a softmax scale of 6 instead of 1/sqrt(d) spreads the logits over several hundred binades: sums of exp2 taken
+    # against anything but the true row maximum overflow, so the cluster kernel has to fall back to its exact
+    # two-sweep statistics; psi is then close to one-hot per window row
+    if path == "twophase":
+        monkeypatch.setenv("MADAKV_SCORE_PATH", "twophase")
+    wl = synth.scaled(TINY, dtype="bf16", B=2, L=2, Hq=4, Hkv=4, d=128, n=3000, w=32, budget=300, theta=0.3)
+    inp = make_case(wl)
+    cfg = config_of(wl, softmax_scale=6.0)
+    g = dev(inp)
+    buf = mk.EvictionBuffers(cfg, capacity_of(wl), want_lse=True)
+    mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], buf.lse, buf.psi, buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    want, want_lse = oracle.score(1, to_np(inp["q_win"]), to_np(inp["k"]), to_np(inp["seq_len"]), scale=6.0,
+                                  want_lse=True)
+    got = buf.psi.cpu().numpy()
+    assert np.isfinite(got).all()
+    # logits of several hundred: fp32 accumulation gives ~1e-4 relative on the big entries
+    psi_close(got, want, PSI_RTOL, atol=1e-6)
+    np.testing.assert_allclose(got.sum(-1), wl.g * wl.w, rtol=1e-4)
+    np.testing.assert_allclose(buf.lse.cpu().numpy(), want_lse, rtol=1e-5, atol=1e-3)
