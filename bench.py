@@ -423,10 +423,10 @@ def launches_per_step(wl):
     return (1 if tc else 3) + 2 + 2 + 1 + 3
 
 
-# dram bytes (read + write) per launch of the dominant kernel (score_tc), per workload, from the ncu capture summarised
-# in profiles/all_kernels_llava.md: 362.7 MB measured on the 4-layer case, times 8 for the 32 layers (traffic grows
-# with the number of units); None = not captured
-TRAFFIC = {"llava": 8 * 362.7e6}
+# dram bytes (read + write) per launch of the dominant kernel (score_cluster), per workload, from the ncu capture
+# summarised in profiles/all_kernels_llava.md: 274.4 MB measured on the 4-layer case, times 8 for the 32 layers
+# (traffic grows with the number of units); None = not captured
+TRAFFIC = {"llava": 8 * 274.4e6}
 
 if __name__ == "__main__":
     main()
