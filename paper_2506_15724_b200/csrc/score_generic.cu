@@ -296,6 +296,11 @@ int launch_score(const madakv_config& c, const void* q, madakv_strides sq, const
     rc = launch_score_tc(c, q, sq, k, sk, seq_len, lse, psi, ws, st);
     if (rc != MADAKV_EUNSUPPORTED) return rc;
   }
+  if (tc_device_ok()) {
+    // wide windows (64 < g * w <= 256): window rows on M, one row per epilogue thread
+    const int rc = launch_score_rows(c, q, sq, k, sk, seq_len, lse, psi, ws, st);
+    if (rc != MADAKV_EUNSUPPORTED) return rc;
+  }
   return launch_score_generic(c, q, sq, k, sk, seq_len, lse, psi, ws, st);
 }
 

@@ -557,11 +557,9 @@ int run_tc(const CUtensorMap& mk, const CUtensorMap& mq, const TcParams& p, int 
 
 }  // namespace
 
-bool score_tc_supported(const madakv_config& c, madakv_strides sq, madakv_strides sk) {
-  const int g = c.n_q_heads / c.n_kv_heads;
-  if (c.dtype != MADAKV_BF16 || g * c.window > 64 || c.window > 256 || g > 256) return false;
-  (void)sq;
-  (void)sk;
+// A tensor-core path can run at all: a compute-capability-10 device, the tensor-map encoder of the driver, and no
+// request for the generic path (MADAKV_SCORE_PATH=generic, tests).
+bool tc_device_ok() {
   int dev = 0, major = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess || major != 10)
@@ -569,6 +567,14 @@ bool score_tc_supported(const madakv_config& c, madakv_strides sq, madakv_stride
   const char* force = getenv("MADAKV_SCORE_PATH");
   if (force && force[0] == 'g') return false;
   return encode_fn() != nullptr;
+}
+
+bool score_tc_supported(const madakv_config& c, madakv_strides sq, madakv_strides sk) {
+  const int g = c.n_q_heads / c.n_kv_heads;
+  if (c.dtype != MADAKV_BF16 || g * c.window > 64 || c.window > 256 || g > 256) return false;
+  (void)sq;
+  (void)sk;
+  return tc_device_ok();
 }
 
 int launch_score_tc(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
