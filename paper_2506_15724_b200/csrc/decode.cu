@@ -13,6 +13,7 @@ namespace madakv {
 namespace {
 
 constexpr int NT = 128;
+constexpr int kDecodeGridX = 32;  // blocks per segment at most
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -32,6 +33,12 @@ struct DecodeParams {
   int L, Hq, Hkv, g, layer, splits;
   float scale2;
 };
+
+__device__ __forceinline__ float fast_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 __device__ __forceinline__ int unit_of(const DecodeParams& p, int y) {
   // y enumerates the (sequence, KV head) pairs of the selected layer, or all units when layer < 0
@@ -98,11 +105,9 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
   __shared__ float s_m[GROUPS][G], s_l[GROUPS][G];
 
   const int u = unit_of(p, blockIdx.y);
-  const int split = blockIdx.x;
   const int len = p.kept_len[u];
-  const int row_begin = split * kDecodeChunk;
-  if (row_begin >= len && !(split == 0)) return;  // split 0 always reports, so an empty segment is well defined
-  const int row_end = min(len, row_begin + kDecodeChunk);
+  // split 0 always reports, so an empty segment is well defined; a block beyond the segment has nothing to do
+  if (blockIdx.x != 0 && (int)blockIdx.x * kDecodeChunk >= len) return;
   const int64_t off = p.seg_off[u];
   const int h = u % p.Hkv, bl = u / p.Hkv;
   const int lane = threadIdx.x % LPR, grp = threadIdx.x / LPR;
@@ -118,6 +123,11 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
       for (int c = 0; c < EPL; ++c) qr[i][c] = 0.f;
     }
   }
+  // the grid has at most kDecodeGridX blocks per segment: a block takes splits blockIdx.x, blockIdx.x + gridDim.x, ...
+  // (segments of an evicted cache are a few splits long, those of a full cache hundreds)
+  for (int split = blockIdx.x; split == 0 || split * kDecodeChunk < len; split += gridDim.x) {
+  const int row_begin = split * kDecodeChunk;
+  const int row_end = min(len, row_begin + kDecodeChunk);
   float m[G], l[G], o[G][EPL];
 #pragma unroll
   for (int i = 0; i < G; ++i) {
@@ -149,24 +159,33 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
       float kf[EPL], vf[EPL];
       Vec16<T>::cvt(kraw[j], kf);
       Vec16<T>::cvt(vraw[j], vf);
+      // all heads of the group at once (heads beyond g have zero queries): the dot products, then the lane
+      // reductions of all heads interleaved, then the softmax updates, so that independent chains overlap
+      float sc[G];
 #pragma unroll
       for (int i = 0; i < G; ++i) {
-        if (i >= p.g) break;
         float s = 0.f;
 #pragma unroll
         for (int c = 0; c < EPL; ++c) s = fmaf(qr[i][c], kf[c], s);
+        sc[i] = s;
+      }
 #pragma unroll
-        for (int sh = LPR / 2; sh >= 1; sh >>= 1) s += __shfl_xor_sync(0xffffffffu, s, sh);
-        s *= p.scale2;
-        if (valid) {
+      for (int sh = LPR / 2; sh >= 1; sh >>= 1) {
+#pragma unroll
+        for (int i = 0; i < G; ++i) sc[i] += __shfl_xor_sync(0xffffffffu, sc[i], sh);
+      }
+      if (valid) {
+#pragma unroll
+        for (int i = 0; i < G; ++i) {
+          const float s = sc[i] * p.scale2;
           if (s > m[i]) {
-            const float f = exp2f(m[i] - s);
+            const float f = fast_ex2(m[i] - s);  // exp2(-inf) = 0 on the first row
             l[i] *= f;
 #pragma unroll
             for (int c = 0; c < EPL; ++c) o[i][c] *= f;
             m[i] = s;
           }
-          const float pw = exp2f(s - m[i]);
+          const float pw = fast_ex2(s - m[i]);
           l[i] += pw;
 #pragma unroll
           for (int c = 0; c < EPL; ++c) o[i][c] = fmaf(pw, vf[c], o[i][c]);
@@ -202,6 +221,8 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
       dst[D] = M;
       dst[D + 1] = Lsum;
     }
+  }
+  __syncthreads();  // the shared arrays are reused by the next split
   }
 }
 
@@ -246,7 +267,7 @@ int run(const DecodeParams& p, const madakv_config& c, cudaStream_t st) {
     append_kernel<D * (int)sizeof(T)><<<(n_sel * LPR + 127) / 128, 128, 0, st>>>(p, n_sel);
   }
   if (n_sel > 65535) return MADAKV_EUNSUPPORTED;
-  const dim3 grid(p.splits, n_sel);
+  const dim3 grid(p.splits < kDecodeGridX ? p.splits : kDecodeGridX, n_sel);
   if (p.g == 1) decode_partial_kernel<T, D, 1><<<grid, NT, 0, st>>>(p);
   else if (p.g == 2) decode_partial_kernel<T, D, 2><<<grid, NT, 0, st>>>(p);
   else if (p.g <= 4) decode_partial_kernel<T, D, 4><<<grid, NT, 0, st>>>(p);
