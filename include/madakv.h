@@ -142,7 +142,9 @@ int madakv_compact(const madakv_config* cfg, const void* k, const void* v, madak
  *   out[b,l,hq,:] = softmax( scale * q[b,l,hq,:] . K_seg^T ) V_seg for the g query heads of the group (Eq. 5)
  *   q, out [B,L,H_q,d] dtype contiguous; k_new, v_new [B,L,H_kv,d] dtype contiguous or both null;
  *   lse_out [B,L,H_q] fp32 or null. An empty segment gives out = 0, lse = -inf.
- * Accumulation is fp32; out is rounded to dtype once.                                                     */
+ * Accumulation is fp32; out is rounded to dtype once. With bf16 and 3 <= g <= 16 the products run on the tensor
+ * cores and the softmax weights enter the P V product rounded to bf16 (the denominator stays fp32).
+ * Supported: g <= 8 for fp32, g <= 16 for bf16; beyond that MADAKV_EUNSUPPORTED.                           */
 int madakv_decode_attn(const madakv_config* cfg, int32_t layer, const void* q, const void* k_new, const void* v_new,
                        void* k_c, void* v_c, const int64_t* seg_off, int32_t* kept_len, int64_t capacity, void* out,
                        float* lse_out, void* ws, size_t ws_bytes, void* stream);

@@ -3,7 +3,8 @@
 //   append   copies k_new / v_new behind every segment of the layer(s) and bumps kept_len
 //   partial  one block per (segment, split of kDecodeChunk rows): a group of LPR lanes owns a cache row (16 bytes
 //            per lane), the g query heads of the KV group share every K/V row read; online softmax in the log2
-//            domain, fp32 accumulation; the block's row groups are merged in shared memory
+//            domain, fp32 accumulation; the block's row groups are merged in shared memory. For bf16 caches with
+//            3 <= g <= 16 the same split is computed by decode_partial_mma_kernel on the tensor cores instead.
 //   merge    one block per query head: fixed-order combination of the split partials, rounding to dtype once
 #include <mutex>
 
@@ -226,6 +227,231 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
   }
 }
 
+// ---- grouped-query partial on the warp-level tensor-core path (bf16, 3 <= g <= 16) ----------------------------------
+// One K/V row serves g query heads: in scalar code that is 2 * g * D fused multiply-adds per 2 * D * 2 bytes read and
+// the kernel is bound by the FMA pipe from g = 4 on. Here the g heads sit on the 16 rows of an m16n8k16 tile (rows
+// beyond g carry zero queries): a warp takes 16 cache rows at a time, S = Q K^T as 2 key blocks x D/16 MMAs, the
+// online softmax on the accumulator fragments, P rounded to bf16 and reused in place as the A operand of O += P V
+// (D/8 MMAs). K and V rows go global -> shared with 16-byte asynchronous copies, double-buffered per warp, rows padded
+// by 16 bytes so that the 8x8 matrix loads are free of bank conflicts. Warps work independently on interleaved
+// 16-row chunks of the split and are merged in shared memory at its end.
+constexpr int kMmaWarps = 4;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+  const int bytes = valid ? 16 : 0;  // zero bytes read: the 16 destination bytes are filled with zeros
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+template <int D>
+struct MmaTile {
+  static constexpr int PITCH = D * 2 + 16;            // bytes from one staged row to the next
+  static constexpr int TILE = 16 * PITCH;             // 16 rows of K or of V
+  static constexpr int WARP = 4 * TILE;               // two buffers of (K, V)
+  static constexpr int OPITCH = D + 8;                // floats from one head's merged row to the next
+  static constexpr int BYTES = kMmaWarps * WARP;
+  static_assert(16 * OPITCH * 4 + 2 * 16 * 4 <= WARP, "the merge staging reuses a warp's K/V buffers");
+};
+
+template <int D>
+__global__ void __launch_bounds__(kMmaWarps * 32, 3) decode_partial_mma_kernel(DecodeParams p) {
+  using MT = MmaTile<D>;
+  constexpr int ROW_BYTES = D * 2;
+  constexpr int LPR = ROW_BYTES / 16;  // 16-byte pieces per row
+  constexpr int KC = D / 16;           // contraction chunks of Q K^T
+  constexpr int NB = D / 8;            // 8-column blocks of the output
+  extern __shared__ __align__(16) unsigned char dsmem[];
+
+  const int u = unit_of(p, blockIdx.y);
+  const int len = p.kept_len[u];
+  if (blockIdx.x != 0 && (int)blockIdx.x * kDecodeChunk >= len) return;
+  const int64_t off = p.seg_off[u];
+  const int h = u % p.Hkv, bl = u / p.Hkv;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int hr = lane / 4, t = lane % 4;  // fragment coordinates: row (head) hr and hr + 8, column pair t
+  unsigned char* wsm = dsmem + warp * MT::WARP;
+  const uint32_t wsm_a = smem_addr(wsm);
+
+  // Q as A fragments, one per contraction chunk: (head hr, d 2t..2t+1), (head hr+8, same), (head hr, d 2t+8..), ...
+  uint32_t qa[KC][4];
+  {
+    const __nv_bfloat16* q0 = reinterpret_cast<const __nv_bfloat16*>(p.q) + ((int64_t)bl * p.Hq + h * p.g) * D;
+#pragma unroll
+    for (int c = 0; c < KC; ++c) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int head = hr + 8 * (j & 1), dcol = c * 16 + 2 * t + 8 * (j >> 1);
+        qa[c][j] = head < p.g ? *reinterpret_cast<const uint32_t*>(q0 + (int64_t)head * D + dcol) : 0u;
+      }
+    }
+  }
+  const char* kc = (const char*)p.k_c + off * ROW_BYTES;
+  const char* vc = (const char*)p.v_c + off * ROW_BYTES;
+  // per-lane shared-memory offsets of the matrix loads: lanes 8i..8i+7 address the rows of the i-th 8x8 matrix
+  const int mi = lane / 8, mr = lane % 8;
+  const uint32_t k_lane = ((mi >> 1) * 8 + mr) * MT::PITCH + (mi & 1) * 16;  // keys (mi/2)*8.., d half mi%2
+  const uint32_t v_lane = ((mi & 1) * 8 + mr) * MT::PITCH + (mi >> 1) * 16;  // keys (mi%2)*8.., column block mi/2
+
+  for (int split = blockIdx.x; split == 0 || split * kDecodeChunk < len; split += gridDim.x) {
+    const int row_begin = split * kDecodeChunk;
+    const int row_end = min(len, row_begin + kDecodeChunk);
+    float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+    float o[NB][4];
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
+
+    auto load_chunk = [&](int r, int buf) {
+      const uint32_t kd = wsm_a + buf * 2 * MT::TILE, vd = kd + MT::TILE;
+#pragma unroll
+      for (int x = lane; x < 16 * LPR; x += 32) {
+        const int rr = x / LPR, cc = x % LPR;
+        const bool valid = r + rr < row_end;
+        const int64_t src = (int64_t)(valid ? r + rr : r) * ROW_BYTES + cc * 16;  // row r itself is always valid
+        cp_async16(kd + rr * MT::PITCH + cc * 16, kc + src, valid);
+        cp_async16(vd + rr * MT::PITCH + cc * 16, vc + src, valid);
+      }
+    };
+    if (row_begin + 16 * warp < row_end) load_chunk(row_begin + 16 * warp, 0);
+    cp_async_commit();
+    for (int it = 0;; ++it) {
+      const int r = row_begin + 16 * (warp + kMmaWarps * it);
+      if (r >= row_end) break;
+      const int buf = it & 1;
+      if (r + 16 * kMmaWarps < row_end) load_chunk(r + 16 * kMmaWarps, buf ^ 1);
+      cp_async_commit();
+      cp_async_wait<1>();
+      __syncwarp();
+      const uint32_t kb = wsm_a + buf * 2 * MT::TILE, vb = kb + MT::TILE;
+
+      float s[2][4];
+#pragma unroll
+      for (int b = 0; b < 2; ++b) s[b][0] = s[b][1] = s[b][2] = s[b][3] = 0.f;
+#pragma unroll
+      for (int c = 0; c < KC; ++c) {
+        uint32_t kf[4];
+        ldmatrix_x4(kb + k_lane + c * 32, kf);
+        mma_bf16_16816(s[0], qa[c], kf[0], kf[1]);
+        mma_bf16_16816(s[1], qa[c], kf[2], kf[3]);
+      }
+      // element j of block b: head hr + 8 * (j / 2), key r + 8 * b + 2 * t + (j & 1)
+#pragma unroll
+      for (int b = 0; b < 2; ++b)
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          s[b][j] = (r + 8 * b + 2 * t + (j & 1) < row_end) ? s[b][j] * p.scale2 : -INFINITY;
+      float f[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        float mx = fmaxf(fmaxf(s[0][2 * e], s[0][2 * e + 1]), fmaxf(s[1][2 * e], s[1][2 * e + 1]));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float mn = fmaxf(m[e], mx);  // finite: key r of the chunk is valid
+        f[e] = fast_ex2(m[e] - mn);        // exp2(-inf) = 0 on the first chunk
+        m[e] = mn;
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+          s[b][2 * e] = fast_ex2(s[b][2 * e] - mn);
+          s[b][2 * e + 1] = fast_ex2(s[b][2 * e + 1] - mn);
+        }
+        l[e] = l[e] * f[e] + ((s[0][2 * e] + s[0][2 * e + 1]) + (s[1][2 * e] + s[1][2 * e + 1]));
+      }
+      if (__any_sync(0xffffffffu, f[0] != 1.f || f[1] != 1.f)) {
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+          o[nb][0] *= f[0]; o[nb][1] *= f[0];
+          o[nb][2] *= f[1]; o[nb][3] *= f[1];
+        }
+      }
+      uint32_t pa[4];
+      pa[0] = pack_bf16x2(s[0][0], s[0][1]);
+      pa[1] = pack_bf16x2(s[0][2], s[0][3]);
+      pa[2] = pack_bf16x2(s[1][0], s[1][1]);
+      pa[3] = pack_bf16x2(s[1][2], s[1][3]);
+#pragma unroll
+      for (int nb = 0; nb < NB; nb += 2) {
+        uint32_t vf[4];
+        ldmatrix_x4_trans(vb + v_lane + nb * 16, vf);
+        mma_bf16_16816(o[nb], pa, vf[0], vf[1]);
+        mma_bf16_16816(o[nb + 1], pa, vf[2], vf[3]);
+      }
+      __syncwarp();  // the buffer is refilled two iterations on
+    }
+    cp_async_wait<0>();
+    __syncwarp();
+    // the warp's state goes to its own (now idle) staging area: o[16][D + 8], then m[16], l[16]
+    float* so = reinterpret_cast<float*>(wsm);
+    float* sm = so + 16 * MT::OPITCH;
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      l[e] += __shfl_xor_sync(0xffffffffu, l[e], 1);
+      l[e] += __shfl_xor_sync(0xffffffffu, l[e], 2);
+      if (t == 0) {
+        sm[hr + 8 * e] = m[e];
+        sm[16 + hr + 8 * e] = l[e];
+      }
+    }
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb) {
+      *reinterpret_cast<float2*>(so + hr * MT::OPITCH + nb * 8 + 2 * t) = make_float2(o[nb][0], o[nb][1]);
+      *reinterpret_cast<float2*>(so + (hr + 8) * MT::OPITCH + nb * 8 + 2 * t) = make_float2(o[nb][2], o[nb][3]);
+    }
+    __syncthreads();
+    for (int x = threadIdx.x; x < p.g * D; x += kMmaWarps * 32) {
+      const int i = x / D, c = x % D;
+      float mw[kMmaWarps], M = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < kMmaWarps; ++w) {
+        mw[w] = reinterpret_cast<const float*>(dsmem + w * MT::WARP)[16 * MT::OPITCH + i];
+        M = fmaxf(M, mw[w]);
+      }
+      float Lsum = 0.f, O = 0.f;
+#pragma unroll
+      for (int w = 0; w < kMmaWarps; ++w) {
+        const float* wo = reinterpret_cast<const float*>(dsmem + w * MT::WARP);
+        const float fw = (mw[w] == -INFINITY) ? 0.f : exp2f(mw[w] - M);
+        Lsum += wo[16 * MT::OPITCH + 16 + i] * fw;
+        O += wo[i * MT::OPITCH + c] * fw;
+      }
+      float* dst = p.part + (((int64_t)bl * p.Hq + h * p.g + i) * p.splits + split) * (D + 2);
+      dst[c] = O;
+      if (c == 0) {
+        dst[D] = M;
+        dst[D + 1] = Lsum;
+      }
+    }
+    __syncthreads();  // the staging areas become K/V buffers again
+  }
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(D) decode_merge_kernel(DecodeParams p) {
   // blockIdx.x enumerates the query heads of the selected layer(s)
@@ -268,7 +494,17 @@ int run(const DecodeParams& p, const madakv_config& c, cudaStream_t st) {
   }
   if (n_sel > 65535) return MADAKV_EUNSUPPORTED;
   const dim3 grid(p.splits < kDecodeGridX ? p.splits : kDecodeGridX, n_sel);
-  if (p.g == 1) decode_partial_kernel<T, D, 1><<<grid, NT, 0, st>>>(p);
+  bool mma = false;
+  if constexpr (sizeof(T) == 2) {
+    if (p.g >= 3 && p.g <= 16) {
+      mma = true;
+      cudaFuncSetAttribute(decode_partial_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           MmaTile<D>::BYTES);
+      decode_partial_mma_kernel<D><<<grid, kMmaWarps * 32, MmaTile<D>::BYTES, st>>>(p);
+    }
+  }
+  if (mma) {
+  } else if (p.g == 1) decode_partial_kernel<T, D, 1><<<grid, NT, 0, st>>>(p);
   else if (p.g == 2) decode_partial_kernel<T, D, 2><<<grid, NT, 0, st>>>(p);
   else if (p.g <= 4) decode_partial_kernel<T, D, 4><<<grid, NT, 0, st>>>(p);
   else if (p.g <= 8) decode_partial_kernel<T, D, 8><<<grid, NT, 0, st>>>(p);

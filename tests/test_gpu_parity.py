@@ -26,6 +26,8 @@ SHAPES = {
     "bf16_d128": synth.scaled(TINY, dtype="bf16", L=3, Hq=4, Hkv=4, d=128, n=1100, w=32, budget=200, theta=0.3,
                               n_needles=8),
     "bf16_gqa7": synth.scaled(TINY, dtype="bf16", L=2, Hq=14, Hkv=2, d=128, n=700, w=32, budget=150, theta=0.3),
+    # twelve query heads per KV head: both row halves of the decode kernel's 16-row tensor-core tile are live
+    "bf16_gqa12": synth.scaled(TINY, dtype="bf16", B=2, L=2, Hq=12, Hkv=1, d=128, n=900, w=8, budget=300, theta=0.3),
     "bf16_d64_long_window": synth.scaled(TINY, dtype="bf16", L=1, Hq=8, Hkv=2, d=64, n=2500, w=64, budget=300,
                                          theta=0.2),
     "f32_d128": synth.scaled(TINY, L=2, Hq=2, Hkv=1, d=128, n=450, w=8, budget=100),
