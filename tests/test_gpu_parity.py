@@ -309,12 +309,18 @@ def test_strided_kv_layout():
     assert torch.equal(a.k_c, b.k_c) and torch.equal(a.v_c, b.v_c)
 
 
-def test_full_size_llava_workload_sampled():
-    """The benchmark workload at full size (32 layers x 32 heads x 8192 tokens, the launch configuration bench.py
-    times): scores of sampled units against the oracle, everything downstream of the scores exactly (the oracle's
-    allocation and selection re-run on all 1024 units of the CUDA path's scores; compacted rows and the decode
-    output on sampled units)."""
-    wl = synth.CONFIGS["llava"]
+# sampled (layers, KV heads per layer, decode units) of the full-size checks: the oracle's share grows with g * w * n
+FULL_SIZE_SAMPLES = {"llava": ((0, 13, 31), 3, 6), "qwen": ((0, 27), 2, 4), "batched": ((5, 27), 1, 4),
+                     "long": ((0, 31), 1, 3)}
+
+
+@pytest.mark.parametrize("name", list(FULL_SIZE_SAMPLES))
+def test_full_size_workload_sampled(name):
+    """The four large workloads at full size, in the launch configuration bench.py times: scores of sampled units
+    against the oracle, everything downstream of the scores exactly (the oracle's allocation and selection re-run
+    on all units of the CUDA path's scores; compacted rows and the decode output on sampled units)."""
+    wl = synth.CONFIGS[name]
+    layers, n_heads, n_dec = FULL_SIZE_SAMPLES[name]
     inp = synth.make_inputs(wl, device="cuda")
     cfg = config_of(wl)
     cap = wl.units * (min(wl.n, 2 * wl.budget) + wl.max_new_tokens)
@@ -328,16 +334,17 @@ def test_full_size_llava_workload_sampled():
     assert mk.madakv_poll_status(buf.ws) == 0
     psi = buf.psi.cpu().numpy()
     mask, sl, bud = to_np(inp["mask"]), to_np(inp["seq_len"]), to_np(inp["budget"])
-    # scores and log-sum-exps of sampled units (first, middle, last layers; a few heads each)
+    # scores and log-sum-exps of sampled units (a few KV heads of a few layers, with the g query heads of each)
     rng = np.random.RandomState(7)
-    for l in (0, 13, wl.L - 1):
-        hs = sorted(rng.choice(wl.Hkv, size=3, replace=False).tolist())
-        q_sub = to_np(inp["q_win"][:, l:l + 1, hs])
+    for l in layers:
+        hs = sorted(rng.choice(wl.Hkv, size=n_heads, replace=False).tolist())
+        qs = [h * wl.g + i for h in hs for i in range(wl.g)]
+        q_sub = to_np(inp["q_win"][:, l:l + 1, qs])
         k_sub = to_np(inp["k"][:, l:l + 1, hs])
         want, want_lse = oracle.score(1, q_sub, k_sub, sl, want_lse=True)
         worst = psi_close(psi[:, l:l + 1, hs], want, PSI_RTOL)
         assert worst < PSI_RTOL_SEEN, worst
-        np.testing.assert_allclose(buf.lse.cpu().numpy()[:, l:l + 1, hs], want_lse, rtol=0, atol=2e-5)
+        np.testing.assert_allclose(buf.lse.cpu().numpy()[:, l:l + 1, qs], want_lse, rtol=0, atol=2e-5)
     np.testing.assert_allclose(psi.sum(-1), wl.g * wl.w, rtol=1e-5)  # every softmax row sums to 1
     # stages 2-4a on all units: bit-exact functions of the fp32 scores
     al = oracle.allocate(psi, mask, sl, bud, float(np.float32(cfg.theta)))
@@ -355,15 +362,18 @@ def test_full_size_llava_workload_sampled():
     assert mk.madakv_poll_status(buf.ws) == 0
     k5 = inp["k"].view(wl.units, wl.n, wl.d)
     v5 = inp["v"].view(wl.units, wl.n, wl.d)
-    out = buf.out.float().cpu().numpy().reshape(wl.units, wl.d)
-    for u in rng.choice(wl.units, size=6, replace=False).tolist() + [0, wl.units - 1]:
+    out = buf.out.float().cpu().numpy().reshape(wl.B * wl.L, wl.Hq, wl.d)
+    q3 = q.view(wl.B * wl.L, wl.Hq, wl.d)
+    for u in rng.choice(wl.units, size=n_dec, replace=False).tolist() + [0, wl.units - 1]:
         a, b = int(seg_off[u]), int(seg_off[u] + kept_len[u])
         idx = torch.from_numpy(kept_idx[a:b].astype(np.int64)).cuda()
         assert torch.equal(buf.k_c[a:b], k5[u][idx]) and torch.equal(buf.v_c[a:b], v5[u][idx]), u
         kc, vc = to_np(buf.k_c[a:b]), to_np(buf.v_c[a:b])
-        rc, want, _ = oracle.decode(1, to_np(q.view(wl.units, 1, 1, wl.d)[u:u + 1]), None, None, kc, vc,
+        bl, h = divmod(u, wl.Hkv)
+        heads = slice(h * wl.g, (h + 1) * wl.g)
+        rc, want, _ = oracle.decode(1, to_np(q3[bl, heads]).reshape(1, 1, wl.g, wl.d), None, None, kc, vc,
                                     np.array([0, b - a], np.int64), np.array([b - a], np.int32), Hkv=1)
-        assert np.abs(out[u] - want.reshape(-1)).max() <= DEC_ATOL["bf16"], u
+        assert np.abs(out[bl, heads] - want.reshape(wl.g, wl.d)).max() <= DEC_ATOL["bf16"], u
 
 
 @pytest.mark.parametrize("path", ["auto", "twophase"])
