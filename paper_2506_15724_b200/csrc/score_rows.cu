@@ -8,11 +8,14 @@
 //   pass 1  per (unit, key split): running maximum and sum of exp2 of every row over the split's keys, in-thread
 //           (per 16 columns: block maximum, one rescale, 16 exponentials); one (max, sum) pair per row and split
 //   merge   per (unit, row): the pairs of all splits -> the row's log-sum-exp (a separate small kernel)
-//   pass 2  per (unit, key split): logits recomputed, psi(i) = sum over rows of exp2(s - lse): a column sum over the
-//           lanes of all epilogue warps (transposing shuffle reduction per warp, then shared memory across warps)
+//   pass 2  per (unit, key split): logits recomputed with the tile turned back (128 keys on M, the window rows on N,
+//           as in the narrow-window kernels): a thread owns one key and psi(i) = sum over rows of exp2(s - lse) is an
+//           in-thread sum over the columns of its TMEM lane; the rows' negated log-sum-exps come as broadcast loads
 // K is streamed twice (the second time mostly from HBM): for these shapes the exponentials take longer than either
 // read. The passes are separate launches, so no CTA ever waits for another CTA. Warp roles: warp 0 TMA producer,
-// warp 1 MMA issuer and TMEM owner, warps 2-9 epilogue (row block = (warp - 2) / 4, TMEM lane quarter = warp % 4).
+// warp 1 MMA issuer and TMEM owner, warps 2-9 epilogue (pass 1: row block = (warp - 2) / 4; pass 2: the two groups
+// of four warps take alternate tiles, each group owning one of the two accumulator buffers; TMEM lane quarter =
+// warp % 4 in both).
 // Every wait is bounded: on expiry the kernel records MADAKV_ETIMEOUT, drains and returns.
 #include "tc_common.cuh"
 
@@ -26,9 +29,9 @@ struct RowParams {
   const int32_t* seq_len;
   float* psi;        // [units, n_max]
   float2* part;      // ws: [units, splits, rs] (max, sum) of every row over a split
-  const float* lse2; // ws: [units, rs] log2-domain log-sum-exp (pass 2)
+  const float* lse2; // ws: [units, rs] NEGATED log2-domain log-sum-exp, padding rows hold kEmptyMax (pass 2)
   int32_t* status;   // ws header
-  int units, L, Hq, Hkv, g, w, R, n_max, causal, splits, rs, mblocks;
+  int units, L, Hq, Hkv, g, w, R, n_max, causal, splits, rs, mblocks, n16;  // n16: R rounded up to 16
   float scale2;
 };
 
@@ -41,11 +44,11 @@ struct RowSmem {
   static constexpr int kKOff = 0;
   static constexpr int kQOff = kStages * kStageBytes;
   static constexpr int kBarOff = kQOff + kQBytes;
-  // full[kStages], empty[kStages], qfull, qempty, tfull[2], tempty[2], drain, ebar
+  // full[kStages], empty[kStages], qfull, qempty, tfull[2], tempty[2], drain
   static constexpr int kNumBars = 2 * kStages + 8;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-  static constexpr int kColOff = kMiscOff + 16;            // column sums [2 tile parities][8 warps][128 keys]
-  static constexpr int kTotal = kColOff + 2 * 8 * 128 * 4;
+  static constexpr int kColOff = kMiscOff + 16;            // window position (row % w) of every row [256]
+  static constexpr int kTotal = kColOff + 256 * 4;
   static constexpr int kAlloc = kTotal + 1024;
 };
 
@@ -71,13 +74,13 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   uint64_t* tfull = qempty + 1;        // [2]       MMA -> epilogue
   uint64_t* tempty = tfull + 2;        // [2]       epilogue -> MMA
   uint64_t* drain = tempty + 2;        // [1]
-  uint64_t* ebar = drain + 1;          // [1]       barrier of the epilogue threads (pass 2), bounded like every wait
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(smem + SL::kMiscOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::kMiscOff + 4);
-  float* colsum = reinterpret_cast<float*>(smem + SL::kColOff);
+  int* rowpos = reinterpret_cast<int*>(smem + SL::kColOff);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_epi = 128 * p.mblocks;  // epilogue threads in use
+  // pass 1: one thread per window row; pass 2: all 8 warps, a group of 4 (128 keys) per accumulator buffer
+  const int n_epi = PASS == 1 ? 128 * p.mblocks : 256;
   const int total_items = p.units * p.splits;
 
   if (threadIdx.x == 0) {
@@ -89,16 +92,16 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     mbar_init(qempty, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&tfull[i], 1);
-      mbar_init(&tempty[i], (uint32_t)n_epi);
+      mbar_init(&tempty[i], PASS == 1 ? (uint32_t)n_epi : 128u);
     }
     mbar_init(drain, 1);
-    mbar_init(ebar, (uint32_t)n_epi);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // rows R..255 of the Q buffer are never written by TMA: keep them zero so their logits are 0
   for (int x = threadIdx.x; x < SL::kQBytes / 16; x += kRowThreads)
     reinterpret_cast<uint4*>(q_s)[x] = make_uint4(0, 0, 0, 0);
+  for (int x = threadIdx.x; x < 256; x += kRowThreads) rowpos[x] = x % p.w;
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_s)),
@@ -182,13 +185,24 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
           if (!ok) break;
           tc_fence_after();
           const uint32_t k_lo = k_lo0 + (uint32_t)stage * (SL::kStageBytes >> 4);
-          for (int mb = 0; mb < p.mblocks; ++mb) {
-            const uint32_t d_tmem = tmem_base + buf * 256 + mb * 128;
+          if (PASS == 1) {  // D[row, key]: a row block of the queries is operand A, the K tile operand B
+            for (int mb = 0; mb < p.mblocks; ++mb) {
+              const uint32_t d_tmem = tmem_base + buf * 256 + mb * 128;
+#pragma unroll
+              for (int ks = 0; ks < D / 16; ++ks) {
+                const int kb = ks >> 2, kk = ks & 3;
+                umma_bf16(d_tmem, q_lo0 + ((kb * 256 * 128 + mb * 128 * 128 + kk * 32) >> 4),
+                          k_lo + ((kb * kTileKeys * 128 + kk * 32) >> 4), kIdescRows, ks > 0 ? 1u : 0u);
+              }
+            }
+          } else {  // D[key, row]: the K tile is operand A, all n16 query rows operand B
+            const uint32_t d_tmem = tmem_base + buf * 256;
+            const uint32_t idesc = instr_desc_bf16(p.n16);
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
               const int kb = ks >> 2, kk = ks & 3;
-              umma_bf16(d_tmem, q_lo0 + ((kb * 256 * 128 + mb * 128 * 128 + kk * 32) >> 4),
-                        k_lo + ((kb * kTileKeys * 128 + kk * 32) >> 4), kIdescRows, ks > 0 ? 1u : 0u);
+              umma_bf16(d_tmem, k_lo + ((kb * kTileKeys * 128 + kk * 32) >> 4),
+                        q_lo0 + ((kb * 256 * 128 + kk * 32) >> 4), idesc, ks > 0 ? 1u : 0u);
             }
           }
           umma_commit(&empty[stage]);  // the K stage may be refilled
@@ -207,8 +221,9 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         while (!mbar_try(drain, 0) && clock64() - t0 < 20000000ll) __nanosleep(200);
       }
     }
-  } else if ((warp - 2) >> 2 < p.mblocks) {
-    // ================================================================ epilogue: a thread owns one window row
+  } else if (PASS == 2 || (warp - 2) >> 2 < p.mblocks) {
+    // ================================================================ epilogue: a thread owns one window row (pass 1)
+    // or one key of every other tile (pass 2)
     const int ew = warp - 2;
     const int mb = ew >> 2;                        // row block
     const int quarter = warp & 3;                  // TMEM lanes [32 * quarter, 32 * quarter + 32)
@@ -217,7 +232,6 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16) + mb * 128;
     const float masked = kEmptyMax;                // raw value given to a logit the row may not see
     int n_tile = 0;
-    uint32_t e_par = 0;
     bool ok = true;
     for (int it = blockIdx.x; ok && it < total_items; it += gridDim.x) {
       const int item = PASS == 1 ? it : total_items - 1 - it;
@@ -287,54 +301,59 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
           p.part[((int64_t)u * p.splits + split) * p.rs + row] = none ? make_float2(kEmptyMax, 0.f) : make_float2(m, z);
         }
       } else {
-        // negated log-sum-exp for the exponent's fused multiply-add; padding rows get a huge shift (weight 0)
-        const float shift = row < p.R ? -__ldg(p.lse2 + (int64_t)u * p.rs + row) : kEmptyMax;
-        const uint64_t sh2 = pack2(shift, shift), sc2 = pack2(p.scale2, p.scale2);
+        // group (warp - 2) / 4 owns accumulator buffer `group` and with it every other tile; this thread's key is
+        // key0 + 32 * quarter + lane and its logits against the n16 window rows are the columns of its TMEM lane
+        const int group = ew >> 2;
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + group * 256;
+        const ulonglong2* ns = reinterpret_cast<const ulonglong2*>(p.lse2 + (int64_t)u * p.rs);
+        const uint64_t sc2 = pack2(p.scale2, p.scale2);
+        const int nblk = p.n16 >> 4;
         for (int t = 0; t < tiles; ++t, ++n_tile) {
-          const int buf = n_tile & 1;
-          ok = __all_sync(0xffffffffu, mbar_wait(&tfull[buf], (uint32_t)(n_tile >> 1) & 1u, abort_flag, p.status, kSiteTile));
+          if ((n_tile & 1) != group) continue;
+          ok = __all_sync(0xffffffffu, mbar_wait(&tfull[group], (uint32_t)(n_tile >> 1) & 1u, abort_flag, p.status, kSiteTile));
           if (!ok) break;
           tc_fence_after();
           const int key0 = key_begin + t * kTileKeys;
-          const uint32_t taddr = tlane + buf * 256;
-          float* cs = colsum + ((n_tile & 1) * 8 + ew) * 128;
+          const int key = key0 + quarter * 32 + lane;
+          // a tile below the window's first position is seen in full by every row; otherwise every logit is checked
+          const bool plain = key0 + kTileKeys <= n - p.w;
+          uint64_t acc = 0ull;
           uint32_t ra[16], rb[16];
-          float v[32];
-          auto block = [&](uint32_t (&r)[16], int c, float* out) {  // weights of columns 16c .. 16c + 15
+          auto block = [&](uint32_t (&r)[16], int c) {  // window rows 16c .. 16c + 15
+            uint64_t sh[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              float lo, hi;
-              unpack2(fma2(pack2u(r[2 * i], r[2 * i + 1]), sc2, sh2), lo, hi);
-              out[2 * i] = key0 + 16 * c + 2 * i < vis ? ex2(lo) : 0.f;
-              out[2 * i + 1] = key0 + 16 * c + 2 * i + 1 < vis ? ex2(hi) : 0.f;
+            for (int j = 0; j < 4; ++j) {
+              const ulonglong2 v = __ldg(ns + 4 * c + j);
+              sh[2 * j] = v.x;
+              sh[2 * j + 1] = v.y;
             }
+            if (!plain) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const int pos = n - p.w + rowpos[16 * c + i];
+                const int vis = pos < 0 ? 0 : (p.causal ? pos + 1 : n);
+                if (key >= vis) r[i] = __float_as_uint(kEmptyMax);
+              }
+            }
+            acc = exp_sum16(r, sc2, sh, acc);
           };
           tmem_ld16_issue(taddr, ra);
 #pragma unroll 1
-          for (int c = 0; c < 8; c += 2) {
+          for (int c = 0; c < nblk; c += 2) {
             tmem_ld_wait16(ra);
-            tmem_ld16_issue(taddr + (c + 1) * 16, rb);
-            block(ra, c, v);
-            tmem_ld_wait16(rb);
-            if (c + 2 < 8) tmem_ld16_issue(taddr + (c + 2) * 16, ra);
-            block(rb, c + 1, v + 16);
-            // sum over the warp's 32 rows: lane j gets the sum of column 16c + j
-            cs[16 * c + lane] = warp_rowsum32(v);
+            if (c + 1 < nblk) tmem_ld16_issue(taddr + (c + 1) * 16, rb);
+            block(ra, c);
+            if (c + 1 < nblk) {
+              tmem_ld_wait16(rb);
+              if (c + 2 < nblk) tmem_ld16_issue(taddr + (c + 2) * 16, ra);
+              block(rb, c + 1);
+            }
           }
           tc_fence_before();
-          mbar_arrive(&tempty[buf]);
-          // all warps' column sums of this tile must be in shared memory
-          mbar_arrive(ebar);
-          ok = __all_sync(0xffffffffu, mbar_wait(ebar, e_par, abort_flag, p.status, kSiteFlag));
-          e_par ^= 1;
-          if (!ok) break;
-          if (eidx < kTileKeys) {
-            const float* c0 = colsum + (n_tile & 1) * 8 * 128 + eidx;
-            float tot = 0.f;
-            for (int e2 = 0; e2 < 4 * p.mblocks; ++e2) tot += c0[e2 * 128];  // fixed order
-            const int key = key0 + eidx;
-            if (key < p.n_max) psi[key] = key < n ? tot : 0.f;
-          }
+          mbar_arrive(&tempty[group]);
+          float lo, hi;
+          unpack2(acc, lo, hi);
+          if (key < p.n_max) psi[key] = key < n ? lo + hi : 0.f;
         }
         if (!ok) break;
         // keys of the item beyond the sequence
@@ -353,11 +372,16 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   }
 }
 
-// merge: per (unit, row) the (max, sum) pairs of all splits, in split order -> log2-domain log-sum-exp
-__global__ void score_rows_merge_kernel(RowParams p, float* lse2, float* lse_out, int total) {
+// merge: per (unit, row) the (max, sum) pairs of all splits, in split order -> log2-domain log-sum-exp, stored
+// negated (pass 2 adds it inside a fused multiply-add); padding rows get a shift that turns every weight into 0
+__global__ void score_rows_merge_kernel(RowParams p, float* nlse2, float* lse_out, int total) {
   const int x = blockIdx.x * blockDim.x + threadIdx.x;
   if (x >= total) return;
-  const int u = x / p.R, row = x % p.R;
+  const int u = x / p.rs, row = x % p.rs;
+  if (row >= p.R) {
+    nlse2[x] = kEmptyMax;
+    return;
+  }
   const float2* part = p.part + (int64_t)u * p.splits * p.rs + row;
   float M = kEmptyMax;
   for (int s = 0; s < p.splits; ++s) M = fmaxf(M, part[(int64_t)s * p.rs].x);
@@ -367,7 +391,7 @@ __global__ void score_rows_merge_kernel(RowParams p, float* lse2, float* lse_out
     Z += v.y * exp2f(v.x - M);  // an empty split has sum 0
   }
   const float l2 = Z > 0.f ? M + log2f(Z) : 0.f;
-  lse2[(int64_t)u * p.rs + row] = l2;
+  nlse2[x] = -l2;
   if (lse_out) {
     const int h = u % p.Hkv, bl = u / p.Hkv;
     const int hq = h * p.g + row / p.w, wr = row % p.w;
@@ -385,7 +409,7 @@ int run_rows(const CUtensorMap& mk, const CUtensorMap& mq, RowParams p, float* l
           cudaSuccess)
     return MADAKV_ECUDA;
   score_rows_kernel<D, 1><<<grid, kRowThreads, SL::kAlloc, st>>>(mk, mq, p);
-  const int total = p.units * p.R;
+  const int total = p.units * p.rs;
   score_rows_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(p, lse2, lse_out, total);
   score_rows_kernel<D, 2><<<grid, kRowThreads, SL::kAlloc, st>>>(mk, mq, p);
   return launch_status();
@@ -418,6 +442,7 @@ int launch_score_rows(const madakv_config& c, const void* q, madakv_strides sq, 
   p.splits = (c.max_seq_len + kSplitKeys - 1) / kSplitKeys;
   p.rs = (R + 31) / 32 * 32;  // row stride of the workspace arrays
   p.mblocks = R <= 128 ? 1 : 2;
+  p.n16 = (R + 15) / 16 * 16;
   p.scale2 = scale_of(c) * kLog2e;
   // the partials reuse the generic path's region: one pair per (1024-key chunk, row) there, per (2048-key split,
   // padded row) here
