@@ -13,22 +13,24 @@
 //           in-thread sum over the columns of its TMEM lane; the rows' negated log-sum-exps come as broadcast loads
 // K is streamed twice (the second time mostly from HBM): for these shapes the exponentials take longer than either
 // read. The passes are separate launches, so no CTA ever waits for another CTA. Warp roles: warp 0 TMA producer,
-// warp 1 MMA issuer and TMEM owner, warps 2-9 epilogue (pass 1: row block = (warp - 2) / 4; pass 2: the two groups
-// of four warps take alternate tiles, each group owning one of the two accumulator buffers; TMEM lane quarter =
-// warp % 4 in both).
+// warp 1 MMA issuer and TMEM owner, warps 2-17 epilogue. Two warps share each (TMEM lane quarter, row block) of
+// pass 1 and each (lane quarter, accumulator buffer) of pass 2 and take one half of a tile's columns each: the
+// exponentials are latency-bound with two warps per scheduler, four keep the special-function unit busy. In pass 1
+// the halves publish separate (max, sum) pairs; in pass 2 the upper half hands its partial psi to the lower half
+// through shared memory. TMEM lane quarter = warp % 4 throughout.
 // Every wait is bounded: on expiry the kernel records MADAKV_ETIMEOUT, drains and returns.
 #include "tc_common.cuh"
 
 namespace madakv {
 namespace {
 
-constexpr int kRowThreads = 320;
+constexpr int kRowThreads = 576;  // 2 + 16 warps
 constexpr int kSplitKeys = 2048;  // keys per work item (16 tiles)
 
 struct RowParams {
   const int32_t* seq_len;
   float* psi;        // [units, n_max]
-  float2* part;      // ws: [units, splits, rs] (max, sum) of every row over a split
+  float2* part;      // ws: [units, splits, 2, rs] (max, sum) of every row over each half of a split's tiles
   const float* lse2; // ws: [units, rs] NEGATED log2-domain log-sum-exp, padding rows hold kEmptyMax (pass 2)
   int32_t* status;   // ws header
   int units, L, Hq, Hkv, g, w, R, n_max, causal, splits, rs, mblocks, n16;  // n16: R rounded up to 16
@@ -44,11 +46,12 @@ struct RowSmem {
   static constexpr int kKOff = 0;
   static constexpr int kQOff = kStages * kStageBytes;
   static constexpr int kBarOff = kQOff + kQBytes;
-  // full[kStages], empty[kStages], qfull, qempty, tfull[2], tempty[2], drain
-  static constexpr int kNumBars = 2 * kStages + 8;
+  // full[kStages], empty[kStages], qfull, qempty, tfull[2], tempty[2], drain, xbar[8]
+  static constexpr int kNumBars = 2 * kStages + 7 + 8;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kColOff = kMiscOff + 16;            // window position (row % w) of every row [256]
-  static constexpr int kTotal = kColOff + 256 * 4;
+  static constexpr int kXchOff = kColOff + 256 * 4;        // pass 2: partial psi of the upper column halves [2][128]
+  static constexpr int kTotal = kXchOff + 2 * 128 * 4;
   static constexpr int kAlloc = kTotal + 1024;
 };
 
@@ -74,13 +77,15 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   uint64_t* tfull = qempty + 1;        // [2]       MMA -> epilogue
   uint64_t* tempty = tfull + 2;        // [2]       epilogue -> MMA
   uint64_t* drain = tempty + 2;        // [1]
+  uint64_t* xbar = drain + 1;          // [8]       pass 2: upper half -> lower half of a (buffer, lane quarter) warp pair
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(smem + SL::kMiscOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::kMiscOff + 4);
   int* rowpos = reinterpret_cast<int*>(smem + SL::kColOff);
+  float* xch = reinterpret_cast<float*>(smem + SL::kXchOff);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // pass 1: one thread per window row; pass 2: all 8 warps, a group of 4 (128 keys) per accumulator buffer
-  const int n_epi = PASS == 1 ? 128 * p.mblocks : 256;
+  // epilogue threads in use. Pass 1: two per window row (column halves); pass 2: all 16 warps, 8 per accumulator buffer
+  const int n_epi = PASS == 1 ? 256 * p.mblocks : 512;
   const int total_items = p.units * p.splits;
 
   if (threadIdx.x == 0) {
@@ -92,9 +97,10 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     mbar_init(qempty, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&tfull[i], 1);
-      mbar_init(&tempty[i], PASS == 1 ? (uint32_t)n_epi : 128u);
+      mbar_init(&tempty[i], PASS == 1 ? (uint32_t)n_epi : 256u);
     }
     mbar_init(drain, 1);
+    for (int i = 0; i < 8; ++i) mbar_init(&xbar[i], 32);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -221,17 +227,19 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         while (!mbar_try(drain, 0) && clock64() - t0 < 20000000ll) __nanosleep(200);
       }
     }
-  } else if (PASS == 2 || (warp - 2) >> 2 < p.mblocks) {
+  } else if (PASS == 2 || (((warp - 2) >> 2) & 1) < p.mblocks) {
     // ================================================================ epilogue: a thread owns one window row (pass 1)
-    // or one key of every other tile (pass 2)
+    // or one key of every other tile (pass 2), in both cases for one half of the tile's columns
     const int ew = warp - 2;
-    const int mb = ew >> 2;                        // row block
+    const int mb = (ew >> 2) & 1;                  // row block (pass 1) or accumulator buffer (pass 2)
+    const int half = ew >> 3;                      // column half
     const int quarter = warp & 3;                  // TMEM lanes [32 * quarter, 32 * quarter + 32)
     const int row = mb * 128 + quarter * 32 + lane;
     const int eidx = ew * 32 + lane;               // index among the epilogue threads in use
     const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16) + mb * 128;
     const float masked = kEmptyMax;                // raw value given to a logit the row may not see
     int n_tile = 0;
+    uint32_t x_par = 0;  // pass 2: phase of the pair's exchange barrier
     bool ok = true;
     for (int it = blockIdx.x; ok && it < total_items; it += gridDim.x) {
       const int item = PASS == 1 ? it : total_items - 1 - it;
@@ -263,32 +271,35 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
               for (int i = 0; i < 16; ++i)
                 if (key0 + 16 * c + i >= vis) r[i] = __float_as_uint(masked);
             }
-            float bm = __uint_as_float(r[0]);
+            float t8[8];  // maximum and sums as trees: short dependency chains (two epilogue warps per scheduler)
 #pragma unroll
-            for (int i = 1; i < 16; ++i) bm = fmaxf(bm, __uint_as_float(r[i]));
+            for (int i = 0; i < 8; ++i) t8[i] = fmaxf(__uint_as_float(r[i]), __uint_as_float(r[i + 8]));
+            const float bm = fmaxf(fmaxf(fmaxf(t8[0], t8[4]), fmaxf(t8[1], t8[5])),
+                                   fmaxf(fmaxf(t8[2], t8[6]), fmaxf(t8[3], t8[7])));
             const float mn = fmaxf(m, bm * p.scale2);
             z *= ex2(m - mn);
             m = mn;
             const uint64_t nm2 = pack2(-mn, -mn), sc2 = pack2(p.scale2, p.scale2);
-            uint64_t acc = 0ull;
+            uint64_t e[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               float lo, hi;
               unpack2(fma2(pack2u(r[2 * i], r[2 * i + 1]), sc2, nm2), lo, hi);
-              acc = add2(acc, pack2(ex2(lo), ex2(hi)));
+              e[i] = pack2(ex2(lo), ex2(hi));
             }
             float lo, hi;
-            unpack2(acc, lo, hi);
+            unpack2(add2(add2(add2(e[0], e[1]), add2(e[2], e[3])), add2(add2(e[4], e[5]), add2(e[6], e[7]))), lo, hi);
             z += lo + hi;
           };
-          tmem_ld16_issue(taddr, ra);
+          const int c0 = 4 * half;  // this warp's 64 columns
+          tmem_ld16_issue(taddr + c0 * 16, ra);
 #pragma unroll 1
-          for (int c = 0; c < 8; c += 2) {
+          for (int c = c0; c < c0 + 4; c += 2) {
             tmem_ld_wait16(ra);
             tmem_ld16_issue(taddr + (c + 1) * 16, rb);
             block(ra, c);
             tmem_ld_wait16(rb);
-            if (c + 2 < 8) tmem_ld16_issue(taddr + (c + 2) * 16, ra);
+            if (c + 2 < c0 + 4) tmem_ld16_issue(taddr + (c + 2) * 16, ra);
             block(rb, c + 1);
           }
           tc_fence_before();
@@ -298,16 +309,19 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         if (row < p.R) {
           // a row that saw no visible key only summed masked entries: it is recorded as empty
           const bool none = m < 0.5f * kEmptyMax * p.scale2;
-          p.part[((int64_t)u * p.splits + split) * p.rs + row] = none ? make_float2(kEmptyMax, 0.f) : make_float2(m, z);
+          p.part[(((int64_t)u * p.splits + split) * 2 + half) * p.rs + row] =
+              none ? make_float2(kEmptyMax, 0.f) : make_float2(m, z);
         }
       } else {
         // group (warp - 2) / 4 owns accumulator buffer `group` and with it every other tile; this thread's key is
         // key0 + 32 * quarter + lane and its logits against the n16 window rows are the columns of its TMEM lane
-        const int group = ew >> 2;
+        const int group = mb;
+        const int pair = group * 4 + quarter;  // the two warps (column halves) that share a key
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + group * 256;
         const ulonglong2* ns = reinterpret_cast<const ulonglong2*>(p.lse2 + (int64_t)u * p.rs);
         const uint64_t sc2 = pack2(p.scale2, p.scale2);
-        const int nblk = p.n16 >> 4;
+        const int nblk = p.n16 >> 4, nlow = (nblk + 1) >> 1;
+        const int cb = half ? nlow : 0, ce = half ? nblk : nlow;  // this warp's blocks of 16 window rows
         for (int t = 0; t < tiles; ++t, ++n_tile) {
           if ((n_tile & 1) != group) continue;
           ok = __all_sync(0xffffffffu, mbar_wait(&tfull[group], (uint32_t)(n_tile >> 1) & 1u, abort_flag, p.status, kSiteTile));
@@ -335,25 +349,43 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
                 if (key >= vis) r[i] = __float_as_uint(kEmptyMax);
               }
             }
-            acc = exp_sum16(r, sc2, sh, acc);
+            uint64_t e[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              float lo, hi;
+              unpack2(fma2(pack2u(r[2 * i], r[2 * i + 1]), sc2, sh[i]), lo, hi);
+              e[i] = pack2(ex2(lo), ex2(hi));
+            }
+            acc = add2(acc, add2(add2(add2(e[0], e[1]), add2(e[2], e[3])), add2(add2(e[4], e[5]), add2(e[6], e[7]))));
           };
-          tmem_ld16_issue(taddr, ra);
+          if (cb < ce) tmem_ld16_issue(taddr + cb * 16, ra);
 #pragma unroll 1
-          for (int c = 0; c < nblk; c += 2) {
+          for (int c = cb; c < ce; c += 2) {
             tmem_ld_wait16(ra);
-            if (c + 1 < nblk) tmem_ld16_issue(taddr + (c + 1) * 16, rb);
+            if (c + 1 < ce) tmem_ld16_issue(taddr + (c + 1) * 16, rb);
             block(ra, c);
-            if (c + 1 < nblk) {
+            if (c + 1 < ce) {
               tmem_ld_wait16(rb);
-              if (c + 2 < nblk) tmem_ld16_issue(taddr + (c + 2) * 16, ra);
+              if (c + 2 < ce) tmem_ld16_issue(taddr + (c + 2) * 16, ra);
               block(rb, c + 1);
             }
           }
-          tc_fence_before();
-          mbar_arrive(&tempty[group]);
           float lo, hi;
           unpack2(acc, lo, hi);
-          if (key < p.n_max) psi[key] = key < n ? lo + hi : 0.f;
+          if (half) {  // hand the partial sum to the warp of the lower half
+            xch[group * 128 + quarter * 32 + lane] = lo + hi;
+            mbar_arrive(&xbar[pair]);
+          } else {
+            ok = __all_sync(0xffffffffu, mbar_wait(&xbar[pair], x_par, abort_flag, p.status, kSiteFlag));
+            x_par ^= 1;
+            if (!ok) break;
+            const float tot = (lo + hi) + xch[group * 128 + quarter * 32 + lane];
+            if (key < p.n_max) psi[key] = key < n ? tot : 0.f;
+          }
+          // the buffer is handed back only after the exchange: the upper half writes its next partial sum after the
+          // next tile of this buffer has been computed, which needs every arrival of this one
+          tc_fence_before();
+          mbar_arrive(&tempty[group]);
         }
         if (!ok) break;
         // keys of the item beyond the sequence
@@ -382,11 +414,12 @@ __global__ void score_rows_merge_kernel(RowParams p, float* nlse2, float* lse_ou
     nlse2[x] = kEmptyMax;
     return;
   }
-  const float2* part = p.part + (int64_t)u * p.splits * p.rs + row;
+  const int entries = 2 * p.splits;  // column halves of every split
+  const float2* part = p.part + (int64_t)u * entries * p.rs + row;
   float M = kEmptyMax;
-  for (int s = 0; s < p.splits; ++s) M = fmaxf(M, part[(int64_t)s * p.rs].x);
+  for (int s = 0; s < entries; ++s) M = fmaxf(M, part[(int64_t)s * p.rs].x);
   float Z = 0.f;
-  for (int s = 0; s < p.splits; ++s) {
+  for (int s = 0; s < entries; ++s) {
     const float2 v = part[(int64_t)s * p.rs];
     Z += v.y * exp2f(v.x - M);  // an empty split has sum 0
   }
@@ -444,9 +477,7 @@ int launch_score_rows(const madakv_config& c, const void* q, madakv_strides sq, 
   p.mblocks = R <= 128 ? 1 : 2;
   p.n16 = (R + 15) / 16 * 16;
   p.scale2 = scale_of(c) * kLog2e;
-  // the partials reuse the generic path's region: one pair per (1024-key chunk, row) there, per (2048-key split,
-  // padded row) here
-  if ((size_t)p.splits * p.rs > (size_t)wl.score_chunks * R) return MADAKV_EUNSUPPORTED;
+  // the workspace layout reserves (max, sum) pairs for [units, splits, 2 halves, rs]
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
