@@ -13,8 +13,9 @@
 //
 // Warp roles per CTA: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 epilogue (two groups of four
 // warps = the four TMEM lane quarters; group e takes the CTA's tiles of parity e; a thread owns one key of a tile and
-// all window rows of it). A tile's TMEM slot is handed back to the MMA warp after its last read, so the MMAs of the
-// next unit start while the last sweep of this one is still running; the TMA ring runs ahead across units.
+// all window rows of it). The TMEM slots form a ring over the CTA's tiles of consecutive units and a tile's slot is
+// handed back to the MMA warp after its last read: when a unit leaves slots free, the MMAs of the next unit run ahead
+// into them during this unit's exchange and last sweep, and the TMA ring runs ahead with them.
 // Synchronisation between CTAs exists only inside a cluster (whose CTAs are co-scheduled by the hardware): every lane
 // of every epilogue warp stores its rows' pairs into each peer's shared memory and arrives on that peer's mbarrier.
 // Every wait is bounded: on expiry the CTA records MADAKV_ETIMEOUT, drains and leaves through the final cluster barrier.
@@ -33,7 +34,7 @@ struct ClParams {
   float* lse_out;   // natural log [B,L,Hq,w] or null
   int32_t* status;  // ws header
   int units, L, Hq, Hkv, g, w, R, n_max, causal, C;
-  int per_max, sets;  // most tiles a CTA gets of one unit; how many such tile sets fit its TMEM (units alternate sets)
+  int per_max;  // most tiles a CTA gets of one unit (at most the number of TMEM slots)
   float scale2;
 };
 
@@ -171,9 +172,10 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
     tile0 = rank * per;
     my_tiles = max(0, min(per, tiles - tile0));
   };
-  // first TMEM slot of the unit: consecutive units of the cluster take alternate sets of slots when two sets fit, so
-  // that the MMAs of the next unit do not have to wait for this unit's last sweep
-  auto slot_base_of = [&](int u) { return (((u - cluster) / n_clusters) % p.sets) * p.per_max; };
+  // TMEM slots are a ring over the CTA's tiles of consecutive units: every role keeps the same running position
+  // (`ring`: slot of the current unit's first tile) and advances it by the unit's tile count.
+  auto slot_at = [&](int ring, int jj) { return (ring + jj) & (kSlots - 1); };
+  static_assert((kSlots & (kSlots - 1)) == 0, "slot ring uses a power-of-two mask");
 
   if (warp == 0) {
     // ================================================================ TMA producer
@@ -182,12 +184,12 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
       const uint64_t pol_q = l2_policy_evict_last();
       // A K stage may be refilled once the MMAs of the tile that used it last have completed: that is the tile's
       // tfull barrier. stage_user remembers the slot, slot_par the parity of the slot's latest use by this thread
-      // (a slot comes round once per unit at most, a stage every kStages tiles, so the latest use of the slot is
-      // the use that read the stage or a later one whose completion implies it).
+      // (a slot comes round every kSlots tiles, a stage every kStages < kSlots tiles, so the latest use of the slot
+      // is the use that read the stage).
       volatile uint32_t* stage_user = reinterpret_cast<volatile uint32_t*>(smem + SL::kMiscOff + 8);
       for (int s2 = 0; s2 < kStages; ++s2) stage_user[s2] = 0;
       uint32_t slot_par = 0, slot_used = 0;
-      int stage = 0, qi = 0;
+      int stage = 0, qi = 0, ring = 0;
       uint32_t q_par = 0;
       bool ok = true;
       for (int u = cluster; ok && u < p.units; u += n_clusters) {
@@ -196,7 +198,8 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
         int tile0, my_tiles;
         my_share(n, tile0, my_tiles);
         if (my_tiles == 0) continue;
-        const int sb = slot_base_of(u);
+        const int sb = ring;
+        ring = slot_at(ring, my_tiles);
         ok = mbar_wait(&qempty[qi], q_par ^ 1, abort_flag, p.status, kSiteQEmpty);
         if (!ok) break;
         mbar_expect_tx(&qfull[qi], (uint32_t)(p.R * 128 * kKBlocks));
@@ -205,7 +208,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
         qi ^= 1;
         if (qi == 0) q_par ^= 1;
         for (int jj = 0; jj < my_tiles; ++jj) {
-          const int j = sb + jj;  // slot
+          const int j = slot_at(sb, jj);
           const uint32_t prev = stage_user[stage];
           if (prev & 0x200u)
             ok = mbar_wait(&tfull[prev & 0xffu], (slot_par >> (prev & 0xffu)) & 1u, abort_flag, p.status, kSiteStage);
@@ -232,7 +235,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
       constexpr uint32_t idesc = instr_desc_bf16(NPAD);
       const uint32_t k_lo0 = smem_desc_lo(smem_u32(k_s)), q_lo0 = smem_desc_lo(smem_u32(q_s));
       uint32_t slot_par = 0, slot_used = 0;  // parity of the current use of every slot
-      int stage = 0, qi = 0;
+      int stage = 0, qi = 0, ring = 0;
       uint32_t stage_par = 0, q_par = 0;
       bool ok = true;
       for (int u = cluster; ok && u < p.units; u += n_clusters) {
@@ -241,12 +244,13 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
         int tile0, my_tiles;
         my_share(n, tile0, my_tiles);
         if (my_tiles == 0) continue;
-        const int sb = slot_base_of(u);
+        const int sb = ring;
+        ring = slot_at(ring, my_tiles);
         ok = mbar_wait(&qfull[qi], q_par, abort_flag, p.status, kSiteQFull);
         if (!ok) break;
         const uint32_t q_lo = q_lo0 + (uint32_t)qi * (SL::kQBytes >> 4);
         for (int jj = 0; jj < my_tiles; ++jj) {
-          const int j = sb + jj;  // slot
+          const int j = slot_at(sb, jj);
           if (slot_used & (1u << j)) slot_par ^= 1u << j;
           slot_used |= 1u << j;
           const uint32_t use_par = (slot_par >> j) & 1u;
@@ -293,8 +297,9 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
     const uint64_t* shift2 = reinterpret_cast<const uint64_t*>(shift_s);
     const uint64_t scale2x = pack2(p.scale2, p.scale2);
     const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    uint32_t slot_par = 0, slot_used = 0;  // parity of the current use of every slot of this group
+    uint32_t slot_par = 0, slot_used = 0;  // parity of the current use of every slot
     uint32_t unit_par = 0;                 // parity of the units this cluster has taken
+    int ring = 0;
     bool ok = true;
     for (int u = cluster; ok && u < p.units; u += n_clusters, unit_par ^= 1) {
       const int h = u % p.Hkv, bl = u / p.Hkv, b = bl / p.L;
@@ -303,19 +308,20 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
       int tile0, my_tiles;
       my_share(n, tile0, my_tiles);
       const int cnt = my_tiles > grp ? (my_tiles - grp + 1) / 2 : 0;  // this group's tiles: grp, grp + 2, ...
-      const int sb = slot_base_of(u);
+      const int sb = ring;
+      ring = slot_at(ring, my_tiles);
       const int all_bound = (n >= p.w) ? (p.causal ? n - p.w + 1 : n) : 0;  // keys below are seen by every row
       if (rank == 0) {  // positions beyond the unit's last tile
         for (int key = ((n + kTileKeys - 1) / kTileKeys) * kTileKeys + ew * 32 + lane; key < p.n_max; key += 256)
           psi[key] = 0.f;
       }
-      for (int i = 0; i < cnt; ++i) {  // parity of this use of the group's slots
-        const int j = sb + grp + 2 * i;
+      for (int jj = 0; jj < my_tiles; ++jj) {  // parity of this use of the unit's slots (either group's: a slot
+        const int j = slot_at(sb, jj);          // serves tiles of both groups as the ring moves on)
         if (slot_used & (1u << j)) slot_par ^= 1u << j;
         slot_used |= 1u << j;
       }
       auto wait_tile = [&](int i) -> bool {
-        const int j = sb + grp + 2 * i;
+        const int j = slot_at(sb, grp + 2 * i);
         const bool w_ok =
             __all_sync(0xffffffffu, mbar_wait(&tfull[j], (slot_par >> j) & 1u, abort_flag, p.status, kSiteTile));
         tc_fence_after();
@@ -323,7 +329,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
       };
       auto release_tile = [&](int i) {
         tc_fence_before();
-        mbar_arrive(&tempty[sb + grp + 2 * i]);
+        mbar_arrive(&tempty[slot_at(sb, grp + 2 * i)]);
       };
       // The group's tiles are read in blocks of 16 window rows (16 TMEM columns); the load of the next block is in
       // flight while the current one is processed. `body(j, r, i)` gets block j of the group's i-th tile.
@@ -331,9 +337,9 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
         if (cnt == 0) return true;
         uint32_t ra[16], rb[16];
         if (!before_tile(0)) return false;
-        tmem_ld16_issue(tlane + (sb + grp) * NPAD, ra);
+        tmem_ld16_issue(tlane + slot_at(sb, grp) * NPAD, ra);
         for (int i = 0; i < cnt; ++i) {
-          const uint32_t taddr = tlane + (sb + grp + 2 * i) * NPAD;
+          const uint32_t taddr = tlane + slot_at(sb, grp + 2 * i) * NPAD;
 #pragma unroll
           for (int j = 0; j < kBlocks; j += 2) {
             tmem_ld_wait16(ra);
@@ -344,7 +350,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
               tmem_ld16_issue(taddr + (j + 2) * 16, ra);
             } else if (i + 1 < cnt) {
               if (!before_tile(i + 1)) return false;
-              tmem_ld16_issue(taddr + 2 * NPAD, ra);
+              tmem_ld16_issue(tlane + slot_at(sb, grp + 2 * i + 2) * NPAD, ra);
             }
             body(j + 1, rb, i);
           }
@@ -599,28 +605,28 @@ int run_cluster(const CUtensorMap& mk, const CUtensorMap& mq, const ClParams& p,
 
 }  // namespace
 
-// The cluster size for a shape, or 0 if the logits of the longest sequence do not fit the TMEM of kMaxCluster CTAs:
-// the smallest size whose per-CTA share of tiles fits. When that share fits twice, consecutive units use alternate
-// halves of the TMEM.
-static int cluster_size_for(const madakv_config& c, int* per_max, int* sets) {
+// The cluster size for a shape, or 0 if the logits of the longest sequence do not fit the TMEM of kMaxCluster CTAs.
+// Any size from 1 to 8 works (a unit's tiles are dealt out in equal shares, the last ranks get the remainder). The
+// default is the smallest size whose per-CTA share fits; MADAKV_CLUSTER_SIZE forces another size that fits.
+static int cluster_size_for(const madakv_config& c, int* per_max) {
   const int R = (c.n_q_heads / c.n_kv_heads) * c.window;
   const int npad = R <= 32 ? 32 : 64;
   const int slots = kTmemCols / npad;
   const int tiles = (c.max_seq_len + kTileKeys - 1) / kTileKeys;
-  // Measured on the 8192-token workload: clusters of 8 (two sets) leave 28 of 148 SMs without a cluster and lose to
-  // clusters of 4 (one set), so the smallest cluster that fits is the default.
-  int first = 1;
-  if (const char* e = getenv("MADAKV_CLUSTER_SETS"))  // tests: 2 = prefer a cluster size where two sets fit
-    if (e[0] == '2') first = 2;
-  for (int want = first; want >= 1; --want)
-    for (int C = 1; C <= kMaxCluster; C *= 2) {
-      const int per = (tiles + C - 1) / C;
-      if (per * want <= slots) {
-        *per_max = per;
-        *sets = slots / per < 2 ? 1 : 2;
-        return C;
-      }
+  if (const char* e = getenv("MADAKV_CLUSTER_SIZE")) {
+    const int C = atoi(e);
+    if (C >= 1 && C <= kMaxCluster && (tiles + C - 1) / C <= slots) {
+      *per_max = (tiles + C - 1) / C;
+      return C;
     }
+  }
+  for (int C = 1; C <= kMaxCluster; ++C) {
+    const int per = (tiles + C - 1) / C;
+    if (per <= slots) {
+      *per_max = per;
+      return C;
+    }
+  }
   return 0;
 }
 
@@ -628,8 +634,8 @@ int launch_score_cluster(const madakv_config& c, const void* q, madakv_strides s
                          const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st) {
   const int g = c.n_q_heads / c.n_kv_heads;
   if (c.dtype != MADAKV_BF16 || g * c.window > 64) return MADAKV_EUNSUPPORTED;
-  int per_max = 0, sets = 0;
-  const int C = cluster_size_for(c, &per_max, &sets);
+  int per_max = 0;
+  const int C = cluster_size_for(c, &per_max);
   if (C == 0) return MADAKV_EUNSUPPORTED;
   if (const char* e = getenv("MADAKV_SCORE_PATH"))
     if (e[0] == 't') return MADAKV_EUNSUPPORTED;  // tests: force the two-phase kernel
@@ -649,7 +655,6 @@ int launch_score_cluster(const madakv_config& c, const void* q, madakv_strides s
   p.causal = c.causal;
   p.C = C;
   p.per_max = per_max;
-  p.sets = sets;
   p.scale2 = scale_of(c) * kLog2e;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
