@@ -123,6 +123,30 @@ class ClockSampler:
         return out
 
 
+def rank_workload(wl, rank):
+    """The batch of rank `rank`: same shape, its own seed. The path shards over independent sequences, so ranks
+    exchange nothing on the data path."""
+    return synth.scaled(wl, seed=wl.seed + 1000 * rank)
+
+
+def reduce_over_ranks(total_ms, tokens, device, world):
+    """Whole-job figures from per-rank ones: the slowest rank's time (MAX) and all ranks' prompt tokens (SUM). The
+    only collectives of a multi-GPU run; any backend (NCCL on GPUs, gloo in the CPU tests)."""
+    t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+    n = torch.tensor([tokens], dtype=torch.int64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(n.item())
+
+
+def job_throughput(total_ms, steps, tokens_all_ranks):
+    """Prompt tokens of all ranks per second of the slowest rank's step."""
+    return tokens_all_ranks / (total_ms / steps * 1e-3)
+
+
 def cpu_oracle_leg(wl, seconds_target=15.0):
     """The oracle, as it stands, on a bounded sample of the workload: the first layers of the same inputs (all of
     them when the whole workload fits the time target), repeated until about `seconds_target` of CPU work is done."""
@@ -237,7 +261,7 @@ def main():
         dist.barrier()
     mk.lib()
 
-    wl_r = synth.scaled(wl, seed=wl.seed + 1000 * rank)  # every rank its own batch
+    wl_r = rank_workload(wl, rank)  # every rank its own batch
     dev = torch.device("cuda", local)
     inp = synth.make_inputs(wl_r, device=dev)
     cfg = mk.make_config(wl.torch_dtype, wl.B, wl.L, wl.Hq, wl.Hkv, wl.d, wl.n, wl.w, max_new_tokens=wl.max_new_tokens,
@@ -295,12 +319,9 @@ def main():
     clocks = sampler.stop() if sampler else None
     total_ms = evs[0][0].elapsed_time(evs[-1][5])
     stage_ms = [sum(e[j].elapsed_time(e[j + 1]) for e in evs) / args.steps for j in range(5)]
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms, tokens_all = reduce_over_ranks(total_ms, tokens, dev, world)
     ms_per_step = total_ms / args.steps
-    value = world * tokens / (ms_per_step * 1e-3)
+    value = job_throughput(total_ms, args.steps, tokens_all)
 
     # bytes the method must move (algorithmic): K read once; kept K/V rows read and written; decode reads K_c + V_c
     rows = int(buf.kept_len.sum().item()) - wl.units  # kept rows before this step's append
@@ -344,11 +365,9 @@ def main():
             e2e_step(i)
         e1.record()
         sync_all()
-        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item()) / args.e2e_steps
-        e2e_value = world * tokens / (e2e_ms * 1e-3)
+        e2e_total, _ = reduce_over_ranks(e0.elapsed_time(e1), tokens, dev, world)
+        e2e_ms = e2e_total / args.e2e_steps
+        e2e_value = job_throughput(e2e_total, args.e2e_steps, tokens_all)
 
     # ---- decode-step latency: compressed cache (per step, all layers in one call) against the full cache
     def time_decode(b, steps=20):
