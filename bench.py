@@ -198,6 +198,15 @@ def cpu_oracle_leg(wl, seconds_target=15.0):
     }, dt
 
 
+def workload_config(wl):
+    """The `config` object of the JSON line: the same for both arms."""
+    k_gb = wl.units * wl.n * wl.d * wl.elem_bytes / 1e9
+    return {"workload": wl.name, "batch": wl.B, "layers": wl.L, "q_heads": wl.Hq, "kv_heads": wl.Hkv,
+            "head_dim": wl.d, "context": wl.n, "window": wl.w, "budget_per_head": wl.budget, "theta": wl.theta,
+            "l2": "inputs larger than L2 (K alone is %.2f GB)" % k_gb,
+            "step": "stages 1-4 + one all-layer decode step with append"}
+
+
 def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -213,7 +222,7 @@ def run_reference(args, wl):
         "impl": "reference", "metric": METRIC, "value": info["value"], "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
-        "config": {"workload": wl.name, "note": "CPU oracle on a bounded sample; each step = the sample once"},
+        "config": dict(workload_config(wl), note="CPU oracle on a bounded sample; each step = the sample once"),
         "cpu_baseline": info,
         "e2e": {"value": info["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -410,10 +419,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": wl.dtype, "data": "synthetic",
-        "config": {"workload": wl.name, "batch": wl.B, "layers": wl.L, "q_heads": wl.Hq, "kv_heads": wl.Hkv,
-                   "head_dim": wl.d, "context": wl.n, "window": wl.w, "budget_per_head": wl.budget, "theta": wl.theta,
-                   "l2": "inputs larger than L2 (K alone is %.2f GB)" % (k_bytes / 1e9),
-                   "step": "stages 1-4 + one all-layer decode step with append"},
+        "config": workload_config(wl),
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms},
