@@ -17,7 +17,8 @@
 // handed back to the MMA warp after its last read: when a unit leaves slots free, the MMAs of the next unit run ahead
 // into them during this unit's exchange and last sweep, and the TMA ring runs ahead with them.
 // Synchronisation between CTAs exists only inside a cluster (whose CTAs are co-scheduled by the hardware): every lane
-// of every epilogue warp stores its rows' pairs into each peer's shared memory and arrives on that peer's mbarrier.
+// of every epilogue warp sends its rows' pairs into each peer's shared memory with asynchronous stores that count
+// their bytes on that peer's mbarrier.
 // Every wait is bounded: on expiry the CTA records MADAKV_ETIMEOUT, drains and leaves through the final cluster barrier.
 #include "tc_common.cuh"
 
@@ -59,15 +60,14 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
   return r;
 }
-__device__ __forceinline__ void st_remote_f2(uint32_t raddr, float a, float b) {
-  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(raddr), "f"(a), "f"(b) : "memory");
+// Asynchronous store of a pair into a CTA of the cluster that, on landing, counts its 8 bytes on an mbarrier of that
+// CTA: the receiver's wait on the barrier's transaction count orders the data, so the sender needs neither a fence
+// nor an arrival of its own and goes straight on to its own wait.
+__device__ __forceinline__ void st_async_f2(uint32_t raddr, float a, float b, uint32_t rbar) {
+  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];" ::"r"(raddr),
+               "f"(a), "f"(b), "r"(rbar)
+               : "memory");
 }
-// Arrive on a peer's barrier without ordering of its own: the caller has fenced its stores at cluster scope once for
-// all peers (a releasing arrive per peer would wait for the remote stores one round trip at a time).
-__device__ __forceinline__ void mbar_arrive_remote_relaxed(uint32_t raddr) {
-  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(raddr) : "memory");
-}
-__device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_try_cluster(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -122,7 +122,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
   uint64_t* qempty = qfull + 2;           // [2]
   uint64_t* tfull = qempty + 2;           // [kSlots]   MMA -> epilogue and TMA
   uint64_t* tempty = tfull + kSlots;      // [kSlots]   epilogue -> MMA (128 arrivals: the four warps of the tile's group)
-  uint64_t* stats_bar = tempty + kSlots;  // [2]        all epilogue lanes of the cluster -> this CTA's epilogue warps
+  uint64_t* stats_bar = tempty + kSlots;  // [2]        bytes sent by all epilogue lanes of the cluster -> this CTA's epilogue warps
   uint64_t* drain = stats_bar + 2;        // [1]        used only when the kernel gives up
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(smem + SL::kMiscOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::kMiscOff + 4);
@@ -139,7 +139,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
     for (int i = 0; i < 2; ++i) {
       mbar_init(&qfull[i], 1);
       mbar_init(&qempty[i], 1);
-      mbar_init(&stats_bar[i], (uint32_t)(C * 256));
+      mbar_init(&stats_bar[i], 1);  // one local arrival that announces the bytes of a unit's exchange
     }
     for (int i = 0; i < kSlots; ++i) {
       mbar_init(&tfull[i], 1);
@@ -478,14 +478,15 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
         }
         mine[cb / 32] = make_float2(m2, zsum);
       }
+      // this CTA's barrier of the unit expects one pair per epilogue lane, window-row block and CTA of the cluster
+      if (ew == 0 && lane == 0) mbar_expect_tx(&stats_bar[unit_par], (uint32_t)(C * 8 * NPAD * sizeof(float2)));
       for (int peer = 0; peer < C; ++peer) {
+        const uint32_t rbar = map_to_rank(smem_u32(&stats_bar[unit_par]), (uint32_t)peer);
 #pragma unroll
         for (int cb = 0; cb < NPAD; cb += 32)
-          st_remote_f2(map_to_rank(smem_u32(my_stats + cb + lane), (uint32_t)peer), mine[cb / 32].x, mine[cb / 32].y);
+          st_async_f2(map_to_rank(smem_u32(my_stats + cb + lane), (uint32_t)peer), mine[cb / 32].x, mine[cb / 32].y,
+                      rbar);
       }
-      fence_cluster();  // this lane's stores to all peers come before its arrivals
-      for (int peer = 0; peer < C; ++peer)
-        mbar_arrive_remote_relaxed(map_to_rank(smem_u32(&stats_bar[unit_par]), (uint32_t)peer));
       // wait for the pairs of every warp of the cluster (bounded)
       {
         // the barrier completes once per two units: its phase parity for this unit is the parity of (units taken / 2)
