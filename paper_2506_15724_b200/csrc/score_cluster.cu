@@ -300,25 +300,44 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
     uint32_t slot_par = 0, slot_used = 0;  // parity of the current use of every slot
     uint32_t unit_par = 0;                 // parity of the units this cluster has taken
     int ring = 0;
+    // what depends on the sequence only is kept from unit to unit (the units of a sequence follow one another)
+    int b = -1, b_end = 0, n = 0, tile0 = 0, my_tiles = 0, all_bound = 0, tiles_end = 0;
     bool ok = true;
     for (int u = cluster; ok && u < p.units; u += n_clusters, unit_par ^= 1) {
-      const int h = u % p.Hkv, bl = u / p.Hkv, b = bl / p.L;
-      const int n = min(p.seq_len[b], p.n_max);
+      if (u >= b_end) {
+        b = u / (p.Hkv * p.L);
+        b_end = (b + 1) * p.Hkv * p.L;
+        n = min(p.seq_len[b], p.n_max);
+        my_share(n, tile0, my_tiles);
+        all_bound = (n >= p.w) ? (p.causal ? n - p.w + 1 : n) : 0;  // keys below are seen by every row
+        tiles_end = ((n + kTileKeys - 1) / kTileKeys) * kTileKeys;
+        __syncwarp();  // the warp's readers of vis_s for the previous sequence are done
+#pragma unroll
+        for (int cb = 0; cb < NPAD; cb += 32) {
+          const int row = cb + lane;
+          int vis = 0;  // per-row visibility bound (exclusive key index)
+          if (row < p.R) {
+            const int pos = n - p.w + row % p.w;
+            if (pos >= 0) vis = p.causal ? pos + 1 : n;
+          }
+          vis_s[row] = vis;
+        }
+        __syncwarp();
+      }
       float* psi = p.psi + (int64_t)u * p.n_max;
-      int tile0, my_tiles;
-      my_share(n, tile0, my_tiles);
       const int cnt = my_tiles > grp ? (my_tiles - grp + 1) / 2 : 0;  // this group's tiles: grp, grp + 2, ...
       const int sb = ring;
       ring = slot_at(ring, my_tiles);
-      const int all_bound = (n >= p.w) ? (p.causal ? n - p.w + 1 : n) : 0;  // keys below are seen by every row
       if (rank == 0) {  // positions beyond the unit's last tile
-        for (int key = ((n + kTileKeys - 1) / kTileKeys) * kTileKeys + ew * 32 + lane; key < p.n_max; key += 256)
-          psi[key] = 0.f;
+        for (int key = tiles_end + ew * 32 + lane; key < p.n_max; key += 256) psi[key] = 0.f;
       }
-      for (int jj = 0; jj < my_tiles; ++jj) {  // parity of this use of the unit's slots (either group's: a slot
-        const int j = slot_at(sb, jj);          // serves tiles of both groups as the ring moves on)
-        if (slot_used & (1u << j)) slot_par ^= 1u << j;
-        slot_used |= 1u << j;
+      {  // parity of this use of the unit's slots (either group's: a slot serves tiles of both groups as the ring
+         // moves on): the slots [sb, sb + my_tiles) of the ring as a bit mask
+        const uint32_t run = my_tiles >= 32 ? 0xffffffffu : (1u << my_tiles) - 1u;
+        const uint32_t all = kSlots >= 32 ? 0xffffffffu : (1u << kSlots) - 1u;
+        const uint32_t used_now = ((run << sb) | (run >> ((kSlots - sb) & 31))) & all;
+        slot_par ^= used_now & slot_used;
+        slot_used |= used_now;
       }
       auto wait_tile = [&](int i) -> bool {
         const int j = slot_at(sb, grp + 2 * i);
@@ -357,19 +376,6 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
         }
         return true;
       };
-
-      __syncwarp();  // the warp's readers of shift_s / vis_s of the previous unit are done
-#pragma unroll
-      for (int cb = 0; cb < NPAD; cb += 32) {
-        const int row = cb + lane;
-        int vis = 0;  // per-row visibility bound (exclusive key index)
-        if (row < p.R) {
-          const int pos = n - p.w + row % p.w;
-          if (pos >= 0) vis = p.causal ? pos + 1 : n;
-        }
-        vis_s[row] = vis;
-      }
-      __syncwarp();
 
       uint64_t z2[NPAD / 2];
       // Exact statistics in two sweeps: the warp's maximum per row, then the sum of exp2 against it. The (negated,
@@ -532,6 +538,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
         // negated for the exponent's fused multiply-add; padding rows get a huge shift (they add exp2(-huge) = 0)
         shift_s[row] = row < p.R ? -lse2 : kEmptyMax;
         if (p.lse_out && rank == 0 && ew == 0 && row < p.R) {
+          const int h = u % p.Hkv, bl = u / p.Hkv;
           const int hq = h * p.g + row / p.w, wr = row % p.w;
           p.lse_out[((int64_t)bl * p.Hq + hq) * p.w + wr] = (Z > 0.f) ? lse2 * 0.6931471805599453f : -INFINITY;
         }
