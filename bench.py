@@ -450,9 +450,9 @@ def launches_per_step(wl):
 
 
 # dram bytes (read + write) per launch of the dominant kernel (score_cluster), per workload, from the ncu capture
-# summarised in profiles/all_kernels_llava.md: 274.3 MB measured on the 4-layer case, times 8 for the 32 layers
+# summarised in profiles/all_kernels_llava.md: 274.2 MB measured on the 4-layer case, times 8 for the 32 layers
 # (traffic grows with the number of units); None = not captured
-TRAFFIC = {"llava": 8 * 274.3e6}
+TRAFFIC = {"llava": 8 * 274.2e6}
 
 if __name__ == "__main__":
     main()
