@@ -238,6 +238,49 @@ def test_edge_cases_budget_extremes_and_single_modality():
             assert (ref["kept_len"] == wl.n).all()
 
 
+@pytest.mark.parametrize("n", [8192, 20000])
+@pytest.mark.parametrize("kind", ["few_values", "all_equal", "flat_with_peaks", "distinct"])
+def test_allocate_and_select_on_crafted_scores(kind, n):
+    """Stages 2-4a on hand-made importance scores, bit-exact against the oracle: thousands of tied values (one
+    radix bucket then holds most keys down to the last pass), a single value, a flat floor with a few peaks, and all-distinct values; one sequence
+    length that fits the registers of a block and one that takes several rounds."""
+    wl = synth.scaled(TINY, B=2, L=2, Hq=2, Hkv=2, n=n, w=8, budget=n // 5, theta=0.4)
+    inp = synth.make_inputs(wl, device="cpu", want_v=False)
+    rng = np.random.RandomState(11)
+    shape = (wl.B, wl.L, wl.Hkv, wl.n)
+    if kind == "few_values":
+        psi = rng.choice(np.array([1e-3, 2e-3, 2.0000002e-3, 0.25, 3e-5], np.float32), size=shape)
+    elif kind == "all_equal":
+        psi = np.full(shape, 1.0 / wl.n, np.float32)
+    elif kind == "flat_with_peaks":
+        psi = np.full(shape, 3e-4, np.float32)
+        psi[..., rng.choice(wl.n, 40, replace=False)] = rng.uniform(0.1, 2.0, size=40).astype(np.float32)
+    else:
+        psi = rng.uniform(1e-6, 1e-2, size=shape).astype(np.float32)
+    psi = np.ascontiguousarray(psi, np.float32)
+    mask, sl, bud = to_np(inp["mask"]), to_np(inp["seq_len"]), to_np(inp["budget"])
+    sl = sl.copy()
+    sl[1] = wl.n - 301  # ragged
+    psi[1, :, :, sl[1]:] = 0.0
+    for theta in (0.05, 0.4, 0.97):
+        cfg = config_of(wl, theta=theta)
+        buf = mk.EvictionBuffers(cfg, capacity_of(wl))
+        d_psi, d_mask = torch.from_numpy(psi).cuda(), inp["mask"].cuda()
+        d_sl, d_bud = torch.from_numpy(sl).cuda(), inp["budget"].cuda()
+        mk.madakv_allocate(cfg, d_psi, d_mask, d_sl, d_bud, buf.mass, buf.pref, buf.demand, buf.phi, buf.budgets,
+                           buf.ws)
+        mk.madakv_select(cfg, d_psi, d_mask, d_sl, buf.budgets, buf.kept_len, buf.seg_off, buf.kept_idx, buf.ws)
+        assert mk.madakv_poll_status(buf.ws) == 0
+        al = oracle.allocate(psi, mask, sl, bud, float(np.float32(theta)))
+        for key in ("mass", "pref", "demand", "phi", "budgets"):
+            assert np.array_equal(getattr(buf, key).cpu().numpy(), al[key]), (key, kind, theta)
+        rc, kept_len, seg_off, kept_idx = oracle.select(psi, mask, sl, al["budgets"], headroom=wl.max_new_tokens,
+                                                        capacity=capacity_of(wl))
+        assert rc == 0
+        assert np.array_equal(buf.kept_len.cpu().numpy(), kept_len)
+        assert_segments_equal(kept_len, seg_off, buf.kept_idx.cpu().numpy(), kept_idx, "kept_idx")
+
+
 def test_short_sequences_and_empty_sequence():
     wl = synth.scaled(TINY, B=4, L=1, n=320 + 8, w=8, budget=16)
     inp = synth.make_inputs(wl)
