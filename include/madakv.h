@@ -101,6 +101,17 @@ int madakv_workspace_bytes(const madakv_config* cfg, size_t* bytes_out);
 int madakv_score(const madakv_config* cfg, const void* q_win, madakv_strides sq, const void* k, madakv_strides sk,
                  const int32_t* seq_len, float* lse, float* psi, void* ws, size_t ws_bytes, void* stream);
 
+/* Stage 1 in a single pass (Eq. 7), for callers that already hold the softmax normalisers: the attention of the
+ * prompt's last w queries was computed during prefill (Eq. 5), and its log-sum-exp per row is what a fused attention
+ * kernel keeps anyway. Same arguments and result as madakv_score, except that
+ *   lse     [B, L, H_q, w] fp32 is an INPUT: the natural-log sum-exp of every window row's scaled logits over the
+ *           keys the row sees (what madakv_score stores in its `lse`); -inf for a row that sees no key.
+ * psi[u][i] = sum over the group's heads and window rows of exp( scale * q.k_i - lse ). K is read once and nothing
+ * is reduced over keys, so the result is only as good as the normalisers supplied. Layer by layer use: pass a
+ * config with n_layers = 1 and pointers to that layer's slices.                                             */
+int madakv_score_lse(const madakv_config* cfg, const void* q_win, madakv_strides sq, const void* k, madakv_strides sk,
+                     const int32_t* seq_len, const float* lse, float* psi, void* ws, size_t ws_bytes, void* stream);
+
 /* Stages 2-3 (Eq. 6, 8, 9, 10, 11). All sums of psi are taken exactly, in 2^-32 fixed point:
  *   Q(x) = floor(x * 2^32) for x > 0, else 0;   W_m = sum_{i in X_m} Q(psi[u][i])                 (Eq. 6)
  *   pref[u][m] = W_m / (W_v + W_t)  (0 if the denominator is 0)                                    (Eq. 8 ratio)

@@ -20,7 +20,8 @@ STATUS_NAMES = ["OK", "EINVAL", "ESHAPE", "EALIGN", "EWORKSPACE", "ECAPACITY", "
 STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = [
-    "madakv_abi_version", "madakv_status_string", "madakv_workspace_bytes", "madakv_score", "madakv_allocate",
+    "madakv_abi_version", "madakv_status_string", "madakv_workspace_bytes", "madakv_score", "madakv_score_lse",
+    "madakv_allocate",
     "madakv_select", "madakv_compact", "madakv_decode_attn", "madakv_decode_attn_static", "madakv_poll_status",
 ]
 
@@ -64,6 +65,7 @@ def lib():
         L.madakv_status_string.argtypes = [ctypes.c_int]
         L.madakv_workspace_bytes.argtypes = [cfgp, ctypes.POINTER(sz)]
         L.madakv_score.argtypes = [cfgp, vp, MadakvStrides, vp, MadakvStrides, vp, vp, vp, vp, sz, vp]
+        L.madakv_score_lse.argtypes = [cfgp, vp, MadakvStrides, vp, MadakvStrides, vp, vp, vp, vp, sz, vp]
         L.madakv_allocate.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.madakv_select.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, i64, vp, sz, vp]
         L.madakv_compact.argtypes = [cfgp, vp, vp, MadakvStrides, vp, vp, vp, vp, vp, i64, vp, sz, vp]
@@ -116,6 +118,12 @@ def new_workspace(cfg, device="cuda"):
 def madakv_score(cfg, q_win, k, seq_len, lse, psi, ws):
     _check("madakv_score", lib().madakv_score(ctypes.byref(cfg), _ptr(q_win), _strides5(q_win), _ptr(k), _strides5(k),
                                               _ptr(seq_len), _ptr(lse), _ptr(psi), _ptr(ws), ws.numel(), _stream()))
+
+
+def madakv_score_lse(cfg, q_win, k, seq_len, lse, psi, ws):
+    _check("madakv_score_lse", lib().madakv_score_lse(ctypes.byref(cfg), _ptr(q_win), _strides5(q_win), _ptr(k),
+                                                      _strides5(k), _ptr(seq_len), _ptr(lse), _ptr(psi), _ptr(ws),
+                                                      ws.numel(), _stream()))
 
 
 def madakv_allocate(cfg, psi, mask, seq_len, budget, mass, pref, demand, phi, budgets, ws):

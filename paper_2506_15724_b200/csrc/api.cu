@@ -44,6 +44,18 @@ int madakv_score(const madakv_config* cfg, const void* q_win, madakv_strides sq,
   return launch_score(*cfg, q_win, sq, k, sk, seq_len, lse, psi, ws, (cudaStream_t)stream);
 }
 
+int madakv_score_lse(const madakv_config* cfg, const void* q_win, madakv_strides sq, const void* k, madakv_strides sk,
+                     const int32_t* seq_len, const float* lse, float* psi, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (!q_win || !k || !seq_len || !lse || !psi) return MADAKV_EINVAL;
+  if (!aligned16(q_win) || !aligned16(k) || !aligned16(psi) || ((uintptr_t)seq_len & 3) || ((uintptr_t)lse & 3))
+    return MADAKV_EALIGN;
+  if (!strides_ok(*cfg, sq) || !strides_ok(*cfg, sk)) return MADAKV_EALIGN;
+  if ((rc = check_ws(*cfg, ws, ws_bytes))) return rc;
+  return launch_score_lse(*cfg, q_win, sq, k, sk, seq_len, lse, psi, ws, (cudaStream_t)stream);
+}
+
 int madakv_allocate(const madakv_config* cfg, const float* psi, const uint8_t* mask, const int32_t* seq_len,
                     const int32_t* budget, double* mass, double* pref, int32_t* demand, double* phi, int32_t* budgets,
                     void* ws, size_t ws_bytes, void* stream) {

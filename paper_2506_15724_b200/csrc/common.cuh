@@ -142,6 +142,10 @@ __device__ __forceinline__ void set_status(void* ws, int code) { atomicCAS((int*
 // Stage launchers implemented in the .cu files (all return a madakv_status).
 int launch_score(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
                  const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st);
+int launch_score_lse(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                     const int32_t* seq_len, const float* lse, float* psi, void* ws, cudaStream_t st);
+int launch_score_lse_rows(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                          const int32_t* seq_len, const float* lse, float* psi, void* ws, cudaStream_t st);
 bool tc_device_ok();
 bool score_tc_supported(const madakv_config& c, madakv_strides sq, madakv_strides sk);
 int launch_score_tc(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,

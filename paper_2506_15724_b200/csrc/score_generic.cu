@@ -240,6 +240,28 @@ __global__ void __launch_bounds__(NT) score_psi_kernel(ScoreParams p) {
   }
 }
 
+// caller-supplied natural-log sum-exps [B, L, H_q, w] -> log2-domain values in the (unit, row) order of the psi kernel
+__global__ void score_given_lse_kernel(ScoreParams p, const float* lse, int total_rows) {
+  const int x = blockIdx.x * blockDim.x + threadIdx.x;
+  if (x >= total_rows) return;
+  const int u = x / p.R, row = x % p.R;
+  const int h = u % p.Hkv, bl = u / p.Hkv;
+  const int hq = h * p.g + row / p.w, wr = row % p.w;
+  p.lse2[x] = lse[((int64_t)bl * p.Hq + hq) * p.w + wr] * 1.4426950408889634f;
+}
+
+template <typename T, int D>
+int run_given_lse(const ScoreParams& p, const float* lse, int units, cudaStream_t st) {
+  const size_t smem = (size_t)(KT + RT) * (D + 4) * sizeof(float);
+  if (cudaFuncSetAttribute(score_psi_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+      cudaSuccess)
+    return MADAKV_ECUDA;
+  const int total_rows = units * p.R;
+  score_given_lse_kernel<<<(total_rows + 255) / 256, 256, 0, st>>>(p, lse, total_rows);
+  score_psi_kernel<T, D><<<dim3((p.n_max + KT - 1) / KT, units), NT, smem, st>>>(p);
+  return launch_status();
+}
+
 template <typename T, int D>
 int run(const ScoreParams& p, int units, cudaStream_t st) {
   const size_t smem = (size_t)(KT + RT) * (D + 4) * sizeof(float);
@@ -257,8 +279,8 @@ int run(const ScoreParams& p, int units, cudaStream_t st) {
 
 }  // namespace
 
-int launch_score_generic(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
-                         const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st) {
+static ScoreParams generic_params(const madakv_config& c, const void* q, madakv_strides sq, const void* k,
+                                  madakv_strides sk, const int32_t* seq_len, float* lse, float* psi, void* ws) {
   const WsLayout wl = ws_layout(c);
   ScoreParams p;
   p.q = q;
@@ -280,10 +302,33 @@ int launch_score_generic(const madakv_config& c, const void* q, madakv_strides s
   p.chunks = wl.score_chunks;
   p.causal = c.causal;
   p.scale2 = scale_of(c) * kLog2e;
+  return p;
+}
+
+int launch_score_generic(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                         const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st) {
+  const ScoreParams p = generic_params(c, q, sq, k, sk, seq_len, lse, psi, ws);
   const int units = c.batch * c.n_layers * c.n_kv_heads;
   if (units > 65535) return MADAKV_EUNSUPPORTED;
   if (c.dtype == MADAKV_F32) return c.head_dim == 64 ? run<float, 64>(p, units, st) : run<float, 128>(p, units, st);
   return c.head_dim == 64 ? run<__nv_bfloat16, 64>(p, units, st) : run<__nv_bfloat16, 128>(p, units, st);
+}
+
+// Single-pass scoring (Eq. 7) with the softmax normalisers supplied: tensor-core kernel for bf16 with g * w <= 256,
+// the fp32 psi kernel otherwise.
+int launch_score_lse(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                     const int32_t* seq_len, const float* lse, float* psi, void* ws, cudaStream_t st) {
+  if (tc_device_ok()) {  // false also when MADAKV_SCORE_PATH asks for the fp32 kernels
+    const int rc = launch_score_lse_rows(c, q, sq, k, sk, seq_len, lse, psi, ws, st);
+    if (rc != MADAKV_EUNSUPPORTED) return rc;
+  }
+  const ScoreParams p = generic_params(c, q, sq, k, sk, seq_len, nullptr, psi, ws);
+  const int units = c.batch * c.n_layers * c.n_kv_heads;
+  if (units > 65535) return MADAKV_EUNSUPPORTED;
+  if (c.dtype == MADAKV_F32)
+    return c.head_dim == 64 ? run_given_lse<float, 64>(p, lse, units, st) : run_given_lse<float, 128>(p, lse, units, st);
+  return c.head_dim == 64 ? run_given_lse<__nv_bfloat16, 64>(p, lse, units, st)
+                          : run_given_lse<__nv_bfloat16, 128>(p, lse, units, st);
 }
 
 int launch_score(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,

@@ -432,6 +432,22 @@ __global__ void score_rows_merge_kernel(RowParams p, float* nlse2, float* lse_ou
   }
 }
 
+// caller-supplied natural-log sum-exps [B, L, H_q, w] -> negated log2-domain values in the (unit, row) layout of pass 2;
+// a row that saw no key (-inf) and the padding rows get the shift that turns every weight into 0
+__global__ void score_rows_given_lse_kernel(RowParams p, const float* lse, float* nlse2, int total) {
+  const int x = blockIdx.x * blockDim.x + threadIdx.x;
+  if (x >= total) return;
+  const int u = x / p.rs, row = x % p.rs;
+  float v = kEmptyMax;
+  if (row < p.R) {
+    const int h = u % p.Hkv, bl = u / p.Hkv;
+    const int hq = h * p.g + row / p.w, wr = row % p.w;
+    const float l = lse[((int64_t)bl * p.Hq + hq) * p.w + wr];
+    if (l > -INFINITY) v = -l * kLog2e;
+  }
+  nlse2[x] = v;
+}
+
 template <int D>
 int run_rows(const CUtensorMap& mk, const CUtensorMap& mq, RowParams p, float* lse2, float* lse_out, int grid,
              cudaStream_t st) {
@@ -450,17 +466,19 @@ int run_rows(const CUtensorMap& mk, const CUtensorMap& mq, RowParams p, float* l
 
 }  // namespace
 
-int launch_score_rows(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
-                      const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st) {
+// parameters shared by the two-pass and the single-pass launch; false if the shape is outside this file's range
+static bool rows_setup(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                       const int32_t* seq_len, float* psi, void* ws, RowParams& p, float*& lse2, CUtensorMap& mk,
+                       CUtensorMap& mq, int& grid, int& rc) {
   const int g = c.n_q_heads / c.n_kv_heads;
   const int R = g * c.window;
-  if (c.dtype != MADAKV_BF16 || R <= 64 || R > 256 || c.window > 256 || g > 256) return MADAKV_EUNSUPPORTED;
+  rc = MADAKV_EUNSUPPORTED;
+  if (c.dtype != MADAKV_BF16 || R > 256 || c.window > 256 || g > 256) return false;
   const WsLayout wl = ws_layout(c);
-  RowParams p;
   p.seq_len = seq_len;
   p.psi = psi;
   p.part = reinterpret_cast<float2*>((char*)ws + wl.score_part_off);
-  float* lse2 = reinterpret_cast<float*>((char*)ws + wl.score_lse_off);
+  lse2 = reinterpret_cast<float*>((char*)ws + wl.score_lse_off);
   p.lse2 = lse2;
   p.status = reinterpret_cast<int32_t*>(ws);
   p.units = c.batch * c.n_layers * c.n_kv_heads;
@@ -477,19 +495,58 @@ int launch_score_rows(const madakv_config& c, const void* q, madakv_strides sq, 
   p.mblocks = R <= 128 ? 1 : 2;
   p.n16 = (R + 15) / 16 * 16;
   p.scale2 = scale_of(c) * kLog2e;
-  // the workspace layout reserves (max, sum) pairs for [units, splits, 2 halves, rs]
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return MADAKV_ECUDA;
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    rc = MADAKV_ECUDA;
+    return false;
+  }
   const long long items = (long long)p.units * p.splits;
-  if (items > 0x3fffffff) return MADAKV_EUNSUPPORTED;
-  const int grid = (int)(items < sms ? items : sms);
-  CUtensorMap mk, mq;
+  if (items > 0x3fffffff) return false;
+  grid = (int)(items < sms ? items : sms);
   if (!make_map(&mk, k, c.head_dim, c.max_seq_len, c.n_kv_heads, c.n_layers, c.batch, sk, kTileKeys, 1) ||
       !make_map(&mq, q, c.head_dim, c.window, c.n_q_heads, c.n_layers, c.batch, sq, c.window, g))
-    return MADAKV_EUNSUPPORTED;
+    return false;
+  return true;
+}
+
+int launch_score_rows(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                      const int32_t* seq_len, float* lse, float* psi, void* ws, cudaStream_t st) {
+  if ((c.n_q_heads / c.n_kv_heads) * c.window <= 64) return MADAKV_EUNSUPPORTED;  // the TMEM-resident kernels' range
+  RowParams p;
+  float* lse2;
+  CUtensorMap mk, mq;
+  int grid, rc;
+  // the workspace layout reserves (max, sum) pairs for [units, splits, 2 halves, rs]
+  if (!rows_setup(c, q, sq, k, sk, seq_len, psi, ws, p, lse2, mk, mq, grid, rc)) return rc;
   return c.head_dim == 128 ? run_rows<128>(mk, mq, p, lse2, lse, grid, st) : run_rows<64>(mk, mq, p, lse2, lse, grid, st);
+}
+
+// Single-pass scoring with the rows' log-sum-exps supplied by the caller: a conversion kernel, then pass 2 alone.
+// Any bf16 shape with g * w <= 256.
+int launch_score_lse_rows(const madakv_config& c, const void* q, madakv_strides sq, const void* k, madakv_strides sk,
+                          const int32_t* seq_len, const float* lse, float* psi, void* ws, cudaStream_t st) {
+  RowParams p;
+  float* lse2;
+  CUtensorMap mk, mq;
+  int grid, rc;
+  if (!rows_setup(c, q, sq, k, sk, seq_len, psi, ws, p, lse2, mk, mq, grid, rc)) return rc;
+  const int total = p.units * p.rs;
+  score_rows_given_lse_kernel<<<(total + 255) / 256, 256, 0, st>>>(p, lse, lse2, total);
+  if (c.head_dim == 128) {
+    using SL = RowSmem<128>;
+    if (cudaFuncSetAttribute(score_rows_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kAlloc) !=
+        cudaSuccess)
+      return MADAKV_ECUDA;
+    score_rows_kernel<128, 2><<<grid, kRowThreads, SL::kAlloc, st>>>(mk, mq, p);
+  } else {
+    using SL = RowSmem<64>;
+    if (cudaFuncSetAttribute(score_rows_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kAlloc) !=
+        cudaSuccess)
+      return MADAKV_ECUDA;
+    score_rows_kernel<64, 2><<<grid, kRowThreads, SL::kAlloc, st>>>(mk, mq, p);
+  }
+  return launch_status();
 }
 
 }  // namespace madakv

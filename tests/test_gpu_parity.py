@@ -95,6 +95,36 @@ def test_score_matches_oracle(name, causal, path, monkeypatch):
     assert torch.equal(again, buf.psi)
 
 
+@pytest.mark.parametrize("name", list(SHAPES))
+@pytest.mark.parametrize("causal", [1, 0])
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_single_pass_score_with_given_lse(name, causal, path, monkeypatch):
+    # madakv_score_lse gets the oracle's log-sum-exps (rounded to fp32) and must reproduce the oracle's psi; "auto"
+    # takes the tensor-core kernel for the bf16 shapes, "generic" the fp32 kernel for all
+    if path == "generic":
+        monkeypatch.setenv("MADAKV_SCORE_PATH", "generic")
+    wl = SHAPES[name]
+    inp = make_case(wl)
+    cfg = config_of(wl, causal=causal)
+    g = dev(inp)
+    want, want_lse = oracle.score(dcode(wl), to_np(inp["q_win"]), to_np(inp["k"]), to_np(inp["seq_len"]),
+                                  causal=causal, want_lse=True)
+    lse = torch.from_numpy(want_lse.astype(np.float32)).cuda()
+    buf = mk.EvictionBuffers(cfg, capacity_of(wl))
+    buf.psi.fill_(7.0)  # the call must overwrite every element, padding included
+    mk.madakv_score_lse(cfg, g["q_win"], g["k"], g["seq_len"], lse, buf.psi, buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    got = buf.psi.cpu().numpy()
+    assert psi_close(got, want, PSI_RTOL) < PSI_RTOL_SEEN
+    for b in range(wl.B):
+        assert (got[b, :, :, int(inp["seq_len"][b]):] == 0).all()
+    # and it agrees with the two-pass call's own normalisers fed back in
+    two = mk.EvictionBuffers(cfg, capacity_of(wl), want_lse=True)
+    mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], two.lse, two.psi, two.ws)
+    mk.madakv_score_lse(cfg, g["q_win"], g["k"], g["seq_len"], two.lse, buf.psi, buf.ws)
+    assert psi_close(buf.psi.cpu().numpy(), two.psi.cpu().numpy().astype(np.float64), 1e-4) < 1e-4
+
+
 @pytest.mark.parametrize("lag", ["8", "9", "40", "1000"])
 def test_tensor_core_score_item_interleaving(lag, monkeypatch):
     # many more work items than the phase-1 lead: exercises the interleaved phase-2 / phase-1 item order and the
@@ -389,6 +419,12 @@ def test_full_size_workload_sampled(name):
         assert worst < PSI_RTOL_SEEN, worst
         np.testing.assert_allclose(buf.lse.cpu().numpy()[:, l:l + 1, qs], want_lse, rtol=0, atol=2e-5)
     np.testing.assert_allclose(psi.sum(-1), wl.g * wl.w, rtol=1e-5)  # every softmax row sums to 1
+    # the single-pass call, fed the normalisers just computed, gives the same scores
+    once = torch.empty_like(buf.psi)
+    mk.madakv_score_lse(cfg, inp["q_win"], inp["k"], inp["seq_len"], buf.lse, once, buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    assert psi_close(once.cpu().numpy(), psi.astype(np.float64), 1e-4) < 1e-4
+    del once
     # stages 2-4a on all units: bit-exact functions of the fp32 scores
     al = oracle.allocate(psi, mask, sl, bud, float(np.float32(cfg.theta)))
     for key in ("mass", "pref", "demand", "phi", "budgets"):
