@@ -393,6 +393,24 @@ def main():
         torch.cuda.synchronize()
         return a.elapsed_time(z) / steps * 1e3
 
+    # ---- stage 1 in a single pass, for callers that bring the prefill's log-sum-exps (here: those of madakv_score)
+    def time_single_pass(steps=20):
+        lse = torch.empty((wl.B, wl.L, wl.Hq, wl.w), dtype=torch.float32, device=dev)
+        psi1 = torch.empty_like(buf.psi)
+        mk.madakv_score(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, buf.psi, buf.ws)
+        for _ in range(3):
+            mk.madakv_score_lse(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, psi1, buf.ws)
+        torch.cuda.synchronize()
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            mk.madakv_score_lse(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, psi1, buf.ws)
+        z.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(z) / steps
+
+    single_ms = time_single_pass()
+
     decode_us = {"compressed": time_decode(buf), "full": None,
                  "compressed_rows_per_head": (rows + wl.units) / wl.units}
     if not args.no_full_cache and rank == 0:
@@ -434,6 +452,9 @@ def main():
         "decode": {"us_per_step": decode_us, "algorithmic_bytes": decode_bytes, "gbs_in_step": dec_gbs,
                    "frac_of_measured_peak_in_step": dec_gbs / peak,
                    "gbs_alone": decode_bytes / (decode_us["compressed"] * 1e-6) / 1e9},
+        "single_pass_score": {"ms": single_ms, "gbs": k_bytes / (single_ms * 1e-3) / 1e9,
+                              "frac_of_measured_peak": k_bytes / (single_ms * 1e-3) / 1e9 / peak,
+                              "note": "madakv_score_lse: stage 1 with the rows' log-sum-exps supplied; not part of the step"},
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))
