@@ -129,6 +129,19 @@ int madakv_allocate(const madakv_config* cfg, const float* psi, const uint8_t* m
                     const int32_t* budget, double* mass, double* pref, int32_t* demand, double* phi, int32_t* budgets,
                     void* ws, size_t ws_bytes, void* stream);
 
+/* Stages 2-3 for ONE layer of a layer-by-layer pass (the order Section 3.3 implies: a layer is evicted right after
+ * its prefill and the budget state goes on to the next layer, Eq. 11). cfg->n_layers = L is the real depth and
+ * `layer` in [0, L) the layer at hand; the per-layer arrays hold that layer only:
+ *   psi [B,H_kv,n_max]; mass, pref [B,H_kv,2] fp64; demand, budgets [B,H_kv,2] int32
+ *   phi [B,L] fp64 is the state carried between calls: layer 0 sets phi[b][0] = budget[b]; every call reads
+ *   phi[b][layer] and, when layer + 1 < L, writes phi[b][layer + 1]  (Eq. 10-11).
+ * Called for layer = 0 .. L-1 in order it produces exactly the phi, mass, pref, demand and budgets that
+ * madakv_allocate produces for the stacked arrays. For stages 1 and 4 of such a pass give madakv_score_lse (or
+ * madakv_score), madakv_select and madakv_compact a config with n_layers = 1 and that layer's slices.        */
+int madakv_allocate_layer(const madakv_config* cfg, int32_t layer, const float* psi, const uint8_t* mask,
+                          const int32_t* seq_len, const int32_t* budget, double* mass, double* pref, int32_t* demand,
+                          double* phi, int32_t* budgets, void* ws, size_t ws_bytes, void* stream);
+
 /* Stage 4a (Section 3.3: modality-specific eviction for each head). For every unit keep, of each modality m,
  * the budgets[u][m] tokens with the largest psi (equal psi: the lower position wins) and list the kept positions
  * in ascending order:

@@ -252,6 +252,68 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
   }
 }
 
+// Visual tokens among the first n of a sequence, counted by the whole block into *s_nv (which the caller has zeroed
+// behind a barrier); the caller synchronises before reading it.
+__device__ __forceinline__ void count_visual(const uint8_t* mask, int n, int* s_nv) {
+  int c = 0;
+  if ((reinterpret_cast<uintptr_t>(mask) & 15) == 0) {  // 16 tokens per load
+    const int n16 = n >> 4;
+    for (int i = threadIdx.x; i < n16; i += blockDim.x) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(mask) + i);
+      const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k)  // a byte counts if it is not zero
+        c += __popc(((w4[k] | (w4[k] >> 1) | (w4[k] >> 2) | (w4[k] >> 3) | (w4[k] >> 4) | (w4[k] >> 5) | (w4[k] >> 6) |
+                      (w4[k] >> 7)) & 0x01010101u));
+    }
+    for (int i = (n16 << 4) + threadIdx.x; i < n; i += blockDim.x) c += mask[i] ? 1 : 0;
+  } else {
+    for (int i = threadIdx.x; i < n; i += blockDim.x) c += mask[i] ? 1 : 0;
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
+  if ((threadIdx.x & 31) == 0 && c) atomicAdd(s_nv, c);
+}
+// Eq. 10's sum over the heads of one layer (both modalities), by one warp; every lane returns it.
+__device__ __forceinline__ long long layer_demand(const int32_t* demand_layer, int Hkv) {
+  long long dem = 0;
+  for (int x = threadIdx.x & 31; x < 2 * Hkv; x += 32) dem += (long long)demand_layer[x];
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) dem += __shfl_xor_sync(0xffffffffu, dem, off);
+  return dem;
+}
+// The layer's integer budget Phi^l from phi^l, and phi^{l+1} (Eq. 10-11); l counts from 1, the update exists for l < L.
+__device__ __forceinline__ double rounded_budget(double ph, double lo, double hi) {
+  return fmin(fmax(floor(__dadd_rn(ph, 0.5)), lo), hi);
+}
+__device__ __forceinline__ double next_phi(double ph, long long dem, int Hkv, int L, int l, int hcc_mode, double lo,
+                                           double hi) {
+  const double K = __dsub_rn((double)dem, __dmul_rn((double)Hkv, ph));  // Eq. 10
+  double next = ph;
+  if (hcc_mode == MADAKV_HCC_PAPER)
+    next = __dsub_rn(ph, __ddiv_rn(K, (double)((long long)Hkv * (L - l))));  // Eq. 11, per-head units
+  else if (hcc_mode == MADAKV_HCC_LITERAL)
+    next = __dsub_rn(ph, __ddiv_rn(K, (double)(L - l)));  // Eq. 11 as printed
+  return fmin(fmax(next, lo), hi);
+}
+// Eq. 8 integerised for one head: the visual share rounded half up, the rest to text, surplus of a modality with too
+// few tokens passed to the other.
+__device__ __forceinline__ void split_budget(const AllocParams& p, int64_t u, double Phi, int n, int n_v, int n_t) {
+  const int P = (int)Phi;
+  int bv, bt;
+  if (p.mpa) {
+    bv = (int)floor(__dadd_rn(__dmul_rn(p.pref[u * 2], Phi), 0.5));  // Eq. 8, rounded half up
+    bt = P - bv;
+    if (bv > n_v) { bt += bv - n_v; bv = n_v; }
+    if (bt > n_t) { bv = min(n_v, bv + (bt - n_t)); bt = n_t; }
+  } else {
+    bv = 0;
+    bt = min(P, n);
+  }
+  p.budgets[u * 2] = bv;
+  p.budgets[u * 2 + 1] = bt;
+}
+
 // One block per sequence: Eq. 10-11 as a scalar scan over layers, then Eq. 8 integerised for every (layer, head).
 __global__ void alloc_seq_kernel(AllocParams p) {
   extern __shared__ double s_Phi[];  // [L] rounded budgets, then [L] demand sums (as long long)
@@ -261,34 +323,10 @@ __global__ void alloc_seq_kernel(AllocParams p) {
   const int n = min(p.seq_len[b], p.n_max);
   if (threadIdx.x == 0) s_nv = 0;
   __syncthreads();
-  int c = 0;
-  {
-    const uint8_t* mask = p.mask + (int64_t)b * p.n_max;
-    if ((reinterpret_cast<uintptr_t>(mask) & 15) == 0) {  // 16 tokens per load
-      const int n16 = n >> 4;
-      for (int i = threadIdx.x; i < n16; i += blockDim.x) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(mask) + i);
-        const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k)  // a byte counts if it is not zero
-          c += __popc(((w4[k] | (w4[k] >> 1) | (w4[k] >> 2) | (w4[k] >> 3) | (w4[k] >> 4) | (w4[k] >> 5) | (w4[k] >> 6) |
-                        (w4[k] >> 7)) & 0x01010101u));
-      }
-      for (int i = (n16 << 4) + threadIdx.x; i < n; i += blockDim.x) c += mask[i] ? 1 : 0;
-    } else {
-      for (int i = threadIdx.x; i < n; i += blockDim.x) c += mask[i] ? 1 : 0;
-    }
-  }
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
-  if ((threadIdx.x & 31) == 0 && c) atomicAdd(&s_nv, c);
+  count_visual(p.mask + (int64_t)b * p.n_max, n, &s_nv);
   // Eq. 10's sum over heads, one warp per layer (integers: any order gives the same sum)
   for (int l = threadIdx.x >> 5; l < p.L; l += blockDim.x >> 5) {
-    long long dem = 0;
-    for (int x = threadIdx.x & 31; x < 2 * p.Hkv; x += 32)
-      dem += (long long)p.demand[((int64_t)b * p.L + l) * p.Hkv * 2 + x];
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) dem += __shfl_xor_sync(0xffffffffu, dem, off);
+    const long long dem = layer_demand(p.demand + ((int64_t)b * p.L + l) * p.Hkv * 2, p.Hkv);
     if ((threadIdx.x & 31) == 0) s_dem[l] = dem;
   }
   __syncthreads();
@@ -298,37 +336,47 @@ __global__ void alloc_seq_kernel(AllocParams p) {
     double ph = (double)p.budget[b];
     for (int l = 1; l <= p.L; ++l) {
       p.phi[(int64_t)b * p.L + (l - 1)] = ph;
-      s_Phi[l - 1] = fmin(fmax(floor(__dadd_rn(ph, 0.5)), lo), hi);
-      if (l < p.L) {
-        const double K = __dsub_rn((double)s_dem[l - 1], __dmul_rn((double)p.Hkv, ph));  // Eq. 10
-        double next = ph;
-        if (p.hcc_mode == MADAKV_HCC_PAPER)
-          next = __dsub_rn(ph, __ddiv_rn(K, (double)((long long)p.Hkv * (p.L - l))));  // Eq. 11, per-head units
-        else if (p.hcc_mode == MADAKV_HCC_LITERAL)
-          next = __dsub_rn(ph, __ddiv_rn(K, (double)(p.L - l)));  // Eq. 11 as printed
-        ph = fmin(fmax(next, lo), hi);
-      }
+      s_Phi[l - 1] = rounded_budget(ph, lo, hi);
+      if (l < p.L) ph = next_phi(ph, s_dem[l - 1], p.Hkv, p.L, l, p.hcc_mode, lo, hi);
     }
   }
   __syncthreads();
-  for (int x = threadIdx.x; x < p.L * p.Hkv; x += blockDim.x) {
-    const int l = x / p.Hkv;
-    const int64_t u = (int64_t)b * p.L * p.Hkv + x;
-    const double Phi = s_Phi[l];
-    const int P = (int)Phi;
-    int bv, bt;
-    if (p.mpa) {
-      bv = (int)floor(__dadd_rn(__dmul_rn(p.pref[u * 2], Phi), 0.5));  // Eq. 8, rounded half up
-      bt = P - bv;
-      if (bv > n_v) { bt += bv - n_v; bv = n_v; }
-      if (bt > n_t) { bv = min(n_v, bv + (bt - n_t)); bt = n_t; }
-    } else {
-      bv = 0;
-      bt = min(P, n);
-    }
-    p.budgets[u * 2] = bv;
-    p.budgets[u * 2 + 1] = bt;
+  for (int x = threadIdx.x; x < p.L * p.Hkv; x += blockDim.x)
+    split_budget(p, (int64_t)b * p.L * p.Hkv + x, s_Phi[x / p.Hkv], n, n_v, n_t);
+}
+
+// One block per sequence, one layer of a layer-by-layer pass: the same arithmetic as one trip of the scan above. The
+// per-layer arrays (pref, demand, budgets) hold this layer only; phi [B, depth] is the state carried between calls.
+__global__ void alloc_layer_kernel(AllocParams p, int depth, int layer) {
+  __shared__ int s_nv;
+  __shared__ double s_Phi;
+  __shared__ long long s_dem;
+  const int b = blockIdx.x;
+  const int n = min(p.seq_len[b], p.n_max);
+  if (threadIdx.x == 0) s_nv = 0;
+  __syncthreads();
+  count_visual(p.mask + (int64_t)b * p.n_max, n, &s_nv);
+  if (threadIdx.x < 32) {
+    const long long dem = layer_demand(p.demand + (int64_t)b * p.Hkv * 2, p.Hkv);
+    if (threadIdx.x == 0) s_dem = dem;
   }
+  __syncthreads();
+  const int n_v = s_nv, n_t = n - n_v;
+  if (threadIdx.x == 0) {
+    const double lo = n >= 1 ? 1.0 : 0.0, hi = (double)n;
+    const int l = layer + 1;  // the paper counts layers from 1
+    double ph;
+    if (layer == 0) {
+      ph = (double)p.budget[b];
+      p.phi[(int64_t)b * depth] = ph;
+    } else {
+      ph = p.phi[(int64_t)b * depth + layer];
+    }
+    s_Phi = rounded_budget(ph, lo, hi);
+    if (l < depth) p.phi[(int64_t)b * depth + l] = next_phi(ph, s_dem, p.Hkv, depth, l, p.hcc_mode, lo, hi);
+  }
+  __syncthreads();
+  for (int x = threadIdx.x; x < p.Hkv; x += blockDim.x) split_budget(p, (int64_t)b * p.Hkv + x, s_Phi, n, n_v, n_t);
 }
 
 }  // namespace
@@ -356,6 +404,31 @@ int launch_allocate(const madakv_config& c, const float* psi, const uint8_t* mas
   const int units = c.batch * c.n_layers * c.n_kv_heads;
   alloc_unit_kernel<<<units, NT, 0, st>>>(p);
   alloc_seq_kernel<<<c.batch, 1024, c.n_layers * (sizeof(double) + sizeof(long long)), st>>>(p);
+  return launch_status();
+}
+
+int launch_allocate_layer(const madakv_config& c, int layer, const float* psi, const uint8_t* mask,
+                          const int32_t* seq_len, const int32_t* budget, double* mass, double* pref, int32_t* demand,
+                          double* phi, int32_t* budgets, void* ws, cudaStream_t st) {
+  (void)ws;
+  AllocParams p;
+  p.psi = psi;
+  p.mask = mask;
+  p.seq_len = seq_len;
+  p.budget = budget;
+  p.mass = mass;
+  p.pref = pref;
+  p.demand = demand;
+  p.phi = phi;
+  p.budgets = budgets;
+  p.L = 1;  // the per-layer arrays hold one layer
+  p.Hkv = c.n_kv_heads;
+  p.n_max = c.max_seq_len;
+  p.mpa = c.mpa;
+  p.hcc_mode = c.hcc_mode;
+  p.theta_fix = (u64)((double)c.theta * 4294967296.0);
+  alloc_unit_kernel<<<c.batch * c.n_kv_heads, NT, 0, st>>>(p);
+  alloc_layer_kernel<<<c.batch, 1024, 0, st>>>(p, c.n_layers, layer);
   return launch_status();
 }
 

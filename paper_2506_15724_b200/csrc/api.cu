@@ -69,6 +69,21 @@ int madakv_allocate(const madakv_config* cfg, const float* psi, const uint8_t* m
   return launch_allocate(*cfg, psi, mask, seq_len, budget, mass, pref, demand, phi, budgets, ws, (cudaStream_t)stream);
 }
 
+int madakv_allocate_layer(const madakv_config* cfg, int32_t layer, const float* psi, const uint8_t* mask,
+                          const int32_t* seq_len, const int32_t* budget, double* mass, double* pref, int32_t* demand,
+                          double* phi, int32_t* budgets, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (layer < 0 || layer >= cfg->n_layers) return MADAKV_ESHAPE;
+  if (!psi || !mask || !seq_len || !budget || !mass || !pref || !demand || !phi || !budgets) return MADAKV_EINVAL;
+  if (!aligned16(psi) || ((uintptr_t)mass & 7) || ((uintptr_t)pref & 7) || ((uintptr_t)phi & 7) ||
+      ((uintptr_t)demand & 7) || ((uintptr_t)budgets & 7) || ((uintptr_t)seq_len & 3) || ((uintptr_t)budget & 3))
+    return MADAKV_EALIGN;
+  if ((rc = check_ws(*cfg, ws, ws_bytes))) return rc;
+  return launch_allocate_layer(*cfg, layer, psi, mask, seq_len, budget, mass, pref, demand, phi, budgets, ws,
+                               (cudaStream_t)stream);
+}
+
 int madakv_select(const madakv_config* cfg, const float* psi, const uint8_t* mask, const int32_t* seq_len,
                   const int32_t* budgets, int32_t* kept_len, int64_t* seg_off, int32_t* kept_idx, int64_t capacity,
                   void* ws, size_t ws_bytes, void* stream) {

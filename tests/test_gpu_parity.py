@@ -311,6 +311,54 @@ def test_allocate_and_select_on_crafted_scores(kind, n):
         assert_segments_equal(kept_len, seg_off, buf.kept_idx.cpu().numpy(), kept_idx, "kept_idx")
 
 
+@pytest.mark.parametrize("name", ["tiny_gqa_ragged", "bf16_d128", "bf16_gqa7", "tc_short_seqs"])
+@pytest.mark.parametrize("hcc", [mk.HCC_PAPER, mk.HCC_LITERAL])
+def test_layer_by_layer_pass_equals_the_all_layer_pass(name, hcc):
+    """The streaming use of the library: layer after layer, single-pass scoring with given log-sum-exps, then
+    madakv_allocate_layer carrying phi, then selection and compaction with one-layer configs on slices of K/V. Given
+    the same fp32 scores everything downstream is bit-identical to the all-layer calls; the single-pass scores
+    themselves agree with the two-pass ones to rounding."""
+    wl = SHAPES[name]
+    inp = make_case(wl)
+    g = dev(inp)
+    cfg = config_of(wl, hcc_mode=hcc)
+    cfg1 = config_of(synth.scaled(wl, L=1), hcc_mode=hcc)
+    ref = mk.EvictionBuffers(cfg, capacity_of(wl), want_lse=True)
+    ref.run_eviction(g["q_win"], g["k"], g["v"], g["mask"], g["seq_len"], g["budget"])
+    assert mk.madakv_poll_status(ref.ws) == 0
+    per = wl.Hkv
+    r_len = ref.kept_len.cpu().numpy().reshape(wl.B, wl.L, per)
+    r_off = ref.seg_off.cpu().numpy()
+    r_idx, r_kc, r_vc = ref.kept_idx.cpu().numpy(), ref.k_c, ref.v_c
+    phi = torch.zeros((wl.B, wl.L), dtype=torch.float64, device="cuda")
+    cap1 = capacity_of(synth.scaled(wl, L=1))
+    for l in range(wl.L):
+        one = mk.EvictionBuffers(cfg1, cap1)
+        q_l, k_l, v_l = g["q_win"][:, l:l + 1], g["k"][:, l:l + 1], g["v"][:, l:l + 1]  # views: strides go through
+        mk.madakv_score_lse(cfg1, q_l, k_l, g["seq_len"], ref.lse[:, l:l + 1].contiguous(), one.psi, one.ws)
+        assert psi_close(one.psi.cpu().numpy(), ref.psi[:, l:l + 1].cpu().numpy().astype(np.float64), 1e-4) < 1e-4
+        psi_l = ref.psi[:, l:l + 1].contiguous()  # from here on the same scores as the all-layer pass
+        mk.madakv_allocate_layer(cfg, l, psi_l, g["mask"], g["seq_len"], g["budget"], one.mass, one.pref, one.demand,
+                                 phi, one.budgets, ref.ws)
+        for key in ("mass", "pref", "demand", "budgets"):
+            assert torch.equal(getattr(one, key)[:, 0], getattr(ref, key)[:, l]), (key, l)
+        mk.madakv_select(cfg1, psi_l, g["mask"], g["seq_len"], one.budgets, one.kept_len, one.seg_off, one.kept_idx,
+                         one.ws)
+        mk.madakv_compact(cfg1, k_l, v_l, one.kept_idx, one.seg_off, one.kept_len, one.k_c, one.v_c, one.ws)
+        assert mk.madakv_poll_status(one.ws) == 0
+        o_len = one.kept_len.cpu().numpy().reshape(wl.B, per)
+        o_off, o_idx = one.seg_off.cpu().numpy(), one.kept_idx.cpu().numpy()
+        assert np.array_equal(o_len, r_len[:, l])
+        for b in range(wl.B):
+            for h in range(per):
+                u_all, u_one = (b * wl.L + l) * per + h, b * per + h
+                a0, a1 = int(r_off[u_all]), int(r_off[u_all]) + int(o_len[b, h])
+                c0, c1 = int(o_off[u_one]), int(o_off[u_one]) + int(o_len[b, h])
+                assert np.array_equal(o_idx[c0:c1], r_idx[a0:a1]), (l, b, h)
+                assert torch.equal(one.k_c[c0:c1], r_kc[a0:a1]) and torch.equal(one.v_c[c0:c1], r_vc[a0:a1])
+    assert torch.equal(phi, ref.phi)
+
+
 def test_short_sequences_and_empty_sequence():
     wl = synth.scaled(TINY, B=4, L=1, n=320 + 8, w=8, budget=16)
     inp = synth.make_inputs(wl)

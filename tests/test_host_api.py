@@ -76,6 +76,15 @@ def test_entry_points_reject_bad_arguments_before_launch(lib):
     assert lib.madakv_compact(cref, FAKE, FAKE, good, FAKE, FAKE, FAKE, FAKE, None, 10, FAKE, need, None) == mk.EINVAL
     assert lib.madakv_decode_attn(cref, -1, FAKE, FAKE, None, FAKE, FAKE, FAKE, FAKE, 10, FAKE, None, FAKE, need,
                                   None) == mk.EINVAL
+    # the single-pass scoring needs its normalisers; the per-layer allocation a layer inside the depth
+    assert lib.madakv_score_lse(cref, FAKE, good, FAKE, good, FAKE, None, FAKE, FAKE, need, None) == mk.EINVAL
+    assert lib.madakv_score_lse(cref, FAKE, good, FAKE, good, FAKE, FAKE, FAKE, FAKE, need - 1, None) == mk.EWORKSPACE
+    assert lib.madakv_allocate_layer(cref, 2, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, need,
+                                     None) == mk.ESHAPE
+    assert lib.madakv_allocate_layer(cref, -1, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, need,
+                                     None) == mk.ESHAPE
+    assert lib.madakv_allocate_layer(cref, 0, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, None, FAKE, FAKE, need,
+                                     None) == mk.EINVAL
     # misaligned pointer / stride
     assert lib.madakv_score(cref, odd, good, FAKE, good, FAKE, None, FAKE, FAKE, need, None) == mk.EALIGN
     assert lib.madakv_score(cref, FAKE, st, FAKE, good, FAKE, None, FAKE, FAKE, need, None) == mk.EALIGN
