@@ -241,6 +241,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-full-cache", action="store_true", help="skip the full-cache decode comparison")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--no-single-pass", action="store_true", help="skip the timing of madakv_score_lse (profiling runs)")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: run a reduced-depth copy of the workload")
     args = ap.parse_args()
     wl = synth.CONFIGS[args.workload]
@@ -409,7 +410,7 @@ def main():
         torch.cuda.synchronize()
         return a.elapsed_time(z) / steps
 
-    single_ms = time_single_pass()
+    single_ms = None if args.no_single_pass else time_single_pass()
 
     decode_us = {"compressed": time_decode(buf), "full": None,
                  "compressed_rows_per_head": (rows + wl.units) / wl.units}
@@ -452,9 +453,10 @@ def main():
         "decode": {"us_per_step": decode_us, "algorithmic_bytes": decode_bytes, "gbs_in_step": dec_gbs,
                    "frac_of_measured_peak_in_step": dec_gbs / peak,
                    "gbs_alone": decode_bytes / (decode_us["compressed"] * 1e-6) / 1e9},
-        "single_pass_score": {"ms": single_ms, "gbs": k_bytes / (single_ms * 1e-3) / 1e9,
-                              "frac_of_measured_peak": k_bytes / (single_ms * 1e-3) / 1e9 / peak,
-                              "note": "madakv_score_lse: stage 1 with the rows' log-sum-exps supplied; not part of the step"},
+        "single_pass_score": None if single_ms is None else {
+            "ms": single_ms, "gbs": k_bytes / (single_ms * 1e-3) / 1e9,
+            "frac_of_measured_peak": k_bytes / (single_ms * 1e-3) / 1e9 / peak,
+            "note": "madakv_score_lse: stage 1 with the rows' log-sum-exps supplied; not part of the step"},
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))
