@@ -243,10 +243,16 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--no-single-pass", action="store_true", help="skip the timing of madakv_score_lse (profiling runs)")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: run a reduced-depth copy of the workload")
+    ap.add_argument("--budget", type=int, default=0, help="budget sweeps: another per-head budget than the workload's")
+    ap.add_argument("--theta", type=float, default=0.0, help="budget sweeps: the Eq. 9 threshold calibrated for --budget "
+                    "(python -m oracle.calibrate_theta workload:budget)")
     args = ap.parse_args()
     wl = synth.CONFIGS[args.workload]
     if args.layers > 0:
         wl = synth.scaled(wl, L=args.layers, name=f"{wl.name}[L={args.layers}]")
+    if args.budget > 0:
+        wl = synth.scaled(wl, budget=args.budget, theta=args.theta if args.theta > 0 else wl.theta,
+                          name=f"{wl.name}[budget={args.budget}]")
     if args.impl == "reference":
         run_reference(args, wl)
         return

@@ -4,7 +4,9 @@ matches the nominal per-head budget (bisection on the CPU oracle; inputs from th
 The paper gives theta no value; on synthetic Gaussian logits an arbitrary theta would make the layer compensation
 of Eq. 10-11 run into its clamps. Run once; the printed values are stored in paper_2506_15724_b200/synth.py CONFIGS.
 
-    python -m oracle.calibrate_theta [workload ...]
+    python -m oracle.calibrate_theta [workload | workload:budget ...]
+
+`workload:budget` calibrates for another per-head budget than the stored one (budget sweeps of bench.py).
 """
 import sys
 
@@ -20,8 +22,10 @@ def to_np(t):
     return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
 
 
-def calibrate(name):
+def calibrate(name, budget=None):
     wl = synth.scaled(synth.CONFIGS[name], L=1)
+    if budget is not None:
+        wl = synth.scaled(wl, budget=int(budget))
     inp = synth.make_inputs(wl, want_v=False)
     mask, sl, bud = to_np(inp["mask"]), to_np(inp["seq_len"]), to_np(inp["budget"])
     psi = oracle.score(0 if wl.dtype == "f32" else 1, to_np(inp["q_win"]), to_np(inp["k"]), sl).astype(np.float32)
@@ -39,6 +43,8 @@ def calibrate(name):
 
 
 if __name__ == "__main__":
-    for name in sys.argv[1:] or list(synth.CONFIGS):
-        theta, dem = calibrate(name)
-        print(f"{name}: theta = {theta:.6f}  (layer-1 demand {dem:.1f}, budget {synth.CONFIGS[name].budget})", flush=True)
+    for arg in sys.argv[1:] or list(synth.CONFIGS):
+        name, _, bud = arg.partition(":")
+        budget = int(bud) if bud else synth.CONFIGS[name].budget
+        theta, dem = calibrate(name, budget)
+        print(f"{name}: theta = {theta:.6f}  (layer-1 demand {dem:.1f}, budget {budget})", flush=True)

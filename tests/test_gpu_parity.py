@@ -431,13 +431,13 @@ def test_strided_kv_layout():
 
 
 # sampled (layers, KV heads per layer, decode units) of the full-size checks: the oracle's share grows with g * w * n
-FULL_SIZE_SAMPLES = {"llava": ((0, 13, 31), 3, 6), "qwen": ((0, 27), 2, 4), "batched": ((5, 27), 1, 4),
-                     "long": ((0, 31), 1, 3)}
+FULL_SIZE_SAMPLES = {"llava": ((0, 13, 31), 3, 6), "llava13b": ((7, 39), 2, 4), "qwen": ((0, 27), 2, 4),
+                     "batched": ((5, 27), 1, 4), "long": ((0, 31), 1, 3)}
 
 
 @pytest.mark.parametrize("name", list(FULL_SIZE_SAMPLES))
 def test_full_size_workload_sampled(name):
-    """The four large workloads at full size, in the launch configuration bench.py times: scores of sampled units
+    """The large workloads at full size, in the launch configuration bench.py times: scores of sampled units
     against the oracle, everything downstream of the scores exactly (the oracle's allocation and selection re-run
     on all units of the CUDA path's scores; compacted rows and the decode output on sampled units)."""
     wl = synth.CONFIGS[name]
