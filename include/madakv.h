@@ -54,8 +54,12 @@ enum { MADAKV_F32 = 0, MADAKV_BF16 = 1 };
  *   OFF      phi^l = phi^1 for every layer (ablation "without HCC", Table 3)
  *   PAPER    phi^{l+1} = phi^l - K^l / (H * (L - l)); the factor H reconciles Eq. 8 (phi^l per head) with Eq. 10
  *            (K^l summed over heads)
- *   LITERAL  phi^{l+1} = phi^l - K^l / (L - l), Eq. 11 exactly as printed                                     */
-enum { MADAKV_HCC_OFF = 0, MADAKV_HCC_PAPER = 1, MADAKV_HCC_LITERAL = 2 };
+ *   LITERAL  phi^{l+1} = phi^l - K^l / (L - l), Eq. 11 exactly as printed
+ *   DEMAND   phi as in PAPER, but every layer except the last keeps what Eq. 9 asks for (budgets = demand) instead
+ *            of Eq. 8's split of phi^l. K^l is then what the layer overspent, Eq. 11 reads "what is left, over the
+ *            layers left", and the last layer (Eq. 8 at phi^L) spends the remainder: the total over all layers
+ *            stays L * H * phi^1 up to rounding and the clamps. One reading of "exceeded its budget" under Eq. 10. */
+enum { MADAKV_HCC_OFF = 0, MADAKV_HCC_PAPER = 1, MADAKV_HCC_LITERAL = 2, MADAKV_HCC_DEMAND = 3 };
 
 typedef struct madakv_config {
   uint32_t struct_size;     /* sizeof(madakv_config), checked                                            */

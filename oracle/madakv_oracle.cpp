@@ -157,7 +157,9 @@ int32_t mo_topp_count_f64(const double* psi, int n, double theta) {
 }
 
 // Stages 2-3. Eq. 6 (masses), Eq. 8 (ratio and, after the layer recurrence, integer budgets), Eq. 9 (demand),
-// Eq. 10-11 (layer compensation). hcc_mode: 0 off, 1 divide by H*(L-l), 2 divide by (L-l) as printed.
+// Eq. 10-11 (layer compensation). hcc_mode: 0 off, 1 divide by H*(L-l), 2 divide by (L-l) as printed, 3 as 1 with
+// every layer but the last keeping what Eq. 9 asks for (then Eq. 11 is "what is left over the layers left" and the
+// last layer, budgeted by Eq. 8, spends the remainder: the total stays L*H*phi^1).
 int mo_allocate(int B, int L, int Hkv, int n_max, const float* psi, const uint8_t* mask, const int32_t* seq_len,
                 const int32_t* budget, float theta, int mpa, int hcc_mode, double* mass, double* pref,
                 int32_t* demand, double* phi, int32_t* budgets, int threads) {
@@ -208,13 +210,17 @@ int mo_allocate(int B, int L, int Hkv, int n_max, const float* psi, const uint8_
           bv = 0;
           bt = std::min(P, n);
         }
+        if (hcc_mode == 3 && l < L) {  // the layer keeps its demand (k_m <= n_m by construction)
+          bv = mpa ? demand[u * 2] : 0;
+          bt = mpa ? demand[u * 2 + 1] : std::min(demand[u * 2] + demand[u * 2 + 1], n);
+        }
         budgets[u * 2] = bv;
         budgets[u * 2 + 1] = bt;
       }
       if (l < L) {
         const double K = (double)dem - (double)Hkv * ph;  // Eq. 10
         double next = ph;
-        if (hcc_mode == 1) next = ph - K / (double)((int64_t)Hkv * (L - l));  // Eq. 11, per-head units
+        if (hcc_mode == 1 || hcc_mode == 3) next = ph - K / (double)((int64_t)Hkv * (L - l));  // Eq. 11, per-head units
         if (hcc_mode == 2) next = ph - K / (double)(L - l);                    // Eq. 11 as printed
         ph = std::min(std::max(next, lo), hi);
       }

@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmadakv.so")
 
 MADAKV_F32, MADAKV_BF16 = 0, 1
-HCC_OFF, HCC_PAPER, HCC_LITERAL = 0, 1, 2
+HCC_OFF, HCC_PAPER, HCC_LITERAL, HCC_DEMAND = 0, 1, 2, 3
 STATUS_NAMES = ["OK", "EINVAL", "ESHAPE", "EALIGN", "EWORKSPACE", "ECAPACITY", "EUNSUPPORTED", "ECUDA", "ETIMEOUT",
                 "ESTATIC"]
 (OK, EINVAL, ESHAPE, EALIGN, EWORKSPACE, ECAPACITY, EUNSUPPORTED, ECUDA, ETIMEOUT, ESTATIC) = range(10)

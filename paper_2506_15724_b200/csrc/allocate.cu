@@ -290,15 +290,23 @@ __device__ __forceinline__ double next_phi(double ph, long long dem, int Hkv, in
                                            double hi) {
   const double K = __dsub_rn((double)dem, __dmul_rn((double)Hkv, ph));  // Eq. 10
   double next = ph;
-  if (hcc_mode == MADAKV_HCC_PAPER)
+  if (hcc_mode == MADAKV_HCC_PAPER || hcc_mode == MADAKV_HCC_DEMAND)
     next = __dsub_rn(ph, __ddiv_rn(K, (double)((long long)Hkv * (L - l))));  // Eq. 11, per-head units
   else if (hcc_mode == MADAKV_HCC_LITERAL)
     next = __dsub_rn(ph, __ddiv_rn(K, (double)(L - l)));  // Eq. 11 as printed
   return fmin(fmax(next, lo), hi);
 }
 // Eq. 8 integerised for one head: the visual share rounded half up, the rest to text, surplus of a modality with too
-// few tokens passed to the other.
-__device__ __forceinline__ void split_budget(const AllocParams& p, int64_t u, double Phi, int n, int n_v, int n_t) {
+// few tokens passed to the other. With `keep_demand` (mode DEMAND, every layer but the last) the head keeps what
+// Eq. 9 asked for instead.
+__device__ __forceinline__ void split_budget(const AllocParams& p, int64_t u, double Phi, int n, int n_v, int n_t,
+                                             bool keep_demand) {
+  if (keep_demand) {
+    const int dv = p.demand[u * 2], dt = p.demand[u * 2 + 1];
+    p.budgets[u * 2] = p.mpa ? dv : 0;
+    p.budgets[u * 2 + 1] = p.mpa ? dt : min(dv + dt, n);
+    return;
+  }
   const int P = (int)Phi;
   int bv, bt;
   if (p.mpa) {
@@ -342,7 +350,8 @@ __global__ void alloc_seq_kernel(AllocParams p) {
   }
   __syncthreads();
   for (int x = threadIdx.x; x < p.L * p.Hkv; x += blockDim.x)
-    split_budget(p, (int64_t)b * p.L * p.Hkv + x, s_Phi[x / p.Hkv], n, n_v, n_t);
+    split_budget(p, (int64_t)b * p.L * p.Hkv + x, s_Phi[x / p.Hkv], n, n_v, n_t,
+                 p.hcc_mode == MADAKV_HCC_DEMAND && x / p.Hkv + 1 < p.L);
 }
 
 // One block per sequence, one layer of a layer-by-layer pass: the same arithmetic as one trip of the scan above. The
@@ -376,7 +385,8 @@ __global__ void alloc_layer_kernel(AllocParams p, int depth, int layer) {
     if (l < depth) p.phi[(int64_t)b * depth + l] = next_phi(ph, s_dem, p.Hkv, depth, l, p.hcc_mode, lo, hi);
   }
   __syncthreads();
-  for (int x = threadIdx.x; x < p.Hkv; x += blockDim.x) split_budget(p, (int64_t)b * p.Hkv + x, s_Phi, n, n_v, n_t);
+  for (int x = threadIdx.x; x < p.Hkv; x += blockDim.x)
+    split_budget(p, (int64_t)b * p.Hkv + x, s_Phi, n, n_v, n_t, p.hcc_mode == MADAKV_HCC_DEMAND && layer + 1 < depth);
 }
 
 }  // namespace

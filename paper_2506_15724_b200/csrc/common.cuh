@@ -89,7 +89,7 @@ inline int check_config(const madakv_config* c) {
   if (c->max_seq_len > (1 << 20)) return MADAKV_EUNSUPPORTED;
   if (c->causal != 0 && c->causal != 1) return MADAKV_EINVAL;
   if (c->mpa != 0 && c->mpa != 1) return MADAKV_EINVAL;
-  if (c->hcc_mode < MADAKV_HCC_OFF || c->hcc_mode > MADAKV_HCC_LITERAL) return MADAKV_EINVAL;
+  if (c->hcc_mode < MADAKV_HCC_OFF || c->hcc_mode > MADAKV_HCC_DEMAND) return MADAKV_EINVAL;
   if (c->max_new_tokens < 0) return MADAKV_ESHAPE;
   if (!(c->theta >= 0.0f && c->theta <= 1.0f)) return MADAKV_EINVAL;
   if (!(c->softmax_scale >= 0.0f)) return MADAKV_EINVAL;

@@ -157,7 +157,8 @@ def test_tensor_core_score_item_interleaving(lag, monkeypatch):
 
 
 @pytest.mark.parametrize("name", list(SHAPES))
-@pytest.mark.parametrize("mpa,hcc", [(1, mk.HCC_PAPER), (1, mk.HCC_LITERAL), (0, mk.HCC_OFF), (0, mk.HCC_PAPER)])
+@pytest.mark.parametrize("mpa,hcc", [(1, mk.HCC_PAPER), (1, mk.HCC_LITERAL), (1, mk.HCC_DEMAND), (0, mk.HCC_OFF),
+                                     (0, mk.HCC_PAPER), (0, mk.HCC_DEMAND)])
 def test_staged_allocate_select_compact_are_bit_exact(name, mpa, hcc):
     wl = SHAPES[name]
     inp = make_case(wl)
@@ -312,7 +313,7 @@ def test_allocate_and_select_on_crafted_scores(kind, n):
 
 
 @pytest.mark.parametrize("name", ["tiny_gqa_ragged", "bf16_d128", "bf16_gqa7", "tc_short_seqs"])
-@pytest.mark.parametrize("hcc", [mk.HCC_PAPER, mk.HCC_LITERAL])
+@pytest.mark.parametrize("hcc", [mk.HCC_PAPER, mk.HCC_LITERAL, mk.HCC_DEMAND])
 def test_layer_by_layer_pass_equals_the_all_layer_pass(name, hcc):
     """The streaming use of the library: layer after layer, single-pass scoring with given log-sum-exps, then
     madakv_allocate_layer carrying phi, then selection and compaction with one-layer configs on slices of K/V. Given

@@ -241,6 +241,35 @@ def test_allocate_invariants_and_mask_swap():
     np.testing.assert_array_equal(nompa["phi"], al["phi"])
 
 
+def test_allocate_demand_mode_conserves_the_total_budget():
+    """Mode DEMAND (each layer but the last keeps what Eq. 9 asks for, phi follows Eq. 10-11 in per-head units): by
+    induction phi^{l+1} * H * (L - l) = L * H * B - (spent so far), so with the last layer budgeted by Eq. 8 the total
+    kept over all layers is L * H * B up to the rounding of the last Phi. Random scores, demands well inside the
+    clamps."""
+    rng = np.random.RandomState(5)
+    B, L, H, n = 2, 6, 3, 400
+    psi = rng.gamma(0.6, 1.0, size=(B, L, H, n)).astype(np.float32)
+    mask = (rng.rand(B, n) < 0.5).astype(np.uint8)
+    sl = np.array([n, n - 37], np.int32)
+    bud = np.array([120, 90], np.int32)
+    al = oracle.allocate(psi, mask, sl, bud, 0.55, hcc_mode=3)
+    pa = oracle.allocate(psi, mask, sl, bud, 0.55, hcc_mode=1)
+    np.testing.assert_array_equal(al["demand"], pa["demand"])
+    for b in range(B):
+        assert al["phi"][b, 0] == bud[b]
+        assert (al["phi"][b] > 1).all() and (al["phi"][b] < sl[b]).all()  # no clamp was hit
+        np.testing.assert_array_equal(al["budgets"][b, : L - 1], al["demand"][b, : L - 1])
+        spent = 0
+        for l in range(L - 1):  # the recurrence, re-derived from its meaning: what is left over the layers left
+            spent += int(al["demand"][b, l].sum())
+            want = (L * H * int(bud[b]) - spent) / (H * (L - 1 - l))
+            assert abs(al["phi"][b, l + 1] - want) < 1e-9 * want
+        Phi_last = math.floor(al["phi"][b, L - 1] + 0.5)
+        assert al["budgets"][b, L - 1].sum() == H * Phi_last
+        total = spent + int(al["budgets"][b, L - 1].sum())
+        assert abs(total - L * H * int(bud[b])) <= H / 2 + 1e-9
+
+
 def test_allocate_surplus_spills_to_other_modality():
     n = 40
     mask = np.zeros((1, n), np.uint8)
