@@ -21,7 +21,7 @@ struct CompactParams {
   const int32_t* seq_len;  // unused (bounds come from n_max); kept for symmetry
   int64_t capacity;
   int64_t stride_b, stride_l, stride_h, stride_t;  // bytes
-  int L, Hkv, n_max, row_bytes;
+  int L, Hkv, n_max, row_bytes, headroom;
 };
 
 template <int LPR>  // 16-byte lanes per row
@@ -31,7 +31,8 @@ __global__ void __launch_bounds__(NT) compact_kernel(CompactParams p) {
   const int row0 = blockIdx.x * ROWS_PER_BLOCK;
   if (row0 >= len) return;
   const int64_t off = p.seg_off[u];
-  if (off + len > p.capacity) return;  // never write past the ragged cache; select has flagged the overflow
+  // a segment that selection refused (MADAKV_ECAPACITY: it would end beyond the cache) has no index list: skip it
+  if (off + len + p.headroom > p.capacity) return;
   const int h = u % p.Hkv, l = (u / p.Hkv) % p.L, b = u / (p.Hkv * p.L);
   const int64_t src_base = b * p.stride_b + l * p.stride_l + h * p.stride_h;
   const int lane = threadIdx.x % LPR, sub = threadIdx.x / LPR;
@@ -75,6 +76,7 @@ int launch_compact(const madakv_config& c, const void* k, const void* v, madakv_
   p.Hkv = c.n_kv_heads;
   p.n_max = c.max_seq_len;
   p.row_bytes = c.head_dim * e;
+  p.headroom = c.max_new_tokens;
   const int units = c.batch * c.n_layers * c.n_kv_heads;
   if (units > 65535) return MADAKV_EUNSUPPORTED;
   const dim3 grid((c.max_seq_len + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK, units);

@@ -48,6 +48,15 @@ __device__ __forceinline__ int unit_of(const DecodeParams& p, int y) {
   return (b * p.L + p.layer) * p.Hkv + h;
 }
 
+// Rows of unit u's segment that attention may read. A segment that does not lie inside the cache (selection reported
+// MADAKV_ECAPACITY and left it unwritten), or that is longer than the split partials provide for, counts as empty:
+// nothing beyond `capacity` rows or beyond the workspace is ever touched.
+__device__ __forceinline__ int segment_rows(const DecodeParams& p, int u) {
+  const int len = p.kept_len[u];
+  const int64_t off = p.seg_off[u];
+  return (len < 0 || off < 0 || off + (int64_t)len > p.capacity || len > p.splits * kDecodeChunk) ? 0 : len;
+}
+
 template <int ROW_BYTES>
 __global__ void append_kernel(DecodeParams p, int n_sel) {
   constexpr int LPR = ROW_BYTES / 16;
@@ -106,7 +115,7 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
   __shared__ float s_m[GROUPS][G], s_l[GROUPS][G];
 
   const int u = unit_of(p, blockIdx.y);
-  const int len = p.kept_len[u];
+  const int len = segment_rows(p, u);
   // split 0 always reports, so an empty segment is well defined; a block beyond the segment has nothing to do
   if (blockIdx.x != 0 && (int)blockIdx.x * kDecodeChunk >= len) return;
   const int64_t off = p.seg_off[u];
@@ -292,7 +301,7 @@ __global__ void __launch_bounds__(kMmaWarps * 32, 3) decode_partial_mma_kernel(D
   extern __shared__ __align__(16) unsigned char dsmem[];
 
   const int u = unit_of(p, blockIdx.y);
-  const int len = p.kept_len[u];
+  const int len = segment_rows(p, u);
   if (blockIdx.x != 0 && (int)blockIdx.x * kDecodeChunk >= len) return;
   const int64_t off = p.seg_off[u];
   const int h = u % p.Hkv, bl = u / p.Hkv;
@@ -464,7 +473,7 @@ __global__ void __launch_bounds__(D) decode_merge_kernel(DecodeParams p) {
   }
   const int bl = row / p.Hq, hq = row % p.Hq;
   const int u = bl * p.Hkv + hq / p.g;
-  const int len = p.kept_len[u];
+  const int len = segment_rows(p, u);
   const int used = max(1, (len + kDecodeChunk - 1) / kDecodeChunk);
   const float* part = p.part + (int64_t)row * p.splits * (D + 2);
   const int c = threadIdx.x;

@@ -392,7 +392,7 @@ def test_capacity_overflow_is_reported_not_written():
     inp = make_case(wl)
     cfg = config_of(wl)
     g = dev(inp)
-    small = 100  # rows: far below 4 units x 129
+    small = 300  # rows: two of the 4 units x 129 rows fit
     buf = mk.EvictionBuffers(cfg, small)
     guard = torch.full((small + 64,), -7, dtype=torch.int32, device="cuda")
     buf.kept_idx = guard[:small]
@@ -400,6 +400,17 @@ def test_capacity_overflow_is_reported_not_written():
     assert mk.madakv_poll_status(buf.ws) == mk.ECAPACITY
     assert mk.madakv_poll_status(buf.ws) == 0  # cleared by the poll
     assert (guard[small:] == -7).all()
+    # decode over a cache some of whose segments did not fit: those count as empty (zeros out), nothing beyond the
+    # cache is read, the segments that fit are attended to as usual
+    q, _, _ = [t.cuda() for t in synth.make_decode_step(wl, 0)]
+    buf.run_decode(q)
+    torch.cuda.synchronize()
+    assert mk.madakv_poll_status(buf.ws) == 0
+    lens, offs = buf.kept_len.cpu().numpy(), buf.seg_off.cpu().numpy()
+    out = buf.out.float().cpu().numpy().reshape(wl.units, wl.g, wl.d)
+    fits = offs[:-1] + lens + wl.max_new_tokens <= small
+    assert fits.any() and not fits.all()
+    assert np.isfinite(out).all() and (out[~fits] == 0).all() and (np.abs(out[fits]).sum(axis=(1, 2)) > 0).all()
     # appending beyond the headroom: first append fits, second is refused and leaves the cache unchanged
     buf = mk.EvictionBuffers(cfg, capacity_of(wl))
     buf.run_eviction(g["q_win"], g["k"], g["v"], g["mask"], g["seq_len"], g["budget"])
