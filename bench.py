@@ -418,6 +418,42 @@ def main():
 
     single_ms = None if args.no_single_pass else time_single_pass()
 
+    # ---- the layer-by-layer order (a layer is evicted right after its prefill): per layer single-pass scoring with
+    # the prefill's log-sum-exps, madakv_allocate_layer carrying phi, selection and compaction of that layer
+    def time_streamed(steps=5):
+        cfg1 = mk.make_config(wl.torch_dtype, wl.B, 1, wl.Hq, wl.Hkv, wl.d, wl.n, wl.w,
+                              max_new_tokens=wl.max_new_tokens, theta=wl.theta)
+        one = mk.EvictionBuffers(cfg1, cap // wl.L + wl.B * wl.Hkv, device=dev)
+        lse = torch.empty((wl.B, wl.L, wl.Hq, wl.w), dtype=torch.float32, device=dev)
+        mk.madakv_score(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, buf.psi, buf.ws)
+        lse_l = [lse[:, l:l + 1].contiguous() for l in range(wl.L)]
+        phi = torch.zeros((wl.B, wl.L), dtype=torch.float64, device=dev)
+
+        def one_pass():
+            for l in range(wl.L):
+                q_l, k_l, v_l = inp["q_win"][:, l:l + 1], inp["k"][:, l:l + 1], inp["v"][:, l:l + 1]
+                mk.madakv_score_lse(cfg1, q_l, k_l, inp["seq_len"], lse_l[l], one.psi, one.ws)
+                mk.madakv_allocate_layer(buf.cfg, l, one.psi, inp["mask"], inp["seq_len"], inp["budget"], one.mass,
+                                         one.pref, one.demand, phi, one.budgets, buf.ws)
+                mk.madakv_select(cfg1, one.psi, inp["mask"], inp["seq_len"], one.budgets, one.kept_len, one.seg_off,
+                                 one.kept_idx, one.ws)
+                mk.madakv_compact(cfg1, k_l, v_l, one.kept_idx, one.seg_off, one.kept_len, one.k_c, one.v_c, one.ws)
+
+        for _ in range(2):
+            one_pass()
+        torch.cuda.synchronize()
+        if mk.madakv_poll_status(one.ws) != 0 or mk.madakv_poll_status(buf.ws) != 0:
+            return None
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            one_pass()
+        z.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(z) / steps
+
+    streamed_ms = None if args.no_single_pass else time_streamed()
+
     decode_us = {"compressed": time_decode(buf), "full": None,
                  "compressed_rows_per_head": (rows + wl.units) / wl.units}
     if not args.no_full_cache and rank == 0:
@@ -463,6 +499,10 @@ def main():
             "ms": single_ms, "gbs": k_bytes / (single_ms * 1e-3) / 1e9,
             "frac_of_measured_peak": k_bytes / (single_ms * 1e-3) / 1e9 / peak,
             "note": "madakv_score_lse: stage 1 with the rows' log-sum-exps supplied; not part of the step"},
+        "streamed_pass": None if streamed_ms is None else {
+            "ms": streamed_ms, "tokens_per_s": tokens / (streamed_ms * 1e-3), "launches": wl.L * 7,
+            "note": "stages 1-4 layer by layer (madakv_score_lse, madakv_allocate_layer, select and compact with "
+                    "one-layer configs), launch-bound at this depth; not part of the step"},
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))
