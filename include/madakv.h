@@ -97,7 +97,8 @@ int madakv_workspace_bytes(const madakv_config* cfg, size_t* bytes_out);
  * cfg->causal the row sees keys 0..position. psi[u][i] = 0 for i >= seq_len[b]. Accumulation is fp32.
  *   q_win   [B, L, H_q, w, d]  dtype, strides sq
  *   k       [B, L, H_kv, n_max, d] dtype, strides sk
- *   seq_len [B] int32, 0 <= seq_len[b] <= n_max
+ *   seq_len [B] int32, 0 <= seq_len[b] <= n_max (device data: a value outside the range is used as the nearest
+ *           bound, in every call that takes seq_len)
  *   lse     [B, L, H_q, w] fp32, natural-log sum-exp of every window row's scaled logits. The call computes
  *           these values and stores them here when `lse` is non-null (may be null).
  *   psi     [B, L, H_kv, n_max] fp32, contiguous, written in full

@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
 
   const int u = blockIdx.x;
   const int b = u / (p.Hkv * p.L);
-  const int n = min(p.seq_len[b], p.n_max);
+  const int n = clamped_len(p.seq_len, b, p.n_max);
   const float* psi = p.psi + (int64_t)u * p.n_max;
   const uint8_t* mask = p.mask + (int64_t)b * p.n_max;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -328,7 +328,7 @@ __global__ void alloc_seq_kernel(AllocParams p) {
   long long* s_dem = reinterpret_cast<long long*>(s_Phi + p.L);
   __shared__ int s_nv;
   const int b = blockIdx.x;
-  const int n = min(p.seq_len[b], p.n_max);
+  const int n = clamped_len(p.seq_len, b, p.n_max);
   if (threadIdx.x == 0) s_nv = 0;
   __syncthreads();
   count_visual(p.mask + (int64_t)b * p.n_max, n, &s_nv);
@@ -361,7 +361,7 @@ __global__ void alloc_layer_kernel(AllocParams p, int depth, int layer) {
   __shared__ double s_Phi;
   __shared__ long long s_dem;
   const int b = blockIdx.x;
-  const int n = min(p.seq_len[b], p.n_max);
+  const int n = clamped_len(p.seq_len, b, p.n_max);
   if (threadIdx.x == 0) s_nv = 0;
   __syncthreads();
   count_visual(p.mask + (int64_t)b * p.n_max, n, &s_nv);

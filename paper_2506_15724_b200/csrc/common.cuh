@@ -130,6 +130,11 @@ __device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v 
 __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 
 // Order-preserving integer image of a non-negative importance value; anything not > 0 (incl. NaN) maps to 0.
+// Length of sequence b as the kernels use it: the caller's seq_len[b] brought into [0, n_max] (the header asks for
+// that range; a value outside it must not turn into an index outside the arrays).
+__device__ __forceinline__ int clamped_len(const int32_t* seq_len, int b, int n_max) {
+  return max(0, min(seq_len[b], n_max));
+}
 __device__ __forceinline__ uint32_t psi_key(float x) { return x > 0.0f ? __float_as_uint(x) : 0u; }
 // floor(x * 2^32) of a key produced by psi_key.
 __device__ __forceinline__ unsigned long long psi_fix(uint32_t key) {

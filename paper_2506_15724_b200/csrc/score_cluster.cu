@@ -194,7 +194,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
       bool ok = true;
       for (int u = cluster; ok && u < p.units; u += n_clusters) {
         const int h = u % p.Hkv, l = (u / p.Hkv) % p.L, b = u / (p.Hkv * p.L);
-        const int n = min(p.seq_len[b], p.n_max);
+        const int n = clamped_len(p.seq_len, b, p.n_max);
         int tile0, my_tiles;
         my_share(n, tile0, my_tiles);
         if (my_tiles == 0) continue;
@@ -240,7 +240,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
       bool ok = true;
       for (int u = cluster; ok && u < p.units; u += n_clusters) {
         const int b = u / (p.Hkv * p.L);
-        const int n = min(p.seq_len[b], p.n_max);
+        const int n = clamped_len(p.seq_len, b, p.n_max);
         int tile0, my_tiles;
         my_share(n, tile0, my_tiles);
         if (my_tiles == 0) continue;
@@ -307,7 +307,7 @@ score_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_co
       if (u >= b_end) {
         b = u / (p.Hkv * p.L);
         b_end = (b + 1) * p.Hkv * p.L;
-        n = min(p.seq_len[b], p.n_max);
+        n = clamped_len(p.seq_len, b, p.n_max);
         my_share(n, tile0, my_tiles);
         all_bound = (n >= p.w) ? (p.causal ? n - p.w + 1 : n) : 0;  // keys below are seen by every row
         tiles_end = ((n + kTileKeys - 1) / kTileKeys) * kTileKeys;

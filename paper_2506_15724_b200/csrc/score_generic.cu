@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(NT) score_stats_kernel(ScoreParams p) {
   float* qs = smem + KT * (D + 4);
   const int u = blockIdx.y, chunk = blockIdx.x;
   const int h = u % p.Hkv, l = (u / p.Hkv) % p.L, b = u / (p.Hkv * p.L);
-  const int n = min(p.seq_len[b], p.n_max);
+  const int n = clamped_len(p.seq_len, b, p.n_max);
   const int kl = threadIdx.x % 16, rg = threadIdx.x / 16;
   const int key_begin = chunk * kScoreChunk, key_end = min(n, key_begin + kScoreChunk);
   const T* kbase = reinterpret_cast<const T*>(p.k) + b * p.sk.batch + l * p.sk.layer + h * p.sk.head;
@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(NT) score_psi_kernel(ScoreParams p) {
   __shared__ float lse_s[RT];
   const int u = blockIdx.y, key0 = blockIdx.x * KT;
   const int h = u % p.Hkv, l = (u / p.Hkv) % p.L, b = u / (p.Hkv * p.L);
-  const int n = min(p.seq_len[b], p.n_max);
+  const int n = clamped_len(p.seq_len, b, p.n_max);
   float* psi = p.psi + (int64_t)u * p.n_max;
   if (key0 >= n) {  // beyond the sequence: psi = 0
     for (int x = threadIdx.x; x < KT; x += NT)

@@ -125,7 +125,7 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     u = item / p.splits;
     const int split = item % p.splits;
     const int b = u / (p.Hkv * p.L);
-    const int n = min(p.seq_len[b], p.n_max);
+    const int n = clamped_len(p.seq_len, b, p.n_max);
     key_begin = split * kSplitKeys;
     tiles = key_begin < n ? (min(n, key_begin + kSplitKeys) - key_begin + kTileKeys - 1) / kTileKeys : 0;
   };
@@ -247,7 +247,7 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
       item_of(item, u, key_begin, tiles);
       const int split = item % p.splits;
       const int b = u / (p.Hkv * p.L);
-      const int n = min(p.seq_len[b], p.n_max);
+      const int n = clamped_len(p.seq_len, b, p.n_max);
       float* psi = p.psi + (int64_t)u * p.n_max;
       // keys the row may see: [0, vis)
       int vis = 0;

@@ -201,7 +201,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
       Item it;
       for (int idx = 0; ok && get_item(blockIdx.x, gridDim.x, idx, total_chunks, p.lag, p.cpu, it); ++idx) {
         const int h = it.unit % p.Hkv, l = (it.unit / p.Hkv) % p.L, b = it.unit / (p.Hkv * p.L);
-        const int n = min(p.seq_len[b], p.n_max);
+        const int n = clamped_len(p.seq_len, b, p.n_max);
         const int key_begin = it.chunk * kItemKeys;
         if (key_begin >= n) continue;  // nothing to load for this item
         const int ib = active % kItemBufs;
@@ -263,7 +263,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
       Item it;
       for (int idx = 0; ok && get_item(blockIdx.x, gridDim.x, idx, total_chunks, p.lag, p.cpu, it); ++idx) {
         const int b = it.unit / (p.Hkv * p.L);
-        const int n = min(p.seq_len[b], p.n_max);
+        const int n = clamped_len(p.seq_len, b, p.n_max);
         const int key_begin = it.chunk * kItemKeys;
         if (key_begin >= n) continue;
         const int ib = active % kItemBufs;
@@ -336,7 +336,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
     Item it;
     for (int idx = 0; ok && get_item(blockIdx.x, gridDim.x, idx, total_chunks, p.lag, p.cpu, it); ++idx) {
       const int h = it.unit % p.Hkv, bl = it.unit / p.Hkv, b = bl / p.L;
-      const int n = min(p.seq_len[b], p.n_max);
+      const int n = clamped_len(p.seq_len, b, p.n_max);
       const int key_begin = it.chunk * kItemKeys;
       float* psi = p.psi + (int64_t)it.unit * p.n_max;
       if (key_begin >= n) {

@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(1024) seg_scan_kernel(SelParams p) {
   __shared__ int s_cnt;
   // visual tokens among the first seq_len[b] positions of every sequence
   for (int b = 0; b < p.B; ++b) {
-    const int n = min(p.seq_len[b], p.n_max);
+    const int n = clamped_len(p.seq_len, b, p.n_max);
     const uint8_t* mask = p.mask + (int64_t)b * p.n_max;
     if (threadIdx.x == 0) s_cnt = 0;
     __syncthreads();
@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(1024) seg_scan_kernel(SelParams p) {
     long long v = 0;
     if (u < p.units) {
       const int b = u / (p.Hkv * p.L);
-      const int n = min(p.seq_len[b], p.n_max);
+      const int n = clamped_len(p.seq_len, b, p.n_max);
       const int n_v = p.seq_nv[b];
       const int len = (p.mpa ? min(max(p.budgets[2 * u], 0), n_v) : 0) + min(max(p.budgets[2 * u + 1], 0), n - n_v);
       p.kept_len[u] = len;
@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
 
   const int u = blockIdx.x;
   const int b = u / (p.Hkv * p.L);
-  const int n = min(p.seq_len[b], p.n_max);
+  const int n = clamped_len(p.seq_len, b, p.n_max);
   const float* psi = p.psi + (int64_t)u * p.n_max;
   const uint8_t* mask = p.mask + (int64_t)b * p.n_max;
   const int64_t off0 = p.seg_off[u];

@@ -387,6 +387,30 @@ def test_short_sequences_and_empty_sequence():
     assert (buf.out[2] == 0).all()  # empty sequence: zeros
 
 
+@pytest.mark.parametrize("name", ["tiny_gqa_ragged", "tc_short_seqs", "bf16_gqa7"])
+def test_sequence_lengths_outside_the_range_are_clamped(name):
+    # seq_len[b] is device data the host cannot check: a value above n_max acts as n_max, a negative one as 0
+    wl = SHAPES[name]
+    inp = synth.make_inputs(wl, device="cpu")
+    g = dev(inp)
+    cfg = config_of(wl)
+    good = torch.full((wl.B,), wl.n, dtype=torch.int32)
+    odd = good.clone()
+    odd[0] = wl.n + 9
+    if wl.B > 1:
+        good[1], odd[1] = 0, -3
+    res = []
+    for sl in (good, odd):
+        buf = mk.EvictionBuffers(cfg, capacity_of(wl))
+        buf.run_eviction(g["q_win"], g["k"], g["v"], g["mask"], sl.cuda(), g["budget"])
+        q, kn, vn = [t.cuda() for t in synth.make_decode_step(wl, 0)]
+        buf.run_decode(q, kn, vn)
+        assert mk.madakv_poll_status(buf.ws) == 0
+        res.append(buf)
+    for key in ("psi", "budgets", "kept_len", "seg_off", "kept_idx", "k_c", "v_c", "out"):
+        assert torch.equal(getattr(res[0], key), getattr(res[1], key)), key
+
+
 def test_capacity_overflow_is_reported_not_written():
     wl = synth.scaled(TINY, L=1, max_new_tokens=1)
     inp = make_case(wl)
