@@ -34,18 +34,24 @@ struct AllocParams {
 
 // Shared histograms of one radix pass: per (modality, digit) a count and an exact 64-bit mass kept as two 32-bit
 // words (32-bit shared atomics are native; the carry of the low word is detected from the value the atomic returns).
+// Bucket b sits at word b + b / 32: the bucket walk has lane j read buckets 8j .. 8j+7, which in a dense array would be
+// an 8-way bank conflict on every load; with the skew the 32 lanes of a load hit 32 different banks.
+constexpr int kHistWords = 512 + 16;
+__device__ __forceinline__ int hist_slot(int bucket) { return bucket + (bucket >> 5); }
 struct Hist {
-  unsigned int cnt[512], mlo[512], mhi[512];
+  unsigned int cnt[kHistWords], mlo[kHistWords], mhi[kHistWords];
 };
 __device__ __forceinline__ void hist_add(Hist& h, int bucket, u64 m) {
-  atomicAdd(&h.cnt[bucket], 1u);
+  const int s = hist_slot(bucket);
+  atomicAdd(&h.cnt[s], 1u);
   const unsigned int add = (unsigned int)m;
-  const unsigned int old = atomicAdd(&h.mlo[bucket], add);
+  const unsigned int old = atomicAdd(&h.mlo[s], add);
   const unsigned int hi = (unsigned int)(m >> 32) + ((unsigned int)(old + add) < old ? 1u : 0u);
-  if (hi) atomicAdd(&h.mhi[bucket], hi);  // rare: importance values are mostly below 1, carries are few
+  if (hi) atomicAdd(&h.mhi[s], hi);  // rare: importance values are mostly below 1, carries are few
 }
 __device__ __forceinline__ u64 hist_mass(const Hist& h, int bucket) {
-  return ((u64)h.mhi[bucket] << 32) | h.mlo[bucket];
+  const int s = hist_slot(bucket);
+  return ((u64)h.mhi[s] << 32) | h.mlo[s];
 }
 
 // One warp walks the 256 buckets of modality m in ascending digit order (digits are taken from kmax - key, so this
@@ -61,7 +67,7 @@ __device__ __forceinline__ int descend(const Hist& h, int m, u64 need_c, u64& ab
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     ms[j] = hist_mass(h, m * 256 + lane * 8 + j);
-    cs[j] = h.cnt[m * 256 + lane * 8 + j];
+    cs[j] = h.cnt[hist_slot(m * 256 + lane * 8 + j)];
     lm += ms[j];
     lc += cs[j];
   }
@@ -76,21 +82,26 @@ __device__ __forceinline__ int descend(const Hist& h, int m, u64 need_c, u64& ab
       sc += tc;
     }
   }
-  u64 a = above + (sm - lm);
-  unsigned int ac = above_c + (sc - lc);
-  int found = -1;
-  unsigned int c_at = 0;
+  // within the lane: the running mass before each of its buckets is monotone, so the first bucket that reaches the
+  // threshold is the number of buckets that do not (no data-dependent branches)
+  const u64 a0 = above + (sm - lm);
+  const unsigned int ac0 = above_c + (sc - lc);
+  u64 run = a0;
+  int below = 0;
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    if (found < 0) {
-      if (a + ms[j] >= need_c || (lane == 31 && j == 7)) {
-        found = j;
-        c_at = cs[j];
-      } else {
-        a += ms[j];
-        ac += cs[j];
-      }
-    }
+    run += ms[j];
+    below += run < need_c ? 1 : 0;
+  }
+  int found = below < 8 ? below : (lane == 31 ? 7 : -1);
+  u64 a = a0;
+  unsigned int ac = ac0, c_at = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const bool before = j < (found < 0 ? 8 : found);
+    a += before ? ms[j] : 0ull;
+    ac += before ? cs[j] : 0u;
+    c_at = j == found ? cs[j] : c_at;
   }
   const unsigned int hit = __ballot_sync(kFull, found >= 0);  // lane 31 always hits
   const int win = __ffs(hit) - 1;
@@ -177,7 +188,7 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
   for (int rem = top, pass = 0; rem > 0; ++pass) {
     const int bits = min(rem, 8), shift = rem - bits;
     const uint32_t dmask = (1u << bits) - 1u;
-    for (int x = threadIdx.x; x < 512; x += NT) {
+    for (int x = threadIdx.x; x < kHistWords; x += NT) {
       hist.cnt[x] = 0;
       hist.mlo[x] = 0;
       hist.mhi[x] = 0;
