@@ -208,7 +208,8 @@ int madakv_poll_status(void* ws, void* stream, int32_t* status_out);
 
 const char* madakv_status_string(int status);
 
-/* Library version, bumped when the ABI changes. */
+/* Library version, bumped when the ABI changes. 2: madakv_score_lse, madakv_allocate_layer and MADAKV_HCC_DEMAND added
+ * (nothing that version 1 had was changed). */
 int madakv_abi_version(void);
 
 #ifdef __cplusplus

@@ -6,7 +6,7 @@ using namespace madakv;
 
 extern "C" {
 
-int madakv_abi_version(void) { return 1; }
+int madakv_abi_version(void) { return 2; }
 
 const char* madakv_status_string(int s) {
   switch (s) {

@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol(lib):
     for name in declared:
         assert hasattr(lib, name), name
     assert declared == set(mk.EXPORTS)
-    assert lib.madakv_abi_version() == 1
+    assert lib.madakv_abi_version() == 2
     assert mk.madakv_status_string(mk.ECAPACITY) == "ragged cache capacity exceeded"
 
 
