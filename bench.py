@@ -1,11 +1,15 @@
 #!/usr/bin/env python
 """Benchmark of the MadaKV eviction pass on B200: prompt tokens evicted per second, decode-step latency and the
-fraction of the HBM roofline, with the CPU oracle timed beside it.
+fraction of the roofline, with the CPU oracle timed beside it.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llava] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload long] [--impl ours|reference]
 
 A step is one pass of the whole hot path over one batch of synthetic input: stages 1-4 (score, allocate, select,
 compact) for every layer and head, then one decode step (append + attention over the ragged cache, all layers).
+The headline (`value`, `roofline`, `e2e`, `cpu_baseline`) is measured on the largest single-GPU workload (`long`:
+131072 tokens, 32 layers, 32 query / 8 KV heads, window 64); the `workloads` object of the same JSON line carries the
+stage times, roofline fractions and decode latencies of every other benchmark workload (llava, qwen at budgets
+1024 / 2048 / 4096, batched), each from its own timed steps.
 With N > 1 (torchrun, one rank per GPU) every rank runs its own batch (different seed): the path shards over
 independent sequences with no data-path collective, so scaling is weak and the value is N batches / slowest rank.
 """
@@ -27,6 +31,12 @@ from paper_2506_15724_b200 import synth  # noqa: E402
 METRIC = "prompt tokens evicted/sec"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+# exp2 results per clock and SM of the special-function unit, measured on this machine's B200 with a register-only
+# kernel of independent ex2.approx chains (15.99 at 16 and at 32 warps per SM, CUDA events and clock64 agree)
+EXP2_PER_CLK_PER_SM = 15.99
+HEADLINE = "long"
+OTHER_WORKLOADS = ("llava", "qwen1024", "qwen", "qwen4096", "batched")
 
 
 def measured_peaks():
@@ -35,6 +45,20 @@ def measured_peaks():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def ncu_traffic(kernel, workload):
+    """DRAM bytes (read + write) per launch of `kernel` on `workload`, from the committed ncu summary table
+    (profiles/dram_traffic.txt: kernel, workload, bytes per launch); None when no capture of the present kernel exists."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) >= 3 and not line.startswith("#") and parts[0] == kernel and parts[1] == workload:
+                    return float(parts[2])
+    except Exception:
+        pass
+    return None
 
 
 class ClockSampler:
@@ -147,55 +171,94 @@ def job_throughput(total_ms, steps, tokens_all_ranks):
     return tokens_all_ranks / (total_ms / steps * 1e-3)
 
 
-def cpu_oracle_leg(wl, seconds_target=15.0):
-    """The oracle, as it stands, on a bounded sample of the workload: the first layers of the same inputs (all of
-    them when the whole workload fits the time target), repeated until about `seconds_target` of CPU work is done."""
-    import numpy as np
+# ----------------------------------------------------------------------------------------------- CPU oracle legs
+class OracleSample:
+    """The oracle, as it stands, on a bounded sample of a workload: the first layers of the same seeded inputs (all
+    KV heads, all tokens, one decode step). The sample is sized by time: as many layers as give every host thread a
+    unit, as long as one pass stays near `seconds_per_pass`."""
 
-    import oracle
+    def __init__(self, wl, seconds_per_pass):
+        import numpy as np
 
-    def to_np(t):
-        t = t.detach().cpu().contiguous()
-        return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
+        import oracle
 
-    code = 0 if wl.dtype == "f32" else 1
+        self.oracle, self.np, self.wl = oracle, np, wl
+        self.cores = oracle.hardware_threads()
+        self.layers = 1
+        self._prepare(1)
+        t0 = time.perf_counter()
+        self.one_pass()
+        t1 = time.perf_counter() - t0
+        per_layer = wl.B * wl.Hkv
+        # one pass of `layers` layers takes about t1 * ceil(layers * per_layer / cores) / ceil(per_layer / cores)
+        rounds1 = -(-per_layer // self.cores)
+        want = 1
+        for layers in range(2, wl.L + 1):
+            rounds = -(-layers * per_layer // self.cores)
+            if t1 * rounds / rounds1 > seconds_per_pass:
+                break
+            want = layers
+            if layers * per_layer >= self.cores and t1 * rounds / rounds1 > seconds_per_pass / 2:
+                break
+        if want > 1:
+            self.layers = want
+            self._prepare(want)
 
-    def prepare(layers):
+    def _prepare(self, layers):
+        np, wl = self.np, self.wl
+
+        def to_np(t):
+            t = t.detach().cpu().contiguous()
+            return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
+
         sub = synth.scaled(wl, L=layers)
         inp = synth.make_inputs(sub)
-        q, k, v = to_np(inp["q_win"]), to_np(inp["k"]), to_np(inp["v"])
-        mask, sl, bud = to_np(inp["mask"]), to_np(inp["seq_len"]), to_np(inp["budget"])
-        dq, kn, vn = [to_np(t) for t in synth.make_decode_step(sub, 0)]
-        cap = sub.units * (sub.n + sub.max_new_tokens)
+        self.sub = sub
+        self.q, self.k, self.v = to_np(inp["q_win"]), to_np(inp["k"]), to_np(inp["v"])
+        self.mask, self.sl, self.bud = to_np(inp["mask"]), to_np(inp["seq_len"]), to_np(inp["budget"])
+        self.dq, self.kn, self.vn = [to_np(t) for t in synth.make_decode_step(sub, 0)]
+        self.cap = sub.units * (sub.n + sub.max_new_tokens)
+        self.tokens = int(self.sl.sum())
+        self.threads = min(self.cores, sub.units)
 
-        def one_pass():
-            psi = oracle.score(code, q, k, sl).astype(np.float32)
-            al = oracle.allocate(psi, mask, sl, bud, wl.theta)
-            rc, kept_len, seg_off, kept_idx = oracle.select(psi, mask, sl, al["budgets"], headroom=sub.max_new_tokens,
-                                                            capacity=cap)
-            k_c, v_c = oracle.compact(code, k, v, kept_idx, seg_off, kept_len, cap)
-            oracle.decode(code, dq, kn, vn, k_c, v_c, seg_off, kept_len, Hkv=sub.Hkv)
+    def one_pass(self):
+        o, np, sub = self.oracle, self.np, self.sub
+        code = 0 if sub.dtype == "f32" else 1
+        psi = o.score(code, self.q, self.k, self.sl).astype(np.float32)
+        al = o.allocate(psi, self.mask, self.sl, self.bud, self.wl.theta)
+        rc, kept_len, seg_off, kept_idx = o.select(psi, self.mask, self.sl, al["budgets"],
+                                                   headroom=sub.max_new_tokens, capacity=self.cap)
+        k_c, v_c = o.compact(code, self.k, self.v, kept_idx, seg_off, kept_len, self.cap)
+        o.decode(code, self.dq, self.kn, self.vn, k_c, v_c, seg_off, kept_len, Hkv=sub.Hkv)
 
-        return sub, one_pass, int(sl.sum())
+    def timed(self, passes):
+        ts = []
+        for _ in range(passes):
+            t0 = time.perf_counter()
+            self.one_pass()
+            ts.append(time.perf_counter() - t0)
+        return ts
 
-    sub, one_pass, tokens = prepare(1)
-    t0 = time.perf_counter()
-    one_pass()
-    t1 = time.perf_counter() - t0
-    layers = int(max(1, min(wl.L, seconds_target / 2 / max(t1, 1e-3))))
-    if layers > 1:
-        sub, one_pass, tokens = prepare(layers)
-    reps = int(max(1, min(16, seconds_target / max(t1 * layers, 1e-3))))
-    t0 = time.perf_counter()
-    for _ in range(reps):
-        one_pass()
-    dt = (time.perf_counter() - t0) / reps
-    value = tokens * (layers / wl.L) / dt  # tokens/s of the full-depth pass at the sampled layers' rate
-    return {
-        "value": value, "unit": UNIT, "cores": oracle.hardware_threads(), "kind": "oracle",
-        "sample": f"{layers} of {wl.L} layers of workload '{wl.name}' (all {sub.Hkv} KV heads, all {wl.n} tokens, "
-                  f"one decode step), {reps} repetition(s), {dt:.2f} s each; value scaled by layers/{wl.L}",
-    }, dt
+    def value(self, dt):
+        """tokens/s of the full-depth pass at the sampled layers' rate"""
+        return self.tokens * (self.layers / self.wl.L) / dt
+
+    def info(self, dt, passes):
+        wl = self.wl
+        return {
+            "value": self.value(dt), "unit": UNIT, "cores": self.threads, "kind": "oracle",
+            "sample": f"{self.layers} of {wl.L} layers of workload '{wl.name}' (all {wl.Hkv} KV heads, all {wl.n} tokens "
+                      f"of every sequence, one decode step), {passes} pass(es), {dt:.2f} s each on {self.threads} of "
+                      f"{self.cores} host threads (one thread per unit); value scaled by layers/{wl.L}",
+        }
+
+
+def cpu_oracle_leg(wl, seconds_target=15.0):
+    s = OracleSample(wl, seconds_per_pass=seconds_target / 2)
+    passes = 2
+    ts = s.timed(passes)
+    dt = sum(ts) / len(ts)
+    return s.info(dt, passes), dt
 
 
 def workload_config(wl):
@@ -208,21 +271,23 @@ def workload_config(wl):
 
 
 def run_reference(args, wl):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    """The reference arm: there is no reference implementation (the reference is a paper), so this arm times the
+    CPU oracle, as it stands, on the host cores: each step is one pass over a bounded sample of the workload."""
+    if int(os.environ.get("RANK", "0")) != 0:
         return
-    times = []
-    info = None
-    for i in range(args.warmup + args.steps):
-        info, dt = cpu_oracle_leg(wl, seconds_target=4.0)
-        if i >= args.warmup:
-            times.append(dt)
-    ms = 1e3 * sum(times) / len(times)
+    n_pass = args.warmup + args.steps
+    per_pass = max(1.0, min(6.0, 150.0 / max(n_pass, 1)))  # the whole run stays within a few minutes
+    s = OracleSample(wl, seconds_per_pass=per_pass)
+    s.timed(args.warmup)
+    ts = s.timed(args.steps)
+    dt = sum(ts) / len(ts)
+    info = s.info(dt, args.steps)
     line = {
         "impl": "reference", "metric": METRIC, "value": info["value"], "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
-        "config": dict(workload_config(wl), note="CPU oracle on a bounded sample; each step = the sample once"),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+        "config": workload_config(wl),
+        "note": "CPU oracle on a bounded sample of the workload; each step = the sample once",
         "cpu_baseline": info,
         "e2e": {"value": info["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -230,18 +295,326 @@ def run_reference(args, wl):
     print(json.dumps(line))
 
 
+# ----------------------------------------------------------------------------------------------- the CUDA arm
+def launches_per_step(wl):
+    """Kernels of this library launched by one step: score 1 (bf16 with g * w <= 64: one tensor-core kernel) or 3
+    (bf16 with g * w <= 256: pass 1, merge, pass 2; otherwise the three fp32 kernels), allocate 2, select 2,
+    compact 1, decode 3 (append, partial, merge)."""
+    one_kernel = wl.dtype == "bf16" and wl.g * wl.w <= 64
+    return (1 if one_kernel else 3) + 2 + 2 + 1 + 3
+
+
+class Bench:
+    """One workload resident on the device: inputs, buffers, and the timed legs."""
+
+    def __init__(self, mk, wl, dev, rank, inputs=None):
+        self.mk, self.wl, self.dev = mk, wl, dev
+        wl_r = rank_workload(wl, rank)  # every rank its own batch
+        self.inp = inputs if inputs is not None else synth.make_inputs(wl_r, device=dev)
+        self.inp["budget"] = torch.full((wl.B,), wl.budget, dtype=torch.int32, device=dev)
+        self.cfg = mk.make_config(wl.torch_dtype, wl.B, wl.L, wl.Hq, wl.Hkv, wl.d, wl.n, wl.w,
+                                  max_new_tokens=wl.max_new_tokens, theta=wl.theta)
+        self.cap = wl.units * (min(wl.n, 2 * wl.budget) + wl.max_new_tokens)
+        self.buf = mk.EvictionBuffers(self.cfg, self.cap, device=dev)
+        self.n_dec = 4
+        self.dec = [synth.make_decode_step(wl_r, s, device=dev) for s in range(self.n_dec)]
+        self.tokens = int(self.inp["seq_len"].sum().item())
+        self.peak, self.peak_kind = measured_peaks()
+
+    def step(self, i, ev=None):
+        mk, c, buf, inp = self.mk, self.cfg, self.buf, self.inp
+        q, kn, vn = self.dec[i % self.n_dec]
+        if ev:
+            ev[0].record()
+        mk.madakv_score(c, inp["q_win"], inp["k"], inp["seq_len"], None, buf.psi, buf.ws)
+        if ev:
+            ev[1].record()
+        mk.madakv_allocate(c, buf.psi, inp["mask"], inp["seq_len"], inp["budget"], buf.mass, buf.pref, buf.demand,
+                           buf.phi, buf.budgets, buf.ws)
+        if ev:
+            ev[2].record()
+        mk.madakv_select(c, buf.psi, inp["mask"], inp["seq_len"], buf.budgets, buf.kept_len, buf.seg_off, buf.kept_idx,
+                         buf.ws)
+        if ev:
+            ev[3].record()
+        mk.madakv_compact(c, inp["k"], inp["v"], buf.kept_idx, buf.seg_off, buf.kept_len, buf.k_c, buf.v_c, buf.ws)
+        if ev:
+            ev[4].record()
+        mk.madakv_decode_attn(c, -1, q, kn, vn, buf.k_c, buf.v_c, buf.seg_off, buf.kept_len, buf.out, buf.lse_dec,
+                              buf.ws)
+        if ev:
+            ev[5].record()
+
+    def check_status(self, where, buf=None):
+        buf = buf or self.buf
+        site = int(buf.ws[4:8].view(torch.int32).item())  # diagnostic word beside the status (which wait gave up)
+        status = self.mk.madakv_poll_status(buf.ws)
+        if status != 0:
+            raise SystemExit(f"device status {self.mk.madakv_status_string(status)} {where} on '{self.wl.name}' "
+                             f"(wait site {site & 255}, block {site >> 8})")
+
+    def timed_steps(self, steps, warmup, sync_all, sampler_index=None):
+        for i in range(warmup):
+            self.step(i)
+        sync_all()
+        self.check_status("after warm-up")
+        sampler = ClockSampler(sampler_index) if sampler_index is not None else None
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(steps)]
+        sync_all()
+        for i in range(steps):
+            self.step(i, evs[i])
+        sync_all()
+        clocks = sampler.stop() if sampler else None
+        total_ms = evs[0][0].elapsed_time(evs[-1][5])
+        stage_ms = [sum(e[j].elapsed_time(e[j + 1]) for e in evs) / steps for j in range(5)]
+        self.check_status("after the timed region")
+        return total_ms, stage_ms, clocks
+
+    # ---- decode-step latency on a fixed cache, all layers in one call (the roofline form)
+    def time_decode(self, b, steps=20):
+        mk = self.mk
+        for i in range(3):
+            q, kn, vn = self.dec[i % self.n_dec]
+            mk.madakv_decode_attn(b.cfg, -1, q, None, None, b.k_c, b.v_c, b.seg_off, b.kept_len, b.out, None, b.ws)
+        torch.cuda.synchronize()
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(steps):
+            q, kn, vn = self.dec[i % self.n_dec]
+            mk.madakv_decode_attn(b.cfg, -1, q, None, None, b.k_c, b.v_c, b.seg_off, b.kept_len, b.out, None, b.ws)
+        z.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(z) / steps * 1e3
+
+    # ---- the decode run of the workload: max_new_tokens steps, each appending one row per KV head (Eq. 4) and
+    # attending over the grown cache (Eq. 5); per-step device times. `layerwise` issues the L dependent per-layer
+    # calls a model makes (layer l + 1's query depends on layer l's output) instead of one all-layer call.
+    def time_decode_run(self, b, layerwise=False, max_steps=None):
+        mk, wl = self.mk, self.wl
+        n_steps = wl.max_new_tokens if max_steps is None else min(max_steps, wl.max_new_tokens)
+        keep = b.kept_len.clone()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps + 1)]
+        torch.cuda.synchronize()
+        evs[0].record()
+        for s in range(n_steps):
+            q, kn, vn = self.dec[s % self.n_dec]
+            if layerwise:
+                for l in range(wl.L):
+                    mk.madakv_decode_attn(b.cfg, l, q, kn, vn, b.k_c, b.v_c, b.seg_off, b.kept_len, b.out, None, b.ws)
+            else:
+                mk.madakv_decode_attn(b.cfg, -1, q, kn, vn, b.k_c, b.v_c, b.seg_off, b.kept_len, b.out, None, b.ws)
+            evs[s + 1].record()
+        torch.cuda.synchronize()
+        grown = int((b.kept_len - keep).min().item()), int((b.kept_len - keep).max().item())
+        self.check_status("after the decode run", b)
+        b.kept_len.copy_(keep)  # the appended rows lie in the headroom: dropping them restores the cache
+        us = sorted(evs[i].elapsed_time(evs[i + 1]) * 1e3 for i in range(n_steps))
+        return {"steps": n_steps, "us_median": us[len(us) // 2], "us_min": us[0], "us_max": us[-1],
+                "us_mean": sum(us) / len(us), "rows_appended_per_segment": grown[0] if grown[0] == grown[1] else grown}
+
+    # ---- stage 1 in a single pass, for callers that bring the prefill's log-sum-exps (here: those of madakv_score)
+    def time_single_pass(self, steps=10):
+        mk, wl, buf, inp = self.mk, self.wl, self.buf, self.inp
+        lse = torch.empty((wl.B, wl.L, wl.Hq, wl.w), dtype=torch.float32, device=self.dev)
+        psi1 = torch.empty_like(buf.psi)
+        mk.madakv_score(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, buf.psi, buf.ws)
+        for _ in range(3):
+            mk.madakv_score_lse(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, psi1, buf.ws)
+        torch.cuda.synchronize()
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            mk.madakv_score_lse(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, psi1, buf.ws)
+        z.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(z) / steps
+
+    # ---- the layer-by-layer order (a layer is evicted right after its prefill): per layer single-pass scoring with
+    # the prefill's log-sum-exps, madakv_allocate_layer carrying phi, selection and compaction of that layer.
+    # Scoring and compaction (HBM streams) run on one stream; allocation and selection of a layer (a few blocks,
+    # latency-bound) run on a second stream and overlap the scoring of the next layer. The only dependencies are
+    # score(l) -> allocate(l) -> select(l) -> compact(l) and phi(l) -> allocate(l + 1), both kept by events.
+    def time_streamed(self, steps=3, two_streams=True):
+        mk, wl, buf, inp = self.mk, self.wl, self.buf, self.inp
+        cfg1 = mk.make_config(wl.torch_dtype, wl.B, 1, wl.Hq, wl.Hkv, wl.d, wl.n, wl.w,
+                              max_new_tokens=wl.max_new_tokens, theta=wl.theta)
+        slots = 2 if two_streams else 1  # per-layer scratch in flight
+        one = [mk.EvictionBuffers(cfg1, self.cap // wl.L + wl.B * wl.Hkv, device=self.dev) for _ in range(slots)]
+        lse = torch.empty((wl.B, wl.L, wl.Hq, wl.w), dtype=torch.float32, device=self.dev)
+        mk.madakv_score(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, buf.psi, buf.ws)
+        lse_l = [lse[:, l:l + 1].contiguous() for l in range(wl.L)]
+        phi = torch.zeros((wl.B, wl.L), dtype=torch.float64, device=self.dev)
+        ws2 = mk.new_workspace(buf.cfg, self.dev)  # allocate_layer's workspace on the second stream
+        main = torch.cuda.current_stream()
+        side = torch.cuda.Stream() if two_streams else main
+
+        def one_pass():
+            done_sel = [None] * slots
+            done_cmp = [None] * slots
+            for l in range(wl.L):
+                o = one[l % slots]
+                q_l, k_l, v_l = inp["q_win"][:, l:l + 1], inp["k"][:, l:l + 1], inp["v"][:, l:l + 1]
+                if two_streams and done_cmp[l % slots] is not None:
+                    pass  # same stream as the compaction that last read this slot: ordered already
+                if two_streams and done_sel[l % slots] is not None:
+                    main.wait_event(done_sel[l % slots])  # psi of this slot is free once its selection has run
+                mk.madakv_score_lse(cfg1, q_l, k_l, inp["seq_len"], lse_l[l], o.psi, o.ws)
+                scored = torch.cuda.Event()
+                scored.record(main)
+                with torch.cuda.stream(side):
+                    side.wait_event(scored)
+                    if two_streams and done_cmp[l % slots] is not None:
+                        side.wait_event(done_cmp[l % slots])  # kept_idx of this slot was read by its compaction
+                    mk.madakv_allocate_layer(buf.cfg, l, o.psi, inp["mask"], inp["seq_len"], inp["budget"], o.mass,
+                                             o.pref, o.demand, phi, o.budgets, ws2)
+                    mk.madakv_select(cfg1, o.psi, inp["mask"], inp["seq_len"], o.budgets, o.kept_len, o.seg_off,
+                                     o.kept_idx, ws2)
+                    sel = torch.cuda.Event()
+                    sel.record(side)
+                done_sel[l % slots] = sel
+                if two_streams:
+                    # compaction of the layer before runs behind this layer's scoring on the main stream
+                    if l > 0:
+                        p = one[(l - 1) % slots]
+                        main.wait_event(done_sel[(l - 1) % slots])
+                        mk.madakv_compact(cfg1, inp["k"][:, l - 1:l], inp["v"][:, l - 1:l], p.kept_idx, p.seg_off,
+                                          p.kept_len, p.k_c, p.v_c, p.ws)
+                        c = torch.cuda.Event()
+                        c.record(main)
+                        done_cmp[(l - 1) % slots] = c
+                else:
+                    mk.madakv_compact(cfg1, k_l, v_l, o.kept_idx, o.seg_off, o.kept_len, o.k_c, o.v_c, o.ws)
+            if two_streams:
+                l = wl.L - 1
+                p = one[l % slots]
+                main.wait_event(done_sel[l % slots])
+                mk.madakv_compact(cfg1, inp["k"][:, l:l + 1], inp["v"][:, l:l + 1], p.kept_idx, p.seg_off, p.kept_len,
+                                  p.k_c, p.v_c, p.ws)
+
+        for _ in range(2):
+            one_pass()
+        torch.cuda.synchronize()
+        bad = [mk.madakv_poll_status(o.ws) for o in one] + [mk.madakv_poll_status(ws2), mk.madakv_poll_status(buf.ws)]
+        if any(bad):
+            return None
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            one_pass()
+        z.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(z) / steps
+
+    def full_cache(self):
+        """The same cache without eviction (budget = context length): what decode costs uncompressed."""
+        wl = self.wl
+        full = self.mk.EvictionBuffers(self.cfg, wl.units * (wl.n + wl.max_new_tokens), device=self.dev)
+        big = torch.full_like(self.inp["budget"], wl.n)
+        full.run_eviction(self.inp["q_win"], self.inp["k"], self.inp["v"], self.inp["mask"], self.inp["seq_len"], big)
+        torch.cuda.synchronize()
+        return full
+
+    def record(self, stage_ms, clocks, args, with_streamed=True):
+        """Per-workload figures of the JSON line from the timed steps and the decode legs."""
+        wl, buf = self.wl, self.buf
+        buf.kept_len.sub_(1)  # the last step's append lies in the headroom: dropping it restores the compacted cache
+        rows = int(buf.kept_len.sum().item())  # kept rows of the pass
+        e = wl.elem_bytes
+        # bytes the method must move (algorithmic): K read once; kept K/V rows read and written; decode reads K_c + V_c
+        k_bytes = wl.units * wl.n * wl.d * e
+        compact_bytes = 4 * rows * wl.d * e
+        decode_bytes = 2 * (rows + wl.units) * wl.d * e  # the step's decode reads the appended row too
+        peak = self.peak
+        score_gbs = k_bytes / (stage_ms[0] * 1e-3) / 1e9
+        pass_ms = sum(stage_ms[:4])
+        pass_gbs = (k_bytes + compact_bytes) / (pass_ms * 1e-3) / 1e9
+        dec_gbs = decode_bytes / (stage_ms[4] * 1e-3) / 1e9
+        # The dominant kernel is the score stage. With up to 64 window rows per KV head it is bound by reading K
+        # once (HBM). With more (the grouped-query workloads) every key meets g * w exponentials in each of the two
+        # passes and the special-function unit binds first: a measured 15.99 exp2 per clock and SM, at the median
+        # SM clock sampled during the timed region.
+        if wl.g * wl.w <= 64:
+            roofline = {"bound": "hbm", "kernel": "score_cluster_kernel (stage 1)", "achieved": score_gbs, "peak": peak,
+                        "unit": "GB/s", "frac": score_gbs / peak,
+                        "traffic": ncu_traffic("score_cluster_kernel", wl.name),
+                        "peak_kind": self.peak_kind, "algorithmic_bytes": k_bytes}
+        else:
+            props = torch.cuda.get_device_properties(self.dev)
+            sm_mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
+            exp_peak = props.multi_processor_count * EXP2_PER_CLK_PER_SM * sm_mhz * 1e6 / 1e12
+            n_exp = 2.0 * wl.g * wl.w * float(self.tokens) * wl.L * wl.Hkv  # two passes over every logit
+            achieved = n_exp / (stage_ms[0] * 1e-3) / 1e12
+            roofline = {"bound": "alu", "kernel": "score_rows_kernel pass 1 + pass 2 (stage 1)", "achieved": achieved,
+                        "peak": exp_peak, "unit": "Texp2/s", "frac": achieved / exp_peak,
+                        "traffic": ncu_traffic("score_rows_kernel", wl.name),
+                        "peak_kind": f"measured: {EXP2_PER_CLK_PER_SM} exp2 per clock and SM (register-only probe) x "
+                                     f"{props.multi_processor_count} SMs x the median SM clock sampled in the timed "
+                                     f"region ({sm_mhz:.0f} MHz)",
+                        "algorithmic_exp2": n_exp,
+                        "hbm": {"achieved": score_gbs, "peak": peak, "unit": "GB/s", "frac": score_gbs / peak,
+                                "algorithmic_bytes": k_bytes, "peak_kind": self.peak_kind,
+                                "exp2_bound_allows_frac": min(1.0, (k_bytes / (peak * 1e9)) / (n_exp / (exp_peak * 1e12)))}}
+        rec = {
+            "config": workload_config(wl),
+            "stages_ms": dict(zip(["score", "allocate", "select", "compact", "decode"], stage_ms)),
+            "roofline": roofline,
+            "eviction_pass": {"ms": pass_ms, "tokens_per_s": self.tokens / (pass_ms * 1e-3),
+                              "algorithmic_bytes": k_bytes + compact_bytes, "gbs": pass_gbs,
+                              "frac_of_measured_peak": pass_gbs / peak, "frac_of_8TBs": pass_gbs / NOMINAL_HBM_GBS,
+                              "kept_rows": rows},
+            "clocks": clocks,
+        }
+        dec = {"algorithmic_bytes": decode_bytes, "gbs_in_step": dec_gbs,
+               "frac_of_measured_peak_in_step": dec_gbs / peak,
+               "compressed_rows_per_head": (rows + wl.units) / wl.units}
+        us = self.time_decode(buf)
+        dec["us_per_step"] = {"compressed": us, "full": None}
+        dec["gbs_alone"] = decode_bytes / (us * 1e-6) / 1e9
+        dec["frac_of_measured_peak_alone"] = dec["gbs_alone"] / peak
+        dec["frac_of_8TBs_alone"] = dec["gbs_alone"] / NOMINAL_HBM_GBS
+        dec["run_with_append"] = {"compressed": self.time_decode_run(buf), "full": None}
+        dec["us_per_step_layer_sequential"] = {"compressed": self.time_decode_run(buf, layerwise=True, max_steps=16),
+                                               "full": None}
+        if not args.no_full_cache:
+            full = self.full_cache()
+            dec["us_per_step"]["full"] = self.time_decode(full, steps=5)
+            dec["run_with_append"]["full"] = self.time_decode_run(full, max_steps=32)
+            dec["us_per_step_layer_sequential"]["full"] = self.time_decode_run(full, layerwise=True, max_steps=4)
+            full_bytes = 2 * int(full.kept_len.sum().item()) * wl.d * e
+            dec["full_cache_gbs"] = full_bytes / (dec["us_per_step"]["full"] * 1e-6) / 1e9
+            dec["speedup_compressed_vs_full"] = dec["us_per_step"]["full"] / us
+            del full
+        rec["decode"] = dec
+        if not args.no_single_pass:
+            single_ms = self.time_single_pass()
+            rec["single_pass_score"] = {
+                "ms": single_ms, "gbs": k_bytes / (single_ms * 1e-3) / 1e9,
+                "frac_of_measured_peak": k_bytes / (single_ms * 1e-3) / 1e9 / peak,
+                "note": "madakv_score_lse: stage 1 with the rows' log-sum-exps supplied; not part of the step"}
+            if with_streamed:
+                s2, s1 = self.time_streamed(two_streams=True), self.time_streamed(two_streams=False)
+                rec["streamed_pass"] = {
+                    "ms_two_streams": s2, "ms_one_stream": s1, "ratio_to_all_layer_pass":
+                    None if s2 is None else s2 / pass_ms, "launches": wl.L * 7,
+                    "note": "stages 1-4 layer by layer (madakv_score_lse, madakv_allocate_layer, select and compact "
+                            "with one-layer configs); two streams: allocation and selection of a layer overlap the "
+                            "scoring of the next; not part of the step"}
+        return rec
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="llava", choices=list(synth.CONFIGS))
+    ap.add_argument("--workload", default=HEADLINE, choices=list(synth.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--only", action="store_true", help="time the headline workload only (no `workloads` records)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-full-cache", action="store_true", help="skip the full-cache decode comparison")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
-    ap.add_argument("--no-single-pass", action="store_true", help="skip the timing of madakv_score_lse (profiling runs)")
+    ap.add_argument("--no-single-pass", action="store_true", help="skip madakv_score_lse and the streamed order")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: run a reduced-depth copy of the workload")
     ap.add_argument("--budget", type=int, default=0, help="budget sweeps: another per-head budget than the workload's")
     ap.add_argument("--theta", type=float, default=0.0, help="budget sweeps: the Eq. 9 threshold calibrated for --budget "
@@ -276,222 +649,97 @@ def main():
     if world > 1:
         dist.barrier()
     mk.lib()
-
-    wl_r = rank_workload(wl, rank)  # every rank its own batch
     dev = torch.device("cuda", local)
-    inp = synth.make_inputs(wl_r, device=dev)
-    cfg = mk.make_config(wl.torch_dtype, wl.B, wl.L, wl.Hq, wl.Hkv, wl.d, wl.n, wl.w, max_new_tokens=wl.max_new_tokens,
-                         theta=wl.theta)
-    cap = wl.units * (min(wl.n, 2 * wl.budget) + wl.max_new_tokens)
-    buf = mk.EvictionBuffers(cfg, cap, device=dev)
-    n_dec = 4
-    dec = [synth.make_decode_step(wl_r, s, device=dev) for s in range(n_dec)]
-    tokens = int(inp["seq_len"].sum().item())
-
-    def step(i, ev=None):
-        c = buf.cfg
-        q, kn, vn = dec[i % n_dec]
-        if ev:
-            ev[0].record()
-        mk.madakv_score(c, inp["q_win"], inp["k"], inp["seq_len"], None, buf.psi, buf.ws)
-        if ev:
-            ev[1].record()
-        mk.madakv_allocate(c, buf.psi, inp["mask"], inp["seq_len"], inp["budget"], buf.mass, buf.pref, buf.demand,
-                           buf.phi, buf.budgets, buf.ws)
-        if ev:
-            ev[2].record()
-        mk.madakv_select(c, buf.psi, inp["mask"], inp["seq_len"], buf.budgets, buf.kept_len, buf.seg_off, buf.kept_idx,
-                         buf.ws)
-        if ev:
-            ev[3].record()
-        mk.madakv_compact(c, inp["k"], inp["v"], buf.kept_idx, buf.seg_off, buf.kept_len, buf.k_c, buf.v_c, buf.ws)
-        if ev:
-            ev[4].record()
-        mk.madakv_decode_attn(c, -1, q, kn, vn, buf.k_c, buf.v_c, buf.seg_off, buf.kept_len, buf.out, buf.lse_dec,
-                              buf.ws)
-        if ev:
-            ev[5].record()
 
     def sync_all():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(args.warmup):
-        step(i)
-    sync_all()
-    site = int(buf.ws[4:8].view(torch.int32).item())  # diagnostic word beside the status (which wait gave up)
-    status = mk.madakv_poll_status(buf.ws)
-    if status != 0:
-        raise SystemExit(f"device status {mk.madakv_status_string(status)} after warm-up (wait site {site & 255}, "
-                         f"block {site >> 8})")
-
-    sampler = ClockSampler(local) if rank == 0 else None
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
-    sync_all()
-    for i in range(args.steps):
-        step(i, evs[i])
-    sync_all()
-    clocks = sampler.stop() if sampler else None
-    total_ms = evs[0][0].elapsed_time(evs[-1][5])
-    stage_ms = [sum(e[j].elapsed_time(e[j + 1]) for e in evs) / args.steps for j in range(5)]
-    total_ms, tokens_all = reduce_over_ranks(total_ms, tokens, dev, world)
+    # ---- headline workload
+    b = Bench(mk, wl, dev, rank)
+    total_ms, stage_ms, clocks = b.timed_steps(args.steps, args.warmup, sync_all, local if rank == 0 else None)
+    total_ms, tokens_all = reduce_over_ranks(total_ms, b.tokens, dev, world)
     ms_per_step = total_ms / args.steps
     value = job_throughput(total_ms, args.steps, tokens_all)
 
-    # bytes the method must move (algorithmic): K read once; kept K/V rows read and written; decode reads K_c + V_c
-    rows = int(buf.kept_len.sum().item()) - wl.units  # kept rows before this step's append
-    e = wl.elem_bytes
-    k_bytes = wl.units * wl.n * wl.d * e
-    compact_bytes = 4 * rows * wl.d * e
-    decode_bytes = 2 * (rows + wl.units) * wl.d * e
-    peak, peak_kind = measured_peaks()
-    score_gbs = k_bytes / (stage_ms[0] * 1e-3) / 1e9
-    pass_ms = sum(stage_ms[:4])
-    pass_gbs = (k_bytes + compact_bytes) / (pass_ms * 1e-3) / 1e9
-    dec_gbs = decode_bytes / (stage_ms[4] * 1e-3) / 1e9
-
-    # The dominant kernel is the score stage. With up to 64 window rows per KV head it is bound by reading K once
-    # (HBM). With more (the grouped-query workloads) every key meets g * w exponentials in each of the two passes and
-    # the special-function unit binds first: 16 exp2 per clock and SM, at the maximum SM clock.
-    if wl.g * wl.w <= 64:
-        roofline = {"bound": "hbm", "kernel": "score stage (stage 1)", "achieved": score_gbs, "peak": peak,
-                    "unit": "GB/s", "frac": score_gbs / peak, "traffic": TRAFFIC.get(wl.name),
-                    "peak_kind": peak_kind, "algorithmic_bytes": k_bytes}
-    else:
-        props = torch.cuda.get_device_properties(dev)
-        sm_ghz = (clocks or {}).get("sm_max_mhz") or 1965.0
-        exp_peak = props.multi_processor_count * 16 * sm_ghz * 1e6 / 1e12
-        n_exp = 2.0 * wl.g * wl.w * float(inp["seq_len"].sum().item()) * wl.L * wl.Hkv  # two passes over every logit
-        achieved = n_exp / (stage_ms[0] * 1e-3) / 1e12
-        roofline = {"bound": "alu", "kernel": "score stage (stage 1)", "achieved": achieved, "peak": exp_peak,
-                    "unit": "Texp2/s", "frac": achieved / exp_peak, "traffic": None,
-                    "peak_kind": "derived: SMs x 16 exp2 per clock x max SM clock", "algorithmic_exp2": n_exp,
-                    "hbm": {"achieved": score_gbs, "peak": peak, "unit": "GB/s", "frac": score_gbs / peak,
-                            "algorithmic_bytes": k_bytes}}
-
     # ---- end to end through the C ABI with host buffers (pinned): H2D of the step's inputs, D2H of its result
     h2d = d2h = 0
+    e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     if not args.no_e2e:
-        host = {k: v.cpu().pin_memory() for k, v in inp.items()}
-        hdec = [tuple(x.cpu().pin_memory() for x in d) for d in dec]
-        h_out = torch.empty_like(buf.out, device="cpu").pin_memory()
-        h_len = torch.empty_like(buf.kept_len, device="cpu").pin_memory()
+        inp, buf = b.inp, b.buf
+
+        def pinned(t):
+            h = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+            h.copy_(t)
+            return h
+
+        host = {k: pinned(v) for k, v in inp.items()}
+        hdec = [tuple(pinned(x) for x in d) for d in b.dec]
+        h_out = torch.empty(buf.out.shape, dtype=buf.out.dtype, pin_memory=True)
+        h_len = torch.empty(buf.kept_len.shape, dtype=buf.kept_len.dtype, pin_memory=True)
         h2d = sum(v.numel() * v.element_size() for v in host.values()) + sum(x.numel() * x.element_size()
                                                                              for x in hdec[0])
         d2h = h_out.numel() * h_out.element_size() + h_len.numel() * h_len.element_size()
 
-    def e2e_step(i):
-        for k_, v_ in host.items():
-            inp[k_].copy_(v_, non_blocking=True)
-        for dst, src in zip(dec[i % n_dec], hdec[i % n_dec]):
-            dst.copy_(src, non_blocking=True)
-        step(i)
-        h_out.copy_(buf.out, non_blocking=True)
-        h_len.copy_(buf.kept_len, non_blocking=True)
+        def e2e_step(i):
+            for k_, v_ in host.items():
+                inp[k_].copy_(v_, non_blocking=True)
+            for dst, src in zip(b.dec[i % b.n_dec], hdec[i % b.n_dec]):
+                dst.copy_(src, non_blocking=True)
+            b.step(i)
+            h_out.copy_(buf.out, non_blocking=True)
+            h_len.copy_(buf.kept_len, non_blocking=True)
 
-    e2e_ms = e2e_value = None
-    if not args.no_e2e:
         e2e_step(0)
         sync_all()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.e2e_steps + 1)]
+        evs[0].record()
         for i in range(args.e2e_steps):
             e2e_step(i)
-        e1.record()
+            evs[i + 1].record()
         sync_all()
-        e2e_total, _ = reduce_over_ranks(e0.elapsed_time(e1), tokens, dev, world)
-        e2e_ms = e2e_total / args.e2e_steps
-        e2e_value = job_throughput(e2e_total, args.e2e_steps, tokens_all)
-
-    # ---- decode-step latency: compressed cache (per step, all layers in one call) against the full cache
-    def time_decode(b, steps=20):
-        for i in range(3):
-            q, kn, vn = dec[i % n_dec]
-            mk.madakv_decode_attn(b.cfg, -1, q, None, None, b.k_c, b.v_c, b.seg_off, b.kept_len, b.out, None, b.ws)
-        torch.cuda.synchronize()
-        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for i in range(steps):
-            q, kn, vn = dec[i % n_dec]
-            mk.madakv_decode_attn(b.cfg, -1, q, None, None, b.k_c, b.v_c, b.seg_off, b.kept_len, b.out, None, b.ws)
-        z.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(z) / steps * 1e3
-
-    # ---- stage 1 in a single pass, for callers that bring the prefill's log-sum-exps (here: those of madakv_score)
-    def time_single_pass(steps=20):
-        lse = torch.empty((wl.B, wl.L, wl.Hq, wl.w), dtype=torch.float32, device=dev)
-        psi1 = torch.empty_like(buf.psi)
-        mk.madakv_score(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, buf.psi, buf.ws)
-        for _ in range(3):
-            mk.madakv_score_lse(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, psi1, buf.ws)
-        torch.cuda.synchronize()
-        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(steps):
-            mk.madakv_score_lse(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, psi1, buf.ws)
-        z.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(z) / steps
-
-    single_ms = None if args.no_single_pass else time_single_pass()
-
-    # ---- the layer-by-layer order (a layer is evicted right after its prefill): per layer single-pass scoring with
-    # the prefill's log-sum-exps, madakv_allocate_layer carrying phi, selection and compaction of that layer
-    def time_streamed(steps=5):
-        cfg1 = mk.make_config(wl.torch_dtype, wl.B, 1, wl.Hq, wl.Hkv, wl.d, wl.n, wl.w,
-                              max_new_tokens=wl.max_new_tokens, theta=wl.theta)
-        one = mk.EvictionBuffers(cfg1, cap // wl.L + wl.B * wl.Hkv, device=dev)
-        lse = torch.empty((wl.B, wl.L, wl.Hq, wl.w), dtype=torch.float32, device=dev)
-        mk.madakv_score(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, buf.psi, buf.ws)
-        lse_l = [lse[:, l:l + 1].contiguous() for l in range(wl.L)]
-        phi = torch.zeros((wl.B, wl.L), dtype=torch.float64, device=dev)
-
-        def one_pass():
-            for l in range(wl.L):
-                q_l, k_l, v_l = inp["q_win"][:, l:l + 1], inp["k"][:, l:l + 1], inp["v"][:, l:l + 1]
-                mk.madakv_score_lse(cfg1, q_l, k_l, inp["seq_len"], lse_l[l], one.psi, one.ws)
-                mk.madakv_allocate_layer(buf.cfg, l, one.psi, inp["mask"], inp["seq_len"], inp["budget"], one.mass,
-                                         one.pref, one.demand, phi, one.budgets, buf.ws)
-                mk.madakv_select(cfg1, one.psi, inp["mask"], inp["seq_len"], one.budgets, one.kept_len, one.seg_off,
-                                 one.kept_idx, one.ws)
-                mk.madakv_compact(cfg1, k_l, v_l, one.kept_idx, one.seg_off, one.kept_len, one.k_c, one.v_c, one.ws)
-
-        for _ in range(2):
-            one_pass()
-        torch.cuda.synchronize()
-        if mk.madakv_poll_status(one.ws) != 0 or mk.madakv_poll_status(buf.ws) != 0:
-            return None
-        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(steps):
-            one_pass()
-        z.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(z) / steps
-
-    streamed_ms = None if args.no_single_pass else time_streamed()
-
-    decode_us = {"compressed": time_decode(buf), "full": None,
-                 "compressed_rows_per_head": (rows + wl.units) / wl.units}
-    if not args.no_full_cache and rank == 0:
-        full = mk.EvictionBuffers(cfg, wl.units * (wl.n + wl.max_new_tokens), device=dev)
-        big = torch.full_like(inp["budget"], wl.n)
-        full.run_eviction(inp["q_win"], inp["k"], inp["v"], inp["mask"], inp["seq_len"], big)
-        torch.cuda.synchronize()
-        decode_us["full"] = time_decode(full, steps=5)
-        del full
-    site = int(buf.ws[4:8].view(torch.int32).item())
-    status = mk.madakv_poll_status(buf.ws)
-    if status != 0:
-        raise SystemExit(f"device status {mk.madakv_status_string(status)} after the timed region (wait site "
-                         f"{site & 255}, block {site >> 8})")
+        per = sorted(evs[i].elapsed_time(evs[i + 1]) for i in range(args.e2e_steps))
+        e2e_total, _ = reduce_over_ranks(evs[0].elapsed_time(evs[-1]), b.tokens, dev, world)
+        e2e = {"value": job_throughput(e2e_total, args.e2e_steps, tokens_all), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_total / args.e2e_steps,
+               "ms_per_step_min": per[0], "ms_per_step_median": per[len(per) // 2], "steps": args.e2e_steps}
+        del host, hdec
 
     if rank != 0:
+        # the other ranks only take part in the headline's timed region
         if world > 1:
             dist.destroy_process_group()
         return
+
+    head = b.record(stage_ms, clocks, args)
+    launches = args.steps * launches_per_step(wl)
+    del b
+    torch.cuda.empty_cache()
+
+    # ---- the other benchmark workloads, each from its own timed steps (rank 0; their decode and streamed legs too)
+    workloads = {wl.name: head}
+    if not args.only and world == 1 and args.layers == 0 and args.budget == 0:
+        shared = {}
+        for name in OTHER_WORKLOADS:
+            if name == wl.name:
+                continue
+            w2 = synth.CONFIGS[name]
+            key = (w2.seed, w2.layout, w2.B, w2.L, w2.Hq, w2.Hkv, w2.n, w2.w)  # the qwen budgets share their inputs
+            if key not in shared:
+                shared.clear()
+                torch.cuda.empty_cache()
+                shared[key] = synth.make_inputs(rank_workload(w2, rank), device=dev)
+            bb = Bench(mk, w2, dev, rank, inputs=shared[key])
+            t_ms, st_ms, clk = bb.timed_steps(max(args.steps, 20), args.warmup, sync_all, local)
+            rec = bb.record(st_ms, clk, args)
+            rec["ms_per_step"] = t_ms / max(args.steps, 20)
+            rec["steps"] = max(args.steps, 20)
+            workloads[name] = rec
+            del bb
+        shared.clear()
+        torch.cuda.empty_cache()
+
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         cpu, _ = cpu_oracle_leg(wl)
@@ -501,44 +749,21 @@ def main():
         "dtype": wl.dtype, "data": "synthetic",
         "config": workload_config(wl),
         "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_ms},
-        "gpu_launches": args.steps * launches_per_step(wl),
-        "roofline": roofline,
-        "stages_ms": dict(zip(["score", "allocate", "select", "compact", "decode"], stage_ms)),
-        "eviction_pass": {"ms": pass_ms, "tokens_per_s": tokens / (pass_ms * 1e-3), "algorithmic_bytes":
-                          k_bytes + compact_bytes, "gbs": pass_gbs, "frac_of_measured_peak": pass_gbs / peak,
-                          "frac_of_8TBs": pass_gbs / 8000.0, "kept_rows": rows},
-        "decode": {"us_per_step": decode_us, "algorithmic_bytes": decode_bytes, "gbs_in_step": dec_gbs,
-                   "frac_of_measured_peak_in_step": dec_gbs / peak,
-                   "gbs_alone": decode_bytes / (decode_us["compressed"] * 1e-6) / 1e9},
-        "single_pass_score": None if single_ms is None else {
-            "ms": single_ms, "gbs": k_bytes / (single_ms * 1e-3) / 1e9,
-            "frac_of_measured_peak": k_bytes / (single_ms * 1e-3) / 1e9 / peak,
-            "note": "madakv_score_lse: stage 1 with the rows' log-sum-exps supplied; not part of the step"},
-        "streamed_pass": None if streamed_ms is None else {
-            "ms": streamed_ms, "tokens_per_s": tokens / (streamed_ms * 1e-3), "launches": wl.L * 7,
-            "note": "stages 1-4 layer by layer (madakv_score_lse, madakv_allocate_layer, select and compact with "
-                    "one-layer configs), launch-bound at this depth; not part of the step"},
+        "e2e": e2e,
+        "gpu_launches": launches,
+        "roofline": head["roofline"],
+        "stages_ms": head["stages_ms"],
+        "eviction_pass": head["eviction_pass"],
+        "decode": head["decode"],
+        "single_pass_score": head.get("single_pass_score"),
+        "streamed_pass": head.get("streamed_pass"),
         "cpu_baseline": cpu,
+        "workloads": workloads,
     }
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
 
-
-def launches_per_step(wl):
-    """Kernels of this library launched by one step: score 1 (bf16 with g * w <= 64: one tensor-core kernel) or 3
-    (bf16 with g * w <= 256: pass 1, merge, pass 2; otherwise the three fp32 kernels), allocate 2, select 2,
-    compact 1, decode 3 (append, partial, merge)."""
-    one_kernel = wl.dtype == "bf16" and wl.g * wl.w <= 64
-    return (1 if one_kernel else 3) + 2 + 2 + 1 + 3
-
-
-# dram bytes (read + write) per launch of the dominant kernel (score_cluster), per workload, from the ncu capture
-# summarised in profiles/all_kernels_llava.md: 274.2 MB measured on the 4-layer case, times 8 for the 32 layers
-# (traffic grows with the number of units); None = not captured
-TRAFFIC = {"llava": 8 * 274.2e6}
 
 if __name__ == "__main__":
     main()

@@ -1,11 +1,13 @@
 // Stage 5: cache append (Eq. 4) and decode attention over the ragged per-head cache (Eq. 5).
 //
 //   append   copies k_new / v_new behind every segment of the layer(s) and bumps kept_len
-//   partial  one block per (segment, split of kDecodeChunk rows): a group of LPR lanes owns a cache row (16 bytes
-//            per lane), the g query heads of the KV group share every K/V row read; online softmax in the log2
-//            domain, fp32 accumulation; the block's row groups are merged in shared memory. For bf16 caches with
-//            3 <= g <= 16 the same split is computed by decode_partial_mma_kernel on the tensor cores instead.
-//   merge    one block per query head: fixed-order combination of the split partials, rounding to dtype once
+//   partial  up to kDecodeSlots blocks per segment, each taking an equal share of the segment's rows (the share is a
+//            function of the segment's length alone: short segments use fewer blocks, never fewer than kDecodeMinRows
+//            rows each): a group of LPR lanes owns a cache row (16 bytes per lane), the g query heads of the KV group
+//            share every K/V row read; online softmax in the log2 domain, fp32 accumulation; the block's row groups
+//            are merged in shared memory. For bf16 caches with 3 <= g <= 16 the same share is computed by
+//            decode_partial_mma_kernel on the tensor cores instead.
+//   merge    one block per query head: fixed-order combination of the blocks' partials, rounding to dtype once
 #include <mutex>
 
 #include "common.cuh"
@@ -14,7 +16,8 @@ namespace madakv {
 namespace {
 
 constexpr int NT = 128;
-constexpr int kDecodeGridX = 32;  // blocks per segment at most
+constexpr int kDecodeSlots = 32;    // blocks (and partials) per segment at most
+constexpr int kDecodeMinRows = 128; // a block's share of a segment is at least this many rows (a multiple of 64)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -29,9 +32,9 @@ struct DecodeParams {
   int64_t capacity;
   void* out;
   float* lse_out;
-  float* part;  // ws: [B*L*Hq, splits, D + 2]
+  float* part;  // ws: [B*L*Hq, slots, D + 2]
   void* ws;
-  int L, Hq, Hkv, g, layer, splits;
+  int L, Hq, Hkv, g, layer, slots;
   float scale2;
 };
 
@@ -48,13 +51,29 @@ __device__ __forceinline__ int unit_of(const DecodeParams& p, int y) {
   return (b * p.L + p.layer) * p.Hkv + h;
 }
 
-// Rows of unit u's segment that attention may read. A segment that does not lie inside the cache (selection reported
-// MADAKV_ECAPACITY and left it unwritten), or that is longer than the split partials provide for, counts as empty:
-// nothing beyond `capacity` rows or beyond the workspace is ever touched.
+// Rows of unit u's segment that attention may read. A segment that selection refused (it, with its headroom, ends
+// beyond the cache: MADAKV_ECAPACITY was reported and neither indices nor rows were written) counts as empty, and so
+// does one whose length does not fit its own slot: nothing beyond `capacity` rows is ever touched.
+__device__ __forceinline__ bool segment_refused(const DecodeParams& p, int u) {
+  const int64_t off = p.seg_off[u], end = p.seg_off[u + 1];
+  return off < 0 || end < off || end > p.capacity;
+}
 __device__ __forceinline__ int segment_rows(const DecodeParams& p, int u) {
   const int len = p.kept_len[u];
-  const int64_t off = p.seg_off[u];
-  return (len < 0 || off < 0 || off + (int64_t)len > p.capacity || len > p.splits * kDecodeChunk) ? 0 : len;
+  if (segment_refused(p, u) || len < 0 || p.seg_off[u] + (int64_t)len > p.seg_off[u + 1]) return 0;
+  return len;
+}
+// The blocks of a segment of `len` rows: how many take part, and the rows of block x (a multiple of 64 each, so
+// that the 16-row chunks of the warps never straddle two blocks). Block 0 always takes part: an empty segment still
+// gets a well-defined partial.
+__device__ __forceinline__ int segment_blocks(const DecodeParams& p, int len) {
+  return max(1, min(p.slots, (len + kDecodeMinRows - 1) / kDecodeMinRows));
+}
+__device__ __forceinline__ void block_rows(const DecodeParams& p, int len, int x, int& row_begin, int& row_end) {
+  const int nb = segment_blocks(p, len);
+  const int share = ((len + nb - 1) / nb + 63) / 64 * 64;
+  row_begin = min(len, x * share);
+  row_end = min(len, row_begin + share);
 }
 
 template <int ROW_BYTES>
@@ -66,7 +85,7 @@ __global__ void append_kernel(DecodeParams p, int n_sel) {
   const int u = unit_of(p, y);
   const int len = p.kept_len[u];
   const int64_t row = p.seg_off[u] + len;
-  if (row + 1 > p.seg_off[u + 1] || row + 1 > p.capacity) {
+  if (segment_refused(p, u) || len < 0 || row + 1 > p.seg_off[u + 1]) {
     if (lane == 0) set_status(p.ws, MADAKV_ECAPACITY);
     return;
   }
@@ -114,10 +133,12 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
   __shared__ float s_o[GROUPS][G][D];
   __shared__ float s_m[GROUPS][G], s_l[GROUPS][G];
 
-  const int u = unit_of(p, blockIdx.y);
+  const int u = unit_of(p, blockIdx.x);
   const int len = segment_rows(p, u);
-  // split 0 always reports, so an empty segment is well defined; a block beyond the segment has nothing to do
-  if (blockIdx.x != 0 && (int)blockIdx.x * kDecodeChunk >= len) return;
+  const int slot = blockIdx.y;
+  if (slot >= segment_blocks(p, len)) return;
+  int row_begin, row_end;
+  block_rows(p, len, slot, row_begin, row_end);
   const int64_t off = p.seg_off[u];
   const int h = u % p.Hkv, bl = u / p.Hkv;
   const int lane = threadIdx.x % LPR, grp = threadIdx.x / LPR;
@@ -133,11 +154,6 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
       for (int c = 0; c < EPL; ++c) qr[i][c] = 0.f;
     }
   }
-  // the grid has at most kDecodeGridX blocks per segment: a block takes splits blockIdx.x, blockIdx.x + gridDim.x, ...
-  // (segments of an evicted cache are a few splits long, those of a full cache hundreds)
-  for (int split = blockIdx.x; split == 0 || split * kDecodeChunk < len; split += gridDim.x) {
-  const int row_begin = split * kDecodeChunk;
-  const int row_end = min(len, row_begin + kDecodeChunk);
   float m[G], l[G], o[G][EPL];
 #pragma unroll
   for (int i = 0; i < G; ++i) {
@@ -225,14 +241,12 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
       Lsum += s_l[gq][i] * f;
       O += s_o[gq][i][c] * f;
     }
-    float* dst = p.part + (((int64_t)bl * p.Hq + h * p.g + i) * p.splits + split) * (D + 2);
+    float* dst = p.part + (((int64_t)bl * p.Hq + h * p.g + i) * p.slots + slot) * (D + 2);
     dst[c] = O;
     if (c == 0) {
       dst[D] = M;
       dst[D + 1] = Lsum;
     }
-  }
-  __syncthreads();  // the shared arrays are reused by the next split
   }
 }
 
@@ -300,9 +314,12 @@ __global__ void __launch_bounds__(kMmaWarps * 32, 3) decode_partial_mma_kernel(D
   constexpr int NB = D / 8;            // 8-column blocks of the output
   extern __shared__ __align__(16) unsigned char dsmem[];
 
-  const int u = unit_of(p, blockIdx.y);
+  const int u = unit_of(p, blockIdx.x);
   const int len = segment_rows(p, u);
-  if (blockIdx.x != 0 && (int)blockIdx.x * kDecodeChunk >= len) return;
+  const int slot = blockIdx.y;
+  if (slot >= segment_blocks(p, len)) return;
+  int row_begin, row_end;
+  block_rows(p, len, slot, row_begin, row_end);
   const int64_t off = p.seg_off[u];
   const int h = u % p.Hkv, bl = u / p.Hkv;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
@@ -330,9 +347,7 @@ __global__ void __launch_bounds__(kMmaWarps * 32, 3) decode_partial_mma_kernel(D
   const uint32_t k_lane = ((mi >> 1) * 8 + mr) * MT::PITCH + (mi & 1) * 16;  // keys (mi/2)*8.., d half mi%2
   const uint32_t v_lane = ((mi & 1) * 8 + mr) * MT::PITCH + (mi >> 1) * 16;  // keys (mi%2)*8.., column block mi/2
 
-  for (int split = blockIdx.x; split == 0 || split * kDecodeChunk < len; split += gridDim.x) {
-    const int row_begin = split * kDecodeChunk;
-    const int row_end = min(len, row_begin + kDecodeChunk);
+  {
     float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
     float o[NB][4];
 #pragma unroll
@@ -450,14 +465,13 @@ __global__ void __launch_bounds__(kMmaWarps * 32, 3) decode_partial_mma_kernel(D
         Lsum += wo[16 * MT::OPITCH + 16 + i] * fw;
         O += wo[i * MT::OPITCH + c] * fw;
       }
-      float* dst = p.part + (((int64_t)bl * p.Hq + h * p.g + i) * p.splits + split) * (D + 2);
+      float* dst = p.part + (((int64_t)bl * p.Hq + h * p.g + i) * p.slots + slot) * (D + 2);
       dst[c] = O;
       if (c == 0) {
         dst[D] = M;
         dst[D + 1] = Lsum;
       }
     }
-    __syncthreads();  // the staging areas become K/V buffers again
   }
 }
 
@@ -474,8 +488,8 @@ __global__ void __launch_bounds__(D) decode_merge_kernel(DecodeParams p) {
   const int bl = row / p.Hq, hq = row % p.Hq;
   const int u = bl * p.Hkv + hq / p.g;
   const int len = segment_rows(p, u);
-  const int used = max(1, (len + kDecodeChunk - 1) / kDecodeChunk);
-  const float* part = p.part + (int64_t)row * p.splits * (D + 2);
+  const int used = segment_blocks(p, len);
+  const float* part = p.part + (int64_t)row * p.slots * (D + 2);
   const int c = threadIdx.x;
   float M = -INFINITY;
   for (int s = 0; s < used; ++s) M = fmaxf(M, part[s * (D + 2) + D]);
@@ -497,27 +511,27 @@ __global__ void __launch_bounds__(D) decode_merge_kernel(DecodeParams p) {
 template <typename T, int D>
 int run(const DecodeParams& p, const madakv_config& c, cudaStream_t st) {
   const int n_sel = (p.layer < 0 ? c.batch * c.n_layers : c.batch) * c.n_kv_heads;
+  // every host-side refusal comes before the first launch (the append below changes the cache)
+  const bool mma = sizeof(T) == 2 && p.g >= 3 && p.g <= 16;
+  if (!mma && p.g > 8) return MADAKV_EUNSUPPORTED;
+  if constexpr (sizeof(T) == 2) {
+    if (mma && cudaFuncSetAttribute(decode_partial_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    MmaTile<D>::BYTES) != cudaSuccess)
+      return MADAKV_ECUDA;
+  }
   if (p.k_new) {
     constexpr int LPR = D * (int)sizeof(T) / 16;
     append_kernel<D * (int)sizeof(T)><<<(n_sel * LPR + 127) / 128, 128, 0, st>>>(p, n_sel);
   }
-  if (n_sel > 65535) return MADAKV_EUNSUPPORTED;
-  const dim3 grid(p.splits < kDecodeGridX ? p.splits : kDecodeGridX, n_sel);
-  bool mma = false;
+  const dim3 grid(n_sel, p.slots);  // segments on x (no 65535 limit), a segment's blocks on y
   if constexpr (sizeof(T) == 2) {
-    if (p.g >= 3 && p.g <= 16) {
-      mma = true;
-      cudaFuncSetAttribute(decode_partial_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           MmaTile<D>::BYTES);
-      decode_partial_mma_kernel<D><<<grid, kMmaWarps * 32, MmaTile<D>::BYTES, st>>>(p);
-    }
+    if (mma) decode_partial_mma_kernel<D><<<grid, kMmaWarps * 32, MmaTile<D>::BYTES, st>>>(p);
   }
   if (mma) {
   } else if (p.g == 1) decode_partial_kernel<T, D, 1><<<grid, NT, 0, st>>>(p);
   else if (p.g == 2) decode_partial_kernel<T, D, 2><<<grid, NT, 0, st>>>(p);
   else if (p.g <= 4) decode_partial_kernel<T, D, 4><<<grid, NT, 0, st>>>(p);
-  else if (p.g <= 8) decode_partial_kernel<T, D, 8><<<grid, NT, 0, st>>>(p);
-  else return MADAKV_EUNSUPPORTED;
+  else decode_partial_kernel<T, D, 8><<<grid, NT, 0, st>>>(p);
   decode_merge_kernel<T, D><<<n_sel * p.g, D, 0, st>>>(p);
   return launch_status();
 }
@@ -546,7 +560,7 @@ int launch_decode(const madakv_config& c, int layer, const void* q, const void* 
   p.Hkv = c.n_kv_heads;
   p.g = c.n_q_heads / c.n_kv_heads;
   p.layer = layer;
-  p.splits = wl.decode_splits;
+  p.slots = wl.decode_splits < kDecodeSlots ? wl.decode_splits : kDecodeSlots;
   p.scale2 = scale_of(c) * kLog2e;
   if (c.dtype == MADAKV_F32) return c.head_dim == 64 ? run<float, 64>(p, c, st) : run<float, 128>(p, c, st);
   return c.head_dim == 64 ? run<__nv_bfloat16, 64>(p, c, st) : run<__nv_bfloat16, 128>(p, c, st);
@@ -627,7 +641,7 @@ extern "C" int madakv_decode_attn_static(const madakv_config* cfg, int32_t layer
   p.Hkv = c.n_kv_heads;
   p.g = c.n_q_heads / c.n_kv_heads;
   p.layer = layer;
-  p.splits = splits;
+  p.slots = splits < kDecodeSlots ? splits : kDecodeSlots;  // what the kernels use of the (larger) documented bound
   p.scale2 = scale_of(c) * kLog2e;
   cudaStream_t st = (cudaStream_t)stream;
   if (c.dtype == MADAKV_F32) return c.head_dim == 64 ? run<float, 64>(p, c, st) : run<float, 128>(p, c, st);

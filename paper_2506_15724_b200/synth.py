@@ -114,6 +114,9 @@ CONFIGS = {
     # second dense shape of the paper's model list (LLaVA-1.5-13B: 40 layers x 40 heads), same prompt recipe as llava
     "llava13b": Workload("llava13b", "bf16", 1, 40, 40, 40, 128, 8192, 32, 1638, 0.472339, 20250620, "llava", 16, 16),
     "qwen": Workload("qwen", "bf16", 1, 28, 28, 4, 128, 32768, 32, 2048, 0.324026, 20250617, "blocks70", 16, 16),
+    # the other two points of the Qwen-shaped budget sweep {1024, 2048, 4096}: same prompt and K/V (same seed)
+    "qwen1024": Workload("qwen1024", "bf16", 1, 28, 28, 4, 128, 32768, 32, 1024, 0.284623, 20250617, "blocks70", 16, 16),
+    "qwen4096": Workload("qwen4096", "bf16", 1, 28, 28, 4, 128, 32768, 32, 4096, 0.395515, 20250617, "blocks70", 16, 16),
     "batched": Workload("batched", "bf16", 8, 28, 28, 4, 128, 16384, 32, 2048, 0.415580, 20250618, "blocks_rand", 16, 128),
     "long": Workload("long", "bf16", 1, 32, 32, 8, 128, 131072, 64, 4096, 0.218545, 20250619, "long", 16, 256),
 }
