@@ -62,9 +62,9 @@ inline WsLayout ws_layout(const madakv_config& c) {
   if (rows <= 64) {
     const size_t tc = units * rows_pad * (size_t)w.score_tc_chunks * 4 * sizeof(float2);
     part = tc > part ? tc : part;
-  } else if (rows <= 256) {  // wide-window path: two column halves per 2048-key split and padded row
+  } else if (rows <= 256) {  // wide-window path: per 2048-key split and padded row one pair for each column share
     const size_t splits = ((size_t)c.max_seq_len + 2047) / 2048;
-    const size_t wide = units * splits * 2 * rows_pad * sizeof(float2);
+    const size_t wide = units * splits * (rows <= 128 ? 4 : 2) * rows_pad * sizeof(float2);
     part = wide > part ? wide : part;
   }
   off = align_up(off + part, 256);

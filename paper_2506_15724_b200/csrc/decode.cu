@@ -17,7 +17,8 @@ namespace {
 
 constexpr int NT = 128;
 constexpr int kDecodeSlots = 32;    // blocks (and partials) per segment at most
-constexpr int kDecodeMinRows = 128; // a block's share of a segment is at least this many rows (a multiple of 64)
+constexpr int kDecodeMinRows = 512; // a block's share of a segment is at least this many rows: shorter shares leave
+                                    // the block's load pipeline no time to fill (measured: 256 rows cost 5-8 %)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -34,7 +35,7 @@ struct DecodeParams {
   float* lse_out;
   float* part;  // ws: [B*L*Hq, slots, D + 2]
   void* ws;
-  int L, Hq, Hkv, g, layer, slots;
+  int L, Hq, Hkv, g, layer, slots, n_sel, min_rows, slot_fast;
   float scale2;
 };
 
@@ -63,15 +64,15 @@ __device__ __forceinline__ int segment_rows(const DecodeParams& p, int u) {
   if (segment_refused(p, u) || len < 0 || p.seg_off[u] + (int64_t)len > p.seg_off[u + 1]) return 0;
   return len;
 }
-// The blocks of a segment of `len` rows: how many take part, and the rows of block x (a multiple of 64 each, so
+// The blocks of a segment of `len` rows: how many take part, and the rows of block x (a multiple of 16 each, so
 // that the 16-row chunks of the warps never straddle two blocks). Block 0 always takes part: an empty segment still
 // gets a well-defined partial.
 __device__ __forceinline__ int segment_blocks(const DecodeParams& p, int len) {
-  return max(1, min(p.slots, (len + kDecodeMinRows - 1) / kDecodeMinRows));
+  return max(1, min(p.slots, (len + p.min_rows - 1) / p.min_rows));
 }
 __device__ __forceinline__ void block_rows(const DecodeParams& p, int len, int x, int& row_begin, int& row_end) {
   const int nb = segment_blocks(p, len);
-  const int share = ((len + nb - 1) / nb + 63) / 64 * 64;
+  const int share = ((len + nb - 1) / nb + 15) / 16 * 16;
   row_begin = min(len, x * share);
   row_end = min(len, row_begin + share);
 }
@@ -133,9 +134,9 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
   __shared__ float s_o[GROUPS][G][D];
   __shared__ float s_m[GROUPS][G], s_l[GROUPS][G];
 
-  const int u = unit_of(p, blockIdx.x);
+  const int u = unit_of(p, p.slot_fast ? blockIdx.x / p.slots : blockIdx.x % p.n_sel);
   const int len = segment_rows(p, u);
-  const int slot = blockIdx.y;
+  const int slot = p.slot_fast ? blockIdx.x % p.slots : blockIdx.x / p.n_sel;
   if (slot >= segment_blocks(p, len)) return;
   int row_begin, row_end;
   block_rows(p, len, slot, row_begin, row_end);
@@ -314,9 +315,9 @@ __global__ void __launch_bounds__(kMmaWarps * 32, 3) decode_partial_mma_kernel(D
   constexpr int NB = D / 8;            // 8-column blocks of the output
   extern __shared__ __align__(16) unsigned char dsmem[];
 
-  const int u = unit_of(p, blockIdx.x);
+  const int u = unit_of(p, p.slot_fast ? blockIdx.x / p.slots : blockIdx.x % p.n_sel);
   const int len = segment_rows(p, u);
-  const int slot = blockIdx.y;
+  const int slot = p.slot_fast ? blockIdx.x % p.slots : blockIdx.x / p.n_sel;
   if (slot >= segment_blocks(p, len)) return;
   int row_begin, row_end;
   block_rows(p, len, slot, row_begin, row_end);
@@ -508,9 +509,20 @@ __global__ void __launch_bounds__(D) decode_merge_kernel(DecodeParams p) {
   if (p.lse_out && c == 0) p.lse_out[row] = Lsum > 0.f ? (M + log2f(Lsum)) * kLn2 : -INFINITY;
 }
 
+// Block order of the grid. With many segments a segment's blocks follow one another (neighbouring blocks stream
+// neighbouring rows); with fewer segments than SMs the grid is a wave or two, and then the blocks are ordered by slot so
+// that every segment's last and shortest block is scheduled last.
+int slot_order(int n_sel) {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return 1;
+  return n_sel >= sms ? 1 : 0;
+}
+
 template <typename T, int D>
-int run(const DecodeParams& p, const madakv_config& c, cudaStream_t st) {
-  const int n_sel = (p.layer < 0 ? c.batch * c.n_layers : c.batch) * c.n_kv_heads;
+int run(const DecodeParams& p, const madakv_config&, cudaStream_t st) {
+  const int n_sel = p.n_sel;
   // every host-side refusal comes before the first launch (the append below changes the cache)
   const bool mma = sizeof(T) == 2 && p.g >= 3 && p.g <= 16;
   if (!mma && p.g > 8) return MADAKV_EUNSUPPORTED;
@@ -523,7 +535,7 @@ int run(const DecodeParams& p, const madakv_config& c, cudaStream_t st) {
     constexpr int LPR = D * (int)sizeof(T) / 16;
     append_kernel<D * (int)sizeof(T)><<<(n_sel * LPR + 127) / 128, 128, 0, st>>>(p, n_sel);
   }
-  const dim3 grid(n_sel, p.slots);  // segments on x (no 65535 limit), a segment's blocks on y
+  const dim3 grid((unsigned)n_sel * p.slots);  // one dimension: no 65535 limit on the number of segments
   if constexpr (sizeof(T) == 2) {
     if (mma) decode_partial_mma_kernel<D><<<grid, kMmaWarps * 32, MmaTile<D>::BYTES, st>>>(p);
   }
@@ -561,6 +573,9 @@ int launch_decode(const madakv_config& c, int layer, const void* q, const void* 
   p.g = c.n_q_heads / c.n_kv_heads;
   p.layer = layer;
   p.slots = wl.decode_splits < kDecodeSlots ? wl.decode_splits : kDecodeSlots;
+  p.n_sel = (layer < 0 ? c.batch * c.n_layers : c.batch) * c.n_kv_heads;
+  p.min_rows = kDecodeMinRows;
+  p.slot_fast = slot_order(p.n_sel);
   p.scale2 = scale_of(c) * kLog2e;
   if (c.dtype == MADAKV_F32) return c.head_dim == 64 ? run<float, 64>(p, c, st) : run<float, 128>(p, c, st);
   return c.head_dim == 64 ? run<__nv_bfloat16, 64>(p, c, st) : run<__nv_bfloat16, 128>(p, c, st);
@@ -642,6 +657,9 @@ extern "C" int madakv_decode_attn_static(const madakv_config* cfg, int32_t layer
   p.g = c.n_q_heads / c.n_kv_heads;
   p.layer = layer;
   p.slots = splits < kDecodeSlots ? splits : kDecodeSlots;  // what the kernels use of the (larger) documented bound
+  p.n_sel = (layer < 0 ? c.batch * c.n_layers : c.batch) * c.n_kv_heads;
+  p.min_rows = kDecodeMinRows;
+  p.slot_fast = slot_order(p.n_sel);
   p.scale2 = scale_of(c) * kLog2e;
   cudaStream_t st = (cudaStream_t)stream;
   if (c.dtype == MADAKV_F32) return c.head_dim == 64 ? run<float, 64>(p, c, st) : run<float, 128>(p, c, st);

@@ -1,24 +1,31 @@
 // Stage 1, tensor-core path for wide windows (Eq. 7 with the softmax of Eq. 5): bf16 inputs with 64 < g * w <= 256
-// window rows per KV head (grouped-query attention with many query heads per KV head).
+// window rows per KV head (grouped-query attention with many query heads per KV head), and the single-pass form of
+// stage 1 (log-sum-exps supplied by the caller) for every bf16 shape with g * w <= 256.
 //
 // With that many rows the work per key byte is dominated by the exponentials (g * w of them per key and pass), not
-// by HBM, and a per-key owner of all rows (as in the narrow-window kernels) would need hundreds of registers. So the
-// tile is turned round: the window rows sit on M (one or two blocks of 128 rows), the 128 keys of a tile on N, and a
-// thread of the epilogue owns ONE window row (a TMEM lane) and sees its logits for the keys of a tile as columns.
-//   pass 1  per (unit, key split): running maximum and sum of exp2 of every row over the split's keys, in-thread
-//           (per 16 columns: block maximum, one rescale, 16 exponentials); one (max, sum) pair per row and split
-//   merge   per (unit, row): the pairs of all splits -> the row's log-sum-exp (a separate small kernel)
-//   pass 2  per (unit, key split): logits recomputed with the tile turned back (128 keys on M, the window rows on N,
-//           as in the narrow-window kernels): a thread owns one key and psi(i) = sum over rows of exp2(s - lse) is an
-//           in-thread sum over the columns of its TMEM lane; the rows' negated log-sum-exps come as broadcast loads
-// K is streamed twice (the second time mostly from HBM): for these shapes the exponentials take longer than either
-// read. The passes are separate launches, so no CTA ever waits for another CTA. Warp roles: warp 0 TMA producer,
-// warp 1 MMA issuer and TMEM owner, warps 2-17 epilogue. Two warps share each (TMEM lane quarter, row block) of
-// pass 1 and each (lane quarter, accumulator buffer) of pass 2 and take one half of a tile's columns each: the
-// exponentials are latency-bound with two warps per scheduler, four keep the special-function unit busy. In pass 1
-// the halves publish separate (max, sum) pairs; in pass 2 the upper half hands its partial psi to the lower half
-// through shared memory. TMEM lane quarter = warp % 4 throughout.
-// Every wait is bounded: on expiry the kernel records MADAKV_ETIMEOUT, drains and returns.
+// by HBM: the special-function unit delivers 16 exp2 per clock and SM, which for 256 rows is 2048 clocks per 128-key
+// tile against ~1400 clocks for reading the tile from HBM. The kernels are therefore built around keeping that unit
+// busy.
+//   pass 1  window rows on M (one or two blocks of 128 rows), the 128 keys of a tile on N: an epilogue thread owns
+//           ONE window row (a TMEM lane) and a share of the tile's columns and keeps a running (max, sum of exp2) of
+//           its row in registers, carried from tile to tile and from work item to work item for as long as the CTA
+//           stays with the same unit; one (max, sum) pair per row, column share and run goes to the workspace
+//   merge   per (unit, row): all pairs -> the row's log-sum-exp (a separate small kernel)
+//   pass 2  the tile turned back (128 keys on M, the window rows on N): a thread owns one key and a quarter of the
+//           window rows, and psi(i) = sum over rows of exp2(s - lse) is an in-thread sum over columns of its TMEM lane.
+//           The shift by the row's log-sum-exp is part of the contraction: one more 16-deep step multiplies a
+//           constant column of ones on the key side with -lse / scale (as three bf16 terms) on the row side, so the
+//           accumulator arrives shifted and the epilogue reads no per-row operand (with the log-sum-exps as
+//           shared-memory broadcasts the loads competed with the tensor core's operand reads and cost a fifth of
+//           the pass). The four warps that share a key add their partial sums up through shared memory in a
+//           fixed order.
+// In both passes all 16 epilogue warps work on the same tile while the MMAs of the next tile fill the other half of
+// the TMEM; the TMEM load of a warp's next 16 columns is in flight while it works on the present ones.
+// K is streamed twice. The passes are separate launches and no CTA ever waits for another CTA. Work items are
+// (unit, 2048 keys); a CTA takes a contiguous range of the non-empty items (equal counts, so ragged batches stay
+// balanced), which makes consecutive items share their unit: queries and log-sum-exps are reloaded only when the
+// unit changes. Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-17 epilogue; TMEM lane
+// quarter = warp % 4 throughout. Every wait is bounded: on expiry the kernel records MADAKV_ETIMEOUT, drains and returns.
 #include "tc_common.cuh"
 
 namespace madakv {
@@ -26,67 +33,113 @@ namespace {
 
 constexpr int kRowThreads = 576;  // 2 + 16 warps
 constexpr int kSplitKeys = 2048;  // keys per work item (16 tiles)
+constexpr int kMaxSeqScan = 1024; // batches up to this size get the exact (ragged-aware) item partition
 
 struct RowParams {
   const int32_t* seq_len;
   float* psi;        // [units, n_max]
-  float2* part;      // ws: [units, splits, 2, rs] (max, sum) of every row over each half of a split's tiles
+  float2* part;      // ws: [units, splits, cparts, rs] (max, sum) of every row over a column share of a run of items
   const float* lse2; // ws: [units, rs] NEGATED log2-domain log-sum-exp, padding rows hold kEmptyMax (pass 2)
   int32_t* status;   // ws header
-  int units, L, Hq, Hkv, g, w, R, n_max, causal, splits, rs, mblocks, n16;  // n16: R rounded up to 16
+  int B, units, L, Hq, Hkv, g, w, R, n_max, causal, splits, rs, mblocks, cparts, n16;  // n16: R rounded up to 16
   float scale2;
 };
 
-template <int D>
+template <int D, int PASS>
 struct RowSmem {
-  static constexpr int kStages = D == 128 ? 3 : 6;
+  // pass 2 gives up one K stage for the operands of its extra contraction step (see the MMA issuer)
+  static constexpr int kStages = (D == 128 ? 4 : 8) - (PASS == 2 ? (D == 128 ? 1 : 2) : 0);
   static constexpr int kKBlocks = D / 64;
   static constexpr int kStageBytes = kTileKeys * D * 2;
   static constexpr int kQBytes = 256 * D * 2;  // up to two blocks of 128 rows
   static constexpr int kKOff = 0;
   static constexpr int kQOff = kStages * kStageBytes;
-  static constexpr int kBarOff = kQOff + kQBytes;
-  // full[kStages], empty[kStages], qfull, qempty, tfull[2], tempty[2], drain, xbar[8]
-  static constexpr int kNumBars = 2 * kStages + 7 + 8;
-  static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-  static constexpr int kColOff = kMiscOff + 16;            // window position (row % w) of every row [256]
-  static constexpr int kXchOff = kColOff + 256 * 4;        // pass 2: partial psi of the upper column halves [2][128]
-  static constexpr int kTotal = kXchOff + 2 * 128 * 4;
+  static constexpr int kOnesOff = kQOff + kQBytes;                          // pass 2: [128 keys][64] bf16, 1 in columns 0-2
+  static constexpr int kShiftOff = kOnesOff + (PASS == 2 ? 128 * 128 : 0);  // pass 2: [256 rows][64] bf16, columns 0-2
+  static constexpr int kBarOff = kShiftOff + (PASS == 2 ? 256 * 128 : 0);
+  // full[kStages], empty[kStages], qfull, qempty, tfull[2], tempty[2], drain, xfull[8], xempty[8]
+  static constexpr int kNumBars = 2 * kStages + 2 + 4 + 1 + 16;
+  static constexpr int kMiscOff = (kBarOff + kNumBars * 8 + 15) / 16 * 16;
+  static constexpr int kColOff = kMiscOff + 32;            // window position (row % w) of every row [256]
+  static constexpr int kXchOff = kColOff + 256 * 4;        // pass 2: partial psi of column shares 1-3 [2][3][128]
+  static constexpr int kTotal = kXchOff + 6 * 128 * 4;
   static constexpr int kAlloc = kTotal + 1024;
+  static_assert(kQOff % 1024 == 0 && kOnesOff % 1024 == 0 && kShiftOff % 1024 == 0 && kBarOff % 8 == 0, "alignment");
+  static_assert(kAlloc <= 227 * 1024, "shared memory");
 };
 
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 128.
 constexpr uint32_t kIdescRows = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
+// exp2 of 8 packed pairs, summed
+__device__ __forceinline__ uint64_t exp2_sum16(const uint64_t (&x)[8]) {
+  uint64_t e[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float lo, hi;
+    unpack2(x[i], lo, hi);
+    e[i] = pack2(ex2(lo), ex2(hi));
+  }
+  return add2(add2(add2(e[0], e[1]), add2(e[2], e[3])), add2(add2(e[4], e[5]), add2(e[6], e[7])));
+}
+
+// The CTA's share of the work: a contiguous range of the non-empty work items in (sequence, layer, KV head, split)
+// order. cursor = (sequence b, index r among the items of b); a sequence of n keys has L * Hkv * ceil(n / 2048) items.
+struct ItemCursor {
+  int b, r, per_b, s_b, left;  // per_b: items of sequence b; s_b: splits of sequence b; left: items still to do
+};
+
+__device__ __forceinline__ int splits_of(const RowParams& p, int b) {
+  return (clamped_len(p.seq_len, b, p.n_max) + kSplitKeys - 1) / kSplitKeys;
+}
+__device__ __forceinline__ void cursor_settle(const RowParams& p, ItemCursor& c, bool exact) {
+  // move on to the next sequence that has items
+  while (c.left > 0 && c.r >= c.per_b) {
+    c.r -= c.per_b;
+    ++c.b;
+    if (c.b >= p.B) {
+      c.left = 0;
+      break;
+    }
+    c.s_b = exact ? splits_of(p, c.b) : p.splits;
+    c.per_b = p.L * p.Hkv * c.s_b;
+  }
+}
+__device__ __forceinline__ void cursor_item(const RowParams& p, const ItemCursor& c, int& u, int& split) {
+  const int ub = c.r / c.s_b;
+  split = c.r - ub * c.s_b;
+  u = c.b * p.L * p.Hkv + ub;
+}
 
 template <int D, int PASS>
-__global__ void __launch_bounds__(kRowThreads, 1)
+__global__ void __launch_bounds__(kRowThreads, 1)  // 96 registers: warps are allocated four at a time (18 -> 20)
 score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_q, RowParams p) {
-  using SL = RowSmem<D>;
+  using SL = RowSmem<D, PASS>;
   constexpr int kStages = SL::kStages;
   constexpr int kKBlocks = SL::kKBlocks;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* k_s = smem + SL::kKOff;
   uint8_t* q_s = smem + SL::kQOff;
+  uint8_t* ones_s = smem + SL::kOnesOff;
+  uint8_t* shift_s = smem + SL::kShiftOff;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kBarOff);
   uint64_t* full = bars;               // [kStages] TMA -> MMA
   uint64_t* empty = bars + kStages;    // [kStages] MMA -> TMA
-  uint64_t* qfull = empty + kStages;   // [1]       TMA -> MMA (queries of the item's unit)
+  uint64_t* qfull = empty + kStages;   // [1]       TMA -> MMA (queries of the unit; in pass 2 also its shift rows)
   uint64_t* qempty = qfull + 1;        // [1]       MMA -> TMA
   uint64_t* tfull = qempty + 1;        // [2]       MMA -> epilogue
   uint64_t* tempty = tfull + 2;        // [2]       epilogue -> MMA
   uint64_t* drain = tempty + 2;        // [1]
-  uint64_t* xbar = drain + 1;          // [8]       pass 2: upper half -> lower half of a (buffer, lane quarter) warp pair
+  uint64_t* xfull = drain + 1;         // [2][4]    pass 2: column shares 1-3 -> share 0, per buffer and lane quarter
+  uint64_t* xempty = xfull + 8;        // [2][4]    pass 2: share 0 -> shares 1-3
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(smem + SL::kMiscOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::kMiscOff + 4);
+  int* range_s = reinterpret_cast<int*>(smem + SL::kMiscOff + 8);  // first sequence, index in it, item count, exact
   int* rowpos = reinterpret_cast<int*>(smem + SL::kColOff);
   float* xch = reinterpret_cast<float*>(smem + SL::kXchOff);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // epilogue threads in use. Pass 1: two per window row (column halves); pass 2: all 16 warps, 8 per accumulator buffer
-  const int n_epi = PASS == 1 ? 256 * p.mblocks : 512;
-  const int total_items = p.units * p.splits;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -97,17 +150,54 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     mbar_init(qempty, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&tfull[i], 1);
-      mbar_init(&tempty[i], PASS == 1 ? (uint32_t)n_epi : 256u);
+      mbar_init(&tempty[i], 512);  // every epilogue thread
     }
     mbar_init(drain, 1);
-    for (int i = 0; i < 8; ++i) mbar_init(&xbar[i], 32);
+    for (int i = 0; i < 8; ++i) {
+      mbar_init(&xfull[i], 96);
+      mbar_init(&xempty[i], 32);
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // this CTA's range of work items
+    const bool exact = p.B <= kMaxSeqScan;
+    long long total = 0;
+    if (exact) {
+      for (int b = 0; b < p.B; ++b) total += (long long)p.L * p.Hkv * splits_of(p, b);
+    } else {
+      total = (long long)p.units * p.splits;
+    }
+    const long long lo = total * blockIdx.x / gridDim.x, hi = total * (blockIdx.x + 1) / gridDim.x;
+    int b0 = 0;
+    long long r0 = lo;
+    if (exact) {
+      while (b0 < p.B) {
+        const long long per = (long long)p.L * p.Hkv * splits_of(p, b0);
+        if (r0 < per) break;
+        r0 -= per;
+        ++b0;
+      }
+    } else {
+      const long long per = (long long)p.L * p.Hkv * p.splits;
+      b0 = (int)(lo / per);
+      r0 = lo - (long long)b0 * per;
+    }
+    range_s[0] = b0;
+    range_s[1] = (int)r0;
+    range_s[2] = (int)(hi - lo);
+    range_s[3] = exact ? 1 : 0;
   }
-  // rows R..255 of the Q buffer are never written by TMA: keep them zero so their logits are 0
-  for (int x = threadIdx.x; x < SL::kQBytes / 16; x += kRowThreads)
+  // rows R..255 of the Q buffer are never written by TMA: keep them zero so their logits are 0. Pass 2: the operands
+  // of the extra contraction step start out as zeros, the key side gets its three ones per row (128-byte rows with
+  // the 128-byte swizzle: the 16-byte piece that holds columns 0-7 of row r sits at position r % 8).
+  for (int x = threadIdx.x; x < (SL::kBarOff - SL::kQOff) / 16; x += kRowThreads)
     reinterpret_cast<uint4*>(q_s)[x] = make_uint4(0, 0, 0, 0);
   for (int x = threadIdx.x; x < 256; x += kRowThreads) rowpos[x] = x % p.w;
+  __syncthreads();
+  if (PASS == 2 && threadIdx.x < kTileKeys) {
+    const int r = threadIdx.x;
+    *reinterpret_cast<uint4*>(ones_s + r * 128 + (r & 7) * 16) = make_uint4(0x3f803f80u, 0x00003f80u, 0u, 0u);
+  }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_s)),
@@ -119,15 +209,29 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_base_s;
+  const bool exact = range_s[3] != 0;
 
-  // item -> (unit, first key, number of tiles); an item beyond its sequence has no tiles
-  auto item_of = [&](int item, int& u, int& key_begin, int& tiles) {
-    u = item / p.splits;
-    const int split = item % p.splits;
+  auto cursor_begin = [&]() {
+    ItemCursor c;
+    c.b = range_s[0];
+    c.r = range_s[1];
+    c.left = c.b < p.B ? range_s[2] : 0;
+    c.s_b = c.left > 0 ? (exact ? splits_of(p, c.b) : p.splits) : 1;
+    c.per_b = p.L * p.Hkv * c.s_b;
+    cursor_settle(p, c, exact);
+    return c;
+  };
+  auto cursor_next = [&](ItemCursor& c) {
+    ++c.r;
+    --c.left;
+    cursor_settle(p, c, exact);
+  };
+  // keys and tiles of an item
+  auto item_tiles = [&](int u, int split, int& key_begin, int& n) {
     const int b = u / (p.Hkv * p.L);
-    const int n = clamped_len(p.seq_len, b, p.n_max);
+    n = clamped_len(p.seq_len, b, p.n_max);
     key_begin = split * kSplitKeys;
-    tiles = key_begin < n ? (min(n, key_begin + kSplitKeys) - key_begin + kTileKeys - 1) / kTileKeys : 0;
+    return key_begin < n ? (min(n, key_begin + kSplitKeys) - key_begin + kTileKeys - 1) / kTileKeys : 0;
   };
 
   if (warp == 0) {
@@ -135,21 +239,41 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     if (lane == 0) {
       const uint64_t pol_k = l2_policy_evict_first();
       const uint64_t pol_q = l2_policy_evict_last();
-      int stage = 0;
+      int stage = 0, cur_u = -1;
       uint32_t stage_par = 0, q_par = 0;
       bool ok = true;
-      for (int it = blockIdx.x; ok && it < total_items; it += gridDim.x) {
-        const int item = PASS == 1 ? it : total_items - 1 - it;  // pass 2 backwards: pass 1's last K is still in L2
-        int u, key_begin, tiles;
-        item_of(item, u, key_begin, tiles);
+      for (ItemCursor c = cursor_begin(); ok && c.left > 0; cursor_next(c)) {
+        int u, split, key_begin, n;
+        cursor_item(p, c, u, split);
+        const int tiles = item_tiles(u, split, key_begin, n);
         if (tiles == 0) continue;
         const int h = u % p.Hkv, l = (u / p.Hkv) % p.L, b = u / (p.Hkv * p.L);
-        ok = mbar_wait(qempty, q_par ^ 1, abort_flag, p.status, kSiteQEmpty);
-        if (!ok) break;
-        q_par ^= 1;
-        mbar_expect_tx(qfull, (uint32_t)(p.R * 128 * kKBlocks));
-        for (int kb = 0; kb < kKBlocks; ++kb)
-          tma_load_5d(q_s + kb * 256 * 128, &tmap_q, qfull, kb * 64, 0, h * p.g, l, b, pol_q);
+        if (u != cur_u) {  // the unit changes: its queries (and, in pass 2, its shift rows)
+          cur_u = u;
+          ok = mbar_wait(qempty, q_par ^ 1, abort_flag, p.status, kSiteQEmpty);
+          if (!ok) break;
+          q_par ^= 1;
+          if (PASS == 2) {
+            // Row r of the shift operand: -lse_r / scale as the sum of three bf16 numbers (24 bits) in columns 0-2.
+            // Multiplied by the key side's ones in the extra contraction step, the accumulator holds q.k - lse / scale
+            // and the epilogue needs no per-row operand at all.
+            const float inv = 1.0f / p.scale2;
+            const float* src = p.lse2 + (int64_t)u * p.rs;
+            for (int r = 0; r < p.n16; ++r) {
+              const float v = src[r] * inv;
+              const float hi = __bfloat162float(__float2bfloat16_rn(v));
+              const float mid = __bfloat162float(__float2bfloat16_rn(v - hi));
+              const float low = __bfloat162float(__float2bfloat16_rn((v - hi) - mid));
+              const uint32_t w0 = (__float_as_uint(hi) >> 16) | (__float_as_uint(mid) & 0xffff0000u);
+              *reinterpret_cast<uint4*>(shift_s + r * 128 + (r & 7) * 16) =
+                  make_uint4(w0, __float_as_uint(low) >> 16, 0u, 0u);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          }
+          mbar_expect_tx(qfull, (uint32_t)(p.R * 128 * kKBlocks));
+          for (int kb = 0; kb < kKBlocks; ++kb)
+            tma_load_5d(q_s + kb * 256 * 128, &tmap_q, qfull, kb * 64, 0, h * p.g, l, b, pol_q);
+        }
         for (int t = 0; t < tiles; ++t) {
           ok = mbar_wait(&empty[stage], stage_par ^ 1, abort_flag, p.status, kSiteStage);
           if (!ok) break;
@@ -169,28 +293,34 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
       }
     }
   } else if (warp == 1) {
-    // ================================================================ MMA issuer: D[row, key] = Q_block . K_tile^T
+    // ================================================================ MMA issuer
     if (lane == 0) {
       const uint32_t k_lo0 = smem_desc_lo(smem_u32(k_s)), q_lo0 = smem_desc_lo(smem_u32(q_s));
-      int stage = 0, n_tile = 0;
+      const uint32_t ones_lo = smem_desc_lo(smem_u32(ones_s)), shift_lo = smem_desc_lo(smem_u32(shift_s));
+      const uint32_t idesc2 = instr_desc_bf16(p.n16);
+      int stage = 0, n_tile = 0, cur_u = -1;
       uint32_t stage_par = 0, q_par = 0;
       bool ok = true;
-      for (int it = blockIdx.x; ok && it < total_items; it += gridDim.x) {
-        const int item = PASS == 1 ? it : total_items - 1 - it;  // pass 2 backwards: pass 1's last K is still in L2
-        int u, key_begin, tiles;
-        item_of(item, u, key_begin, tiles);
+      for (ItemCursor c = cursor_begin(); ok && c.left > 0; cursor_next(c)) {
+        int u, split, key_begin, n;
+        cursor_item(p, c, u, split);
+        const int tiles = item_tiles(u, split, key_begin, n);
         if (tiles == 0) continue;
-        ok = mbar_wait(qfull, q_par, abort_flag, p.status, kSiteQFull);
-        if (!ok) break;
-        q_par ^= 1;
+        if (u != cur_u) {
+          if (cur_u >= 0) umma_commit(qempty);  // the queries may be replaced once the MMAs issued so far are done
+          cur_u = u;
+          ok = mbar_wait(qfull, q_par, abort_flag, p.status, kSiteQFull);
+          if (!ok) break;
+          q_par ^= 1;
+        }
         for (int t = 0; t < tiles; ++t, ++n_tile) {
           const int buf = n_tile & 1;
           const uint32_t use_par = (uint32_t)(n_tile >> 1) & 1u;
+          const uint32_t k_lo = k_lo0 + (uint32_t)stage * (SL::kStageBytes >> 4);
           ok = mbar_wait(&tempty[buf], use_par ^ 1, abort_flag, p.status, kSiteTEmpty) &&
                mbar_wait(&full[stage], stage_par, abort_flag, p.status, kSiteFull);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t k_lo = k_lo0 + (uint32_t)stage * (SL::kStageBytes >> 4);
           if (PASS == 1) {  // D[row, key]: a row block of the queries is operand A, the K tile operand B
             for (int mb = 0; mb < p.mblocks; ++mb) {
               const uint32_t d_tmem = tmem_base + buf * 256 + mb * 128;
@@ -201,15 +331,14 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
                           k_lo + ((kb * kTileKeys * 128 + kk * 32) >> 4), kIdescRows, ks > 0 ? 1u : 0u);
               }
             }
-          } else {  // D[key, row]: the K tile is operand A, all n16 query rows operand B
-            const uint32_t d_tmem = tmem_base + buf * 256;
-            const uint32_t idesc = instr_desc_bf16(p.n16);
+          } else {  // D[key, row]: the K tile is operand A, all n16 query rows operand B; then the shift step
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
               const int kb = ks >> 2, kk = ks & 3;
-              umma_bf16(d_tmem, k_lo + ((kb * kTileKeys * 128 + kk * 32) >> 4),
-                        q_lo0 + ((kb * 256 * 128 + kk * 32) >> 4), idesc, ks > 0 ? 1u : 0u);
+              umma_bf16(tmem_base + buf * 256, k_lo + ((kb * kTileKeys * 128 + kk * 32) >> 4),
+                        q_lo0 + ((kb * 256 * 128 + kk * 32) >> 4), idesc2, ks > 0 ? 1u : 0u);
             }
+            umma_bf16(tmem_base + buf * 256, ones_lo, shift_lo, idesc2, 1u);
           }
           umma_commit(&empty[stage]);  // the K stage may be refilled
           umma_commit(&tfull[buf]);    // the accumulators are ready
@@ -218,8 +347,6 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
             stage_par ^= 1;
           }
         }
-        if (!ok) break;
-        umma_commit(qempty);  // the queries may be replaced once this item's MMAs are done
       }
       if (!ok) {  // abandoned: TMEM may only be freed once this thread's MMAs have completed
         umma_commit(drain);
@@ -227,170 +354,168 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         while (!mbar_try(drain, 0) && clock64() - t0 < 20000000ll) __nanosleep(200);
       }
     }
-  } else if (PASS == 2 || (((warp - 2) >> 2) & 1) < p.mblocks) {
-    // ================================================================ epilogue: a thread owns one window row (pass 1)
-    // or one key of every other tile (pass 2), in both cases for one half of the tile's columns
+  } else {
+    // ================================================================ epilogue (warps 2-17)
+    // All 16 warps work on the same tile while the MMAs of the next tile fill the other accumulator buffer;
+    // warp = (TMEM lane quarter, column share); the TMEM load of a warp's next 16 columns is in flight while it works.
     const int ew = warp - 2;
-    const int mb = (ew >> 2) & 1;                  // row block (pass 1) or accumulator buffer (pass 2)
-    const int half = ew >> 3;                      // column half
-    const int quarter = warp & 3;                  // TMEM lanes [32 * quarter, 32 * quarter + 32)
-    const int row = mb * 128 + quarter * 32 + lane;
-    const int eidx = ew * 32 + lane;               // index among the epilogue threads in use
-    const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16) + mb * 128;
-    const float masked = kEmptyMax;                // raw value given to a logit the row may not see
-    int n_tile = 0;
-    uint32_t x_par = 0;  // pass 2: phase of the pair's exchange barrier
+    const int quarter = warp & 3;  // TMEM lanes [32 * quarter, 32 * quarter + 32)
+    // pass 1: (row block mb, column share): two row blocks x 2 shares of 64 keys, or one row block x 4 shares of 32
+    // pass 2: column share = a quarter of the n16 / 16 blocks of window rows (as even as possible)
+    const int mb = PASS == 1 && p.mblocks == 2 ? (ew >> 2) & 1 : 0;
+    const int share = PASS == 1 ? (p.mblocks == 2 ? ew >> 3 : ew >> 2) : ew >> 2;
+    int blk0, nblk;  // this warp's 16-column blocks of a tile's accumulator: blk0 .. blk0 + nblk - 1
+    if (PASS == 1) {
+      nblk = 8 / p.cparts;
+      blk0 = nblk * share;
+    } else {
+      const int total = p.n16 >> 4, base = total >> 2, rem = total & 3;
+      nblk = base + (share < rem ? 1 : 0);
+      blk0 = share * base + min(share, rem);
+    }
+    const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16) + (PASS == 1 ? mb * 128 : 0) + blk0 * 16;
+    const uint64_t sc2 = pack2(p.scale2, p.scale2);
+    int n_tile = 0, cur_u = -1;
     bool ok = true;
-    for (int it = blockIdx.x; ok && it < total_items; it += gridDim.x) {
-      const int item = PASS == 1 ? it : total_items - 1 - it;
-      int u, key_begin, tiles;
-      item_of(item, u, key_begin, tiles);
-      const int split = item % p.splits;
-      const int b = u / (p.Hkv * p.L);
-      const int n = clamped_len(p.seq_len, b, p.n_max);
+    // pass 1 state: running maximum and sums of the thread's window row, log2 domain; m starts below any masked
+    // logit. The sum is kept on two levels (the item at hand, the run's earlier items): one accumulator over a whole
+    // long sequence would lose the small terms to rounding.
+    const int row = mb * 128 + quarter * 32 + lane;
+    float m = 4.f * kEmptyMax, z = 0.f, z_run = 0.f;
+    float* xslot = xch + quarter * 32 + lane;  // pass 2: [buffer][share - 1][128 keys]
+
+    for (ItemCursor c = cursor_begin(); ok && c.left > 0; cursor_next(c)) {
+      int u, split, key_begin, n;
+      cursor_item(p, c, u, split);
+      const int tiles = item_tiles(u, split, key_begin, n);
       float* psi = p.psi + (int64_t)u * p.n_max;
-      // keys the row may see: [0, vis)
-      int vis = 0;
-      if (row < p.R) {
+      if (PASS == 1 && u != cur_u) {
+        cur_u = u;
+        m = 4.f * kEmptyMax;
+        z_run = 0.f;
+      }
+      z = 0.f;
+      int vis = 0;  // pass 1: keys the row may see: [0, vis)
+      if (PASS == 1 && row < p.R) {
         const int pos = n - p.w + row % p.w;
         if (pos >= 0) vis = p.causal ? pos + 1 : n;
       }
-      if (PASS == 1) {
-        float m = 4.f * kEmptyMax, z = 0.f;  // scaled (log2) domain; below any masked logit
-        for (int t = 0; t < tiles; ++t, ++n_tile) {
-          const int buf = n_tile & 1;
-          ok = __all_sync(0xffffffffu, mbar_wait(&tfull[buf], (uint32_t)(n_tile >> 1) & 1u, abort_flag, p.status, kSiteTile));
-          if (!ok) break;
-          tc_fence_after();
-          const int key0 = key_begin + t * kTileKeys;
-          const uint32_t taddr = tlane + buf * 256;
-          uint32_t ra[16], rb[16];
-          auto block = [&](uint32_t (&r)[16], int c) {  // columns 16c .. 16c + 15 of the tile
-            if (key0 + 16 * c + 16 > vis) {
+      for (int t = 0; t < tiles; ++t, ++n_tile) {
+        const int buf = n_tile & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(&tfull[buf], (uint32_t)(n_tile >> 1) & 1u, abort_flag, p.status, kSiteTile));
+        if (!ok) break;
+        tc_fence_after();
+        const int key0 = key_begin + t * kTileKeys;
+        const uint32_t taddr = tlane + buf * 256;
+        uint32_t ra[16], rb[16];
+        uint64_t acc = 0ull;  // pass 2: the key's sum over this warp's window rows
+        const int key = key0 + quarter * 32 + lane;                // pass 2: the thread's key
+        const bool plain = key0 + kTileKeys <= n - p.w;            // pass 2: every row sees the whole tile
+        auto block = [&](uint32_t (&r)[16], int j) {  // block blk0 + j of the accumulator
+          if (PASS == 1) {
+            const int col0 = key0 + 16 * (blk0 + j);  // first key of the block
+            if (col0 + 16 > vis) {
 #pragma unroll
               for (int i = 0; i < 16; ++i)
-                if (key0 + 16 * c + i >= vis) r[i] = __float_as_uint(masked);
+                if (col0 + i >= vis) r[i] = __float_as_uint(kEmptyMax);
             }
-            float t8[8];  // maximum and sums as trees: short dependency chains (two epilogue warps per scheduler)
-#pragma unroll
-            for (int i = 0; i < 8; ++i) t8[i] = fmaxf(__uint_as_float(r[i]), __uint_as_float(r[i + 8]));
-            const float bm = fmaxf(fmaxf(fmaxf(t8[0], t8[4]), fmaxf(t8[1], t8[5])),
-                                   fmaxf(fmaxf(t8[2], t8[6]), fmaxf(t8[3], t8[7])));
-            const float mn = fmaxf(m, bm * p.scale2);
-            z *= ex2(m - mn);
-            m = mn;
-            const uint64_t nm2 = pack2(-mn, -mn), sc2 = pack2(p.scale2, p.scale2);
-            uint64_t e[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              float lo, hi;
-              unpack2(fma2(pack2u(r[2 * i], r[2 * i + 1]), sc2, nm2), lo, hi);
-              e[i] = pack2(ex2(lo), ex2(hi));
+            const float a0 = max3f(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
+            const float a1 = max3f(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
+            const float a2 = max3f(__uint_as_float(r[6]), __uint_as_float(r[7]), __uint_as_float(r[8]));
+            const float a3 = max3f(__uint_as_float(r[9]), __uint_as_float(r[10]), __uint_as_float(r[11]));
+            const float a4 = max3f(__uint_as_float(r[12]), __uint_as_float(r[13]), __uint_as_float(r[14]));
+            const float bm = max3f(max3f(a0, a1, a2), a3, fmaxf(a4, __uint_as_float(r[15]))) * p.scale2;
+            // the running maximum rarely grows once a few hundred keys have been seen; the rescaling (one more
+            // exponential) is predicated on it
+            if (bm > m) {
+              const float f = ex2(m - bm);
+              z *= f;
+              z_run *= f;
+              m = bm;
             }
+            const uint64_t nm2 = pack2(-m, -m);
+            uint64_t x[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[i] = fma2(pack2u(r[2 * i], r[2 * i + 1]), sc2, nm2);
             float lo, hi;
-            unpack2(add2(add2(add2(e[0], e[1]), add2(e[2], e[3])), add2(add2(e[4], e[5]), add2(e[6], e[7]))), lo, hi);
+            unpack2(exp2_sum16(x), lo, hi);
             z += lo + hi;
-          };
-          const int c0 = 4 * half;  // this warp's 64 columns
-          tmem_ld16_issue(taddr + c0 * 16, ra);
-#pragma unroll 1
-          for (int c = c0; c < c0 + 4; c += 2) {
-            tmem_ld_wait16(ra);
-            tmem_ld16_issue(taddr + (c + 1) * 16, rb);
-            block(ra, c);
-            tmem_ld_wait16(rb);
-            if (c + 2 < c0 + 4) tmem_ld16_issue(taddr + (c + 2) * 16, ra);
-            block(rb, c + 1);
-          }
-          tc_fence_before();
-          mbar_arrive(&tempty[buf]);
-        }
-        if (!ok) break;
-        if (row < p.R) {
-          // a row that saw no visible key only summed masked entries: it is recorded as empty
-          const bool none = m < 0.5f * kEmptyMax * p.scale2;
-          p.part[(((int64_t)u * p.splits + split) * 2 + half) * p.rs + row] =
-              none ? make_float2(kEmptyMax, 0.f) : make_float2(m, z);
-        }
-      } else {
-        // group (warp - 2) / 4 owns accumulator buffer `group` and with it every other tile; this thread's key is
-        // key0 + 32 * quarter + lane and its logits against the n16 window rows are the columns of its TMEM lane
-        const int group = mb;
-        const int pair = group * 4 + quarter;  // the two warps (column halves) that share a key
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + group * 256;
-        const ulonglong2* ns = reinterpret_cast<const ulonglong2*>(p.lse2 + (int64_t)u * p.rs);
-        const uint64_t sc2 = pack2(p.scale2, p.scale2);
-        const int nblk = p.n16 >> 4, nlow = (nblk + 1) >> 1;
-        const int cb = half ? nlow : 0, ce = half ? nblk : nlow;  // this warp's blocks of 16 window rows
-        for (int t = 0; t < tiles; ++t, ++n_tile) {
-          if ((n_tile & 1) != group) continue;
-          ok = __all_sync(0xffffffffu, mbar_wait(&tfull[group], (uint32_t)(n_tile >> 1) & 1u, abort_flag, p.status, kSiteTile));
-          if (!ok) break;
-          tc_fence_after();
-          const int key0 = key_begin + t * kTileKeys;
-          const int key = key0 + quarter * 32 + lane;
-          // a tile below the window's first position is seen in full by every row; otherwise every logit is checked
-          const bool plain = key0 + kTileKeys <= n - p.w;
-          uint64_t acc = 0ull;
-          uint32_t ra[16], rb[16];
-          auto block = [&](uint32_t (&r)[16], int c) {  // window rows 16c .. 16c + 15
-            uint64_t sh[8];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const ulonglong2 v = __ldg(ns + 4 * c + j);
-              sh[2 * j] = v.x;
-              sh[2 * j + 1] = v.y;
-            }
-            if (!plain) {
+          } else {
+            if (!plain) {  // the tiles at the window: every logit is checked against what its row may see
 #pragma unroll
               for (int i = 0; i < 16; ++i) {
-                const int pos = n - p.w + rowpos[16 * c + i];
-                const int vis = pos < 0 ? 0 : (p.causal ? pos + 1 : n);
-                if (key >= vis) r[i] = __float_as_uint(kEmptyMax);
+                const int pos = n - p.w + rowpos[16 * (blk0 + j) + i];
+                const int v = pos < 0 ? 0 : (p.causal ? pos + 1 : n);
+                if (key >= v) r[i] = __float_as_uint(kEmptyMax);
               }
             }
-            uint64_t e[8];
+            uint64_t x[8];  // the accumulator already holds q.k - lse / scale
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              float lo, hi;
-              unpack2(fma2(pack2u(r[2 * i], r[2 * i + 1]), sc2, sh[i]), lo, hi);
-              e[i] = pack2(ex2(lo), ex2(hi));
-            }
-            acc = add2(acc, add2(add2(add2(e[0], e[1]), add2(e[2], e[3])), add2(add2(e[4], e[5]), add2(e[6], e[7]))));
-          };
-          if (cb < ce) tmem_ld16_issue(taddr + cb * 16, ra);
+            for (int i = 0; i < 8; ++i) x[i] = mul2(pack2u(r[2 * i], r[2 * i + 1]), sc2);
+            acc = add2(acc, exp2_sum16(x));
+          }
+        };
+        if (nblk > 0) {
+          tmem_ld16_issue(taddr, ra);
 #pragma unroll 1
-          for (int c = cb; c < ce; c += 2) {
+          for (int j = 0; j < nblk; j += 2) {
             tmem_ld_wait16(ra);
-            if (c + 1 < ce) tmem_ld16_issue(taddr + (c + 1) * 16, rb);
-            block(ra, c);
-            if (c + 1 < ce) {
+            if (j + 1 < nblk) tmem_ld16_issue(taddr + (j + 1) * 16, rb);
+            block(ra, j);
+            if (j + 1 < nblk) {
               tmem_ld_wait16(rb);
-              if (c + 2 < ce) tmem_ld16_issue(taddr + (c + 2) * 16, ra);
-              block(rb, c + 1);
+              if (j + 2 < nblk) tmem_ld16_issue(taddr + (j + 2) * 16, ra);
+              block(rb, j + 1);
             }
           }
+        }
+        tc_fence_before();
+        mbar_arrive(&tempty[buf]);
+        if (PASS == 2) {
+          // the four warps that share the key add up in a fixed order: shares 1-3 hand their sums to share 0 (a
+          // slot is free once share 0 has taken the tile before last)
           float lo, hi;
           unpack2(acc, lo, hi);
-          if (half) {  // hand the partial sum to the warp of the lower half
-            xch[group * 128 + quarter * 32 + lane] = lo + hi;
-            mbar_arrive(&xbar[pair]);
-          } else {
-            ok = __all_sync(0xffffffffu, mbar_wait(&xbar[pair], x_par, abort_flag, p.status, kSiteFlag));
-            x_par ^= 1;
+          float total = lo + hi;
+          const uint32_t xp = (uint32_t)(n_tile >> 1) & 1u;
+          if (share) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&xempty[buf * 4 + quarter], xp ^ 1, abort_flag, p.status, kSiteFlag));
             if (!ok) break;
-            const float tot = (lo + hi) + xch[group * 128 + quarter * 32 + lane];
-            if (key < p.n_max) psi[key] = key < n ? tot : 0.f;
+            xslot[(buf * 3 + share - 1) * 128] = total;
+            mbar_arrive(&xfull[buf * 4 + quarter]);
+          } else {
+            ok = __all_sync(0xffffffffu, mbar_wait(&xfull[buf * 4 + quarter], xp, abort_flag, p.status, kSiteFlag));
+            if (!ok) break;
+            total = ((total + xslot[(buf * 3 + 0) * 128]) + xslot[(buf * 3 + 1) * 128]) + xslot[(buf * 3 + 2) * 128];
+            mbar_arrive(&xempty[buf * 4 + quarter]);
+            if (key < p.n_max) psi[key] = key < n ? total : 0.f;
           }
-          // the buffer is handed back only after the exchange: the upper half writes its next partial sum after the
-          // next tile of this buffer has been computed, which needs every arrival of this one
-          tc_fence_before();
-          mbar_arrive(&tempty[group]);
         }
-        if (!ok) break;
-        // keys of the item beyond the sequence
-        for (int key = key_begin + tiles * kTileKeys + eidx; key < min(key_begin + kSplitKeys, p.n_max); key += n_epi)
-          psi[key] = 0.f;
+      }
+      if (!ok) break;
+      if (PASS == 1) {
+        z_run += z;
+        if (row < p.R && tiles > 0) {
+          // the pair goes out with the last item of the run (the next item is another unit's, holds no keys, or does
+          // not exist); the run's other items leave an empty pair so that the merge finds every split that holds keys
+          ItemCursor nx = c;
+          cursor_next(nx);
+          bool last = nx.left <= 0;
+          if (!last) {
+            int u2, s2, kb2, n2;
+            cursor_item(p, nx, u2, s2);
+            last = u2 != u || item_tiles(u2, s2, kb2, n2) == 0;
+          }
+          // a row that saw no visible key only summed masked entries: it is recorded as empty
+          const bool none = m < 0.5f * kEmptyMax * p.scale2;
+          p.part[(((int64_t)u * p.splits + split) * p.cparts + share) * p.rs + row] =
+              (!last || none) ? make_float2(kEmptyMax, 0.f) : make_float2(m, z_run);
+        }
+      } else {
+        // keys of the item beyond its last tile (the remainder of psi's padding is cleared by the kernel that
+        // prepares the log-sum-exps)
+        for (int k2 = key_begin + tiles * kTileKeys + ew * 32 + lane; k2 < min(key_begin + kSplitKeys, p.n_max); k2 += 512)
+          psi[k2] = 0.f;
       }
     }
   }
@@ -404,24 +529,36 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   }
 }
 
-// merge: per (unit, row) the (max, sum) pairs of all splits, in split order -> log2-domain log-sum-exp, stored
-// negated (pass 2 adds it inside a fused multiply-add); padding rows get a shift that turns every weight into 0
+// psi of the keys no work item covers: everything from the first split that lies wholly beyond the sequence
+__device__ __forceinline__ void clear_tail(const RowParams& p, int u, int row) {
+  const int b = u / (p.Hkv * p.L);
+  const int n = clamped_len(p.seq_len, b, p.n_max);
+  const int from = (n + kSplitKeys - 1) / kSplitKeys * kSplitKeys;
+  float* psi = p.psi + (int64_t)u * p.n_max;
+  for (int key = from + row; key < p.n_max; key += p.rs) psi[key] = 0.f;
+}
+
+// merge: per (unit, row) the (max, sum) pairs of all splits and column shares, in a fixed order -> log2-domain
+// log-sum-exp, stored negated (pass 2 adds it inside a fused multiply-add); padding rows get a shift that turns
+// every weight into 0
 __global__ void score_rows_merge_kernel(RowParams p, float* nlse2, float* lse_out, int total) {
   const int x = blockIdx.x * blockDim.x + threadIdx.x;
   if (x >= total) return;
   const int u = x / p.rs, row = x % p.rs;
+  clear_tail(p, u, row);
   if (row >= p.R) {
     nlse2[x] = kEmptyMax;
     return;
   }
-  const int entries = 2 * p.splits;  // column halves of every split
-  const float2* part = p.part + (int64_t)u * entries * p.rs + row;
+  const int b = u / (p.Hkv * p.L);
+  const int entries = p.cparts * splits_of(p, b);  // the splits that hold keys of this sequence
+  const float2* part = p.part + (int64_t)u * p.cparts * p.splits * p.rs + row;
   float M = kEmptyMax;
   for (int s = 0; s < entries; ++s) M = fmaxf(M, part[(int64_t)s * p.rs].x);
   float Z = 0.f;
   for (int s = 0; s < entries; ++s) {
     const float2 v = part[(int64_t)s * p.rs];
-    Z += v.y * exp2f(v.x - M);  // an empty split has sum 0
+    Z += v.y * exp2f(v.x - M);  // an empty pair has sum 0
   }
   const float l2 = Z > 0.f ? M + log2f(Z) : 0.f;
   nlse2[x] = -l2;
@@ -438,6 +575,7 @@ __global__ void score_rows_given_lse_kernel(RowParams p, const float* lse, float
   const int x = blockIdx.x * blockDim.x + threadIdx.x;
   if (x >= total) return;
   const int u = x / p.rs, row = x % p.rs;
+  clear_tail(p, u, row);
   float v = kEmptyMax;
   if (row < p.R) {
     const int h = u % p.Hkv, bl = u / p.Hkv;
@@ -448,20 +586,14 @@ __global__ void score_rows_given_lse_kernel(RowParams p, const float* lse, float
   nlse2[x] = v;
 }
 
-template <int D>
-int run_rows(const CUtensorMap& mk, const CUtensorMap& mq, RowParams p, float* lse2, float* lse_out, int grid,
-             cudaStream_t st) {
-  using SL = RowSmem<D>;
-  if (cudaFuncSetAttribute(score_rows_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kAlloc) !=
-          cudaSuccess ||
-      cudaFuncSetAttribute(score_rows_kernel<D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kAlloc) !=
-          cudaSuccess)
+template <int D, int PASS>
+int launch_pass(const CUtensorMap& mk, const CUtensorMap& mq, const RowParams& p, int grid, cudaStream_t st) {
+  using SL = RowSmem<D, PASS>;
+  if (cudaFuncSetAttribute(score_rows_kernel<D, PASS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kAlloc) !=
+      cudaSuccess)
     return MADAKV_ECUDA;
-  score_rows_kernel<D, 1><<<grid, kRowThreads, SL::kAlloc, st>>>(mk, mq, p);
-  const int total = p.units * p.rs;
-  score_rows_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(p, lse2, lse_out, total);
-  score_rows_kernel<D, 2><<<grid, kRowThreads, SL::kAlloc, st>>>(mk, mq, p);
-  return launch_status();
+  score_rows_kernel<D, PASS><<<grid, kRowThreads, SL::kAlloc, st>>>(mk, mq, p);
+  return MADAKV_OK;
 }
 
 }  // namespace
@@ -481,6 +613,7 @@ static bool rows_setup(const madakv_config& c, const void* q, madakv_strides sq,
   lse2 = reinterpret_cast<float*>((char*)ws + wl.score_lse_off);
   p.lse2 = lse2;
   p.status = reinterpret_cast<int32_t*>(ws);
+  p.B = c.batch;
   p.units = c.batch * c.n_layers * c.n_kv_heads;
   p.L = c.n_layers;
   p.Hq = c.n_q_heads;
@@ -493,6 +626,7 @@ static bool rows_setup(const madakv_config& c, const void* q, madakv_strides sq,
   p.splits = (c.max_seq_len + kSplitKeys - 1) / kSplitKeys;
   p.rs = (R + 31) / 32 * 32;  // row stride of the workspace arrays
   p.mblocks = R <= 128 ? 1 : 2;
+  p.cparts = R <= 128 ? 4 : 2;
   p.n16 = (R + 15) / 16 * 16;
   p.scale2 = scale_of(c) * kLog2e;
   int dev = 0, sms = 0;
@@ -517,9 +651,15 @@ int launch_score_rows(const madakv_config& c, const void* q, madakv_strides sq, 
   float* lse2;
   CUtensorMap mk, mq;
   int grid, rc;
-  // the workspace layout reserves (max, sum) pairs for [units, splits, 2 halves, rs]
+  // the workspace layout reserves (max, sum) pairs for [units, splits, column shares, rs]
   if (!rows_setup(c, q, sq, k, sk, seq_len, psi, ws, p, lse2, mk, mq, grid, rc)) return rc;
-  return c.head_dim == 128 ? run_rows<128>(mk, mq, p, lse2, lse, grid, st) : run_rows<64>(mk, mq, p, lse2, lse, grid, st);
+  const int total = p.units * p.rs;
+  rc = c.head_dim == 128 ? launch_pass<128, 1>(mk, mq, p, grid, st) : launch_pass<64, 1>(mk, mq, p, grid, st);
+  if (rc) return rc;
+  score_rows_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(p, lse2, lse, total);
+  rc = c.head_dim == 128 ? launch_pass<128, 2>(mk, mq, p, grid, st) : launch_pass<64, 2>(mk, mq, p, grid, st);
+  if (rc) return rc;
+  return launch_status();
 }
 
 // Single-pass scoring with the rows' log-sum-exps supplied by the caller: a conversion kernel, then pass 2 alone.
@@ -533,19 +673,8 @@ int launch_score_lse_rows(const madakv_config& c, const void* q, madakv_strides 
   if (!rows_setup(c, q, sq, k, sk, seq_len, psi, ws, p, lse2, mk, mq, grid, rc)) return rc;
   const int total = p.units * p.rs;
   score_rows_given_lse_kernel<<<(total + 255) / 256, 256, 0, st>>>(p, lse, lse2, total);
-  if (c.head_dim == 128) {
-    using SL = RowSmem<128>;
-    if (cudaFuncSetAttribute(score_rows_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kAlloc) !=
-        cudaSuccess)
-      return MADAKV_ECUDA;
-    score_rows_kernel<128, 2><<<grid, kRowThreads, SL::kAlloc, st>>>(mk, mq, p);
-  } else {
-    using SL = RowSmem<64>;
-    if (cudaFuncSetAttribute(score_rows_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kAlloc) !=
-        cudaSuccess)
-      return MADAKV_ECUDA;
-    score_rows_kernel<64, 2><<<grid, kRowThreads, SL::kAlloc, st>>>(mk, mq, p);
-  }
+  rc = c.head_dim == 128 ? launch_pass<128, 2>(mk, mq, p, grid, st) : launch_pass<64, 2>(mk, mq, p, grid, st);
+  if (rc) return rc;
   return launch_status();
 }
 

@@ -38,6 +38,16 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Non-blocking test of a barrier phase (try_wait may suspend the thread for a while; this never does).
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Records a wait that ran out: the status word, and (for diagnosis) which wait it was.
 enum { kSiteQEmpty = 1, kSiteStage = 2, kSiteQFull = 3, kSiteTEmpty = 4, kSiteFull = 5, kSiteTile = 6, kSiteFlag = 7,
        kSiteDrain = 8 };
@@ -127,6 +137,10 @@ __device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16
 __device__ __forceinline__ void tmem_ld_wait16(uint32_t (&a)[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" : MADAKV_R8(a, 0), MADAKV_R8(a, 8) : : "memory");
 }
+// Ties 16 more registers to the wait before them (no instruction): the second half of a 32-column chunk.
+__device__ __forceinline__ void tmem_ld_tie16(uint32_t (&a)[16]) {
+  asm volatile("" : MADAKV_R8(a, 0), MADAKV_R8(a, 8) : : "memory");
+}
 #undef MADAKV_R8
 __device__ __forceinline__ float warp_max(float v) {
   float r;
@@ -155,6 +169,17 @@ __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
 __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
   uint64_t r;
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+// three-input maximum (sm_100)
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
 __device__ __forceinline__ float ex2(float x) {
