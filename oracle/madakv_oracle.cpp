@@ -11,7 +11,10 @@
 //   mo_allocate  Eq. 6, 8, 9, 10, 11                pinned piecewise (subset brute force, closed-form scalars,
 //                                                   worked case); the way Eq. 8 and Eq. 10-11 are composed where
 //                                                   the paper's units disagree is a stated reading: parity unpinned
-//   mo_select    top-budget per modality            pinned (full-sort brute force, worked case)
+//   mo_select    top-budget per modality            pinned (full-sort brute force, worked case); score pooling and
+//                                                   forced retention of the window are readings of this build, not
+//                                                   of the paper (it defines neither): parity unpinned by the paper,
+//                                                   pinned against a library maximum filter and worked cases
 //   mo_compact   row gather                         pinned (definition)
 //   mo_decode    Eq. 4 + Eq. 5                      pinned (library attention, worked case)
 //
@@ -160,9 +163,13 @@ int32_t mo_topp_count_f64(const double* psi, int n, double theta) {
 // Eq. 10-11 (layer compensation). hcc_mode: 0 off, 1 divide by H*(L-l), 2 divide by (L-l) as printed, 3 as 1 with
 // every layer but the last keeping what Eq. 9 asks for (then Eq. 11 is "what is left over the layers left" and the
 // last layer, budgeted by Eq. 8, spends the remainder: the total stays L*H*phi^1).
+// keep_window (not in the paper): the proxy tokens (the last min(window, n) positions) are always retained, so a
+// head's budgets are floored at the window's token counts per modality: with lo_v, lo_t those counts and
+// P' = max(Phi^l, lo_v + lo_t), the visual budget of Eq. 8 is brought into [lo_v, P' - lo_t] and the text budget is
+// P' minus it. Masses, preferences, Eq. 9 and Eq. 10-11 are untouched.
 int mo_allocate(int B, int L, int Hkv, int n_max, const float* psi, const uint8_t* mask, const int32_t* seq_len,
-                const int32_t* budget, float theta, int mpa, int hcc_mode, double* mass, double* pref,
-                int32_t* demand, double* phi, int32_t* budgets, int threads) {
+                const int32_t* budget, float theta, int mpa, int hcc_mode, int keep_window, int window, double* mass,
+                double* pref, int32_t* demand, double* phi, int32_t* budgets, int threads) {
   const int64_t units = (int64_t)B * L * Hkv;
   for_units(units, threads, [=](int64_t u) {
     const int b = (int)(u / ((int64_t)Hkv * L));
@@ -189,6 +196,9 @@ int mo_allocate(int B, int L, int Hkv, int n_max, const float* psi, const uint8_
     int n_v = 0;
     for (int i = 0; i < n; ++i) n_v += mask[(int64_t)b * n_max + i] ? 1 : 0;
     const int n_t = n - n_v;
+    int lo_v = 0, lo_t = 0;  // window tokens per modality (forced retention), 0 without keep_window
+    if (keep_window)
+      for (int i = std::max(0, n - window); i < n; ++i) (mask[(int64_t)b * n_max + i] ? lo_v : lo_t) += 1;
     const double lo = n >= 1 ? 1.0 : 0.0, hi = (double)n;
     double ph = (double)budget[b];  // phi^1
     for (int l = 1; l <= L; ++l) {
@@ -200,9 +210,10 @@ int mo_allocate(int B, int L, int Hkv, int n_max, const float* psi, const uint8_
         const int64_t u = ((int64_t)b * L + (l - 1)) * Hkv + h;
         dem += (int64_t)demand[u * 2] + demand[u * 2 + 1];
         int32_t bv, bt;
-        const int32_t P = (int32_t)Phi;
+        const int32_t P = std::max((int32_t)Phi, lo_v + lo_t);
         if (mpa) {
           bv = (int32_t)std::floor(pref[u * 2] * Phi + 0.5);  // Eq. 8, rounded half up
+          bv = std::min(std::max(bv, lo_v), P - lo_t);         // forced retention of the window (no-op without it)
           bt = P - bv;
           if (bv > n_v) { bt += bv - n_v; bv = n_v; }
           if (bt > n_t) { bv = std::min(n_v, bv + (bt - n_t)); bt = n_t; }
@@ -211,8 +222,9 @@ int mo_allocate(int B, int L, int Hkv, int n_max, const float* psi, const uint8_
           bt = std::min(P, n);
         }
         if (hcc_mode == 3 && l < L) {  // the layer keeps its demand (k_m <= n_m by construction)
-          bv = mpa ? demand[u * 2] : 0;
-          bt = mpa ? demand[u * 2 + 1] : std::min(demand[u * 2] + demand[u * 2 + 1], n);
+          bv = mpa ? std::max(demand[u * 2], lo_v) : 0;
+          bt = mpa ? std::max(demand[u * 2 + 1], lo_t)
+                   : std::min(std::max(demand[u * 2] + demand[u * 2 + 1], lo_v + lo_t), n);
         }
         budgets[u * 2] = bv;
         budgets[u * 2 + 1] = bt;
@@ -229,11 +241,17 @@ int mo_allocate(int B, int L, int Hkv, int n_max, const float* psi, const uint8_
   return 0;
 }
 
-// Stage 4a: keep, of each modality, the budgeted number of highest-psi tokens; list them by position.
+// Stage 4a: keep, of each modality, the budgeted number of highest-scoring tokens; list them by position.
+// Two options the paper does not have (both off by default):
+//   pool_kernel p (odd): tokens are ranked by the maximum of psi over the p positions centred on them (positions
+//     outside the sequence do not count) instead of psi itself: a token next to a strongly attended one is kept with
+//     it. Only the ranking uses the pooled score.
+//   keep_window: the last min(window, n) positions are kept whatever their score; they count towards their
+//     modality's budget, and a budget smaller than their number is raised to it.
 // Returns 5 if a segment would not fit into `capacity` rows (that segment and all later ones are not written).
 int mo_select(int B, int L, int Hkv, int n_max, const float* psi, const uint8_t* mask, const int32_t* seq_len,
-              const int32_t* budgets, int mpa, int headroom, int32_t* kept_len, int64_t* seg_off, int32_t* kept_idx,
-              int64_t capacity) {
+              const int32_t* budgets, int mpa, int headroom, int keep_window, int window, int pool_kernel,
+              int32_t* kept_len, int64_t* seg_off, int32_t* kept_idx, int64_t capacity) {
   const int64_t units = (int64_t)B * L * Hkv;
   int64_t off = 0;
   for (int64_t u = 0; u < units; ++u) {
@@ -241,13 +259,26 @@ int mo_select(int B, int L, int Hkv, int n_max, const float* psi, const uint8_t*
     const int n = seq_len[b];
     const float* p = psi + u * n_max;
     const uint8_t* mk = mask + (int64_t)b * n_max;
-    std::vector<Cand> c[2];
-    for (int i = 0; i < n; ++i) c[(mpa && mk[i]) ? 0 : 1].push_back(Cand{p[i], i});
+    const int r = (pool_kernel - 1) / 2;
+    std::vector<Cand> c[2];  // candidates by score
     std::vector<int32_t> keep;
+    int forced[2] = {0, 0}, count[2] = {0, 0};
+    for (int i = 0; i < n; ++i) {
+      const int m = (mpa && mk[i]) ? 0 : 1;
+      count[m] += 1;
+      if (keep_window && i >= n - window) {  // a proxy token: kept unconditionally
+        keep.push_back(i);
+        forced[m] += 1;
+        continue;
+      }
+      float pooled = p[i];
+      for (int j = std::max(0, i - r); j <= std::min(n - 1, i + r); ++j) pooled = std::max(pooled, p[j]);
+      c[m].push_back(Cand{pooled, i});
+    }
     for (int m = 0; m < 2; ++m) {
       std::sort(c[m].begin(), c[m].end(), before);
-      const int take = std::min<int>(budgets[u * 2 + m], (int)c[m].size());
-      for (int j = 0; j < take; ++j) keep.push_back(c[m][j].pos);
+      const int want = std::min<int>(std::max<int>(budgets[u * 2 + m], forced[m]), count[m]);
+      for (int j = 0; j < want - forced[m]; ++j) keep.push_back(c[m][j].pos);
     }
     std::sort(keep.begin(), keep.end());
     seg_off[u] = off;

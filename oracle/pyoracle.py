@@ -67,8 +67,9 @@ def score(dtype, q_win, k, seq_len, causal=1, scale=None, threads=0, want_lse=Fa
     return (psi, lse) if want_lse else psi
 
 
-def allocate(psi, mask, seq_len, budget, theta, mpa=1, hcc_mode=1, threads=0):
-    """Eq. 6, 8, 9, 10, 11. psi [B,L,Hkv,n_max] float32 -> dict(mass, pref, demand, phi, budgets)."""
+def allocate(psi, mask, seq_len, budget, theta, mpa=1, hcc_mode=1, keep_window=0, window=0, threads=0):
+    """Eq. 6, 8, 9, 10, 11. psi [B,L,Hkv,n_max] float32 -> dict(mass, pref, demand, phi, budgets).
+    keep_window (with the window size): budgets floored at the proxy tokens' counts per modality."""
     psi = _c(psi, np.float32)
     B, L, Hkv, n_max = psi.shape
     mask, seq_len, budget = _c(mask, np.uint8), _c(seq_len, np.int32), _c(budget, np.int32)
@@ -80,26 +81,29 @@ def allocate(psi, mask, seq_len, budget, theta, mpa=1, hcc_mode=1, threads=0):
         budgets=np.zeros((B, L, Hkv, 2), np.int32),
     )
     rc = _load().mo_allocate(B, L, Hkv, n_max, _p(psi), _p(mask), _p(seq_len), _p(budget), ctypes.c_float(theta),
-                             int(mpa), int(hcc_mode), _p(out["mass"]), _p(out["pref"]), _p(out["demand"]),
-                             _p(out["phi"]), _p(out["budgets"]), threads)
+                             int(mpa), int(hcc_mode), int(keep_window), int(window), _p(out["mass"]), _p(out["pref"]),
+                             _p(out["demand"]), _p(out["phi"]), _p(out["budgets"]), threads)
     assert rc == 0, rc
     return out
 
 
-def select(psi, mask, seq_len, budgets, mpa=1, headroom=0, capacity=None):
-    """Stage 4a. Returns (rc, kept_len [units], seg_off [units+1], kept_idx [capacity]); rc 5 = capacity exceeded."""
+def select(psi, mask, seq_len, budgets, mpa=1, headroom=0, capacity=None, keep_window=0, window=0, pool_kernel=1):
+    """Stage 4a. Returns (rc, kept_len [units], seg_off [units+1], kept_idx [capacity]); rc 5 = capacity exceeded.
+    pool_kernel (odd): rank by the maximum of psi over that many positions; keep_window: the last `window` positions
+    of every sequence are always kept."""
+    assert pool_kernel >= 1 and pool_kernel % 2 == 1
     psi = _c(psi, np.float32)
     B, L, Hkv, n_max = psi.shape
     units = B * L * Hkv
     budgets = _c(budgets, np.int32)
     if capacity is None:
-        capacity = int(budgets.reshape(units, 2).sum()) + units * headroom
+        capacity = int(budgets.reshape(units, 2).sum()) + units * (headroom + (window if keep_window else 0))
     kept_len = np.zeros(units, np.int32)
     seg_off = np.zeros(units + 1, np.int64)
     kept_idx = np.full(max(capacity, 1), -1, np.int32)
     rc = _load().mo_select(B, L, Hkv, n_max, _p(psi), _p(_c(mask, np.uint8)), _p(_c(seq_len, np.int32)), _p(budgets),
-                           int(mpa), int(headroom), _p(kept_len), _p(seg_off), _p(kept_idx),
-                           ctypes.c_int64(capacity))
+                           int(mpa), int(headroom), int(keep_window), int(window), int(pool_kernel), _p(kept_len),
+                           _p(seg_off), _p(kept_idx), ctypes.c_int64(capacity))
     return rc, kept_len, seg_off, kept_idx
 
 

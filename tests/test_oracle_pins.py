@@ -336,6 +336,103 @@ def test_select_equals_full_sort_brute_force():
     assert rc == 5
 
 
+def test_pooling_and_window_retention_handworked_case():
+    # options this build adds to the paper's selection step (the paper defines neither): values worked by hand
+    with open(os.path.join(GOLDEN, "pooling_window_16.json")) as f:
+        g = json.load(f)
+    h = _hand()
+    q, k, _, mask, sl = _hand_inputs(h)
+    psi = oracle.score(0, q, k, sl, scale=1 / 8).astype(np.float32)
+    bud8 = np.array([[[[3, 5]]]], np.int32)
+
+    def kept(budgets, **kw):
+        rc, kl, so, ki = oracle.select(psi, mask, sl, budgets, **kw)
+        assert rc == 0
+        return ki[: kl[0]].tolist()
+
+    assert kept(bud8, pool_kernel=3) == g["kept_pool3"]
+    assert kept(bud8, pool_kernel=3, keep_window=1, window=2) == g["kept_pool3_keep_window"]
+    assert kept(bud8, keep_window=1, window=2) == g["kept_pool1_keep_window"]
+    assert kept(bud8) == h["kept_idx"]  # both options off: the base case
+    for budget, key in ((2, "budget_2_keep_window"), (1, "budget_1_keep_window")):
+        al = oracle.allocate(psi, mask, sl, np.array([budget], np.int32), 0.5, keep_window=1, window=2)
+        assert al["budgets"][0, 0, 0].tolist() == [g[key]["b_v"], g[key]["b_t"]]
+        assert kept(al["budgets"], keep_window=1, window=2) == g[key]["kept"]
+    al = oracle.allocate(psi, mask, sl, np.array([2], np.int32), 0.5)
+    assert al["budgets"][0, 0, 0].tolist() == [g["budget_2_no_keep"]["b_v"], g["budget_2_no_keep"]["b_t"]]
+    assert kept(al["budgets"]) == g["budget_2_no_keep"]["kept"]
+    al8 = oracle.allocate(psi, mask, sl, np.array([8], np.int32), 0.5, keep_window=1, window=2)
+    assert al8["budgets"][0, 0, 0].tolist() == [g["budget_8"]["b_v"], g["budget_8"]["b_t"]]
+
+
+@pytest.mark.parametrize("pool", [1, 3, 7, 15])
+@pytest.mark.parametrize("keep", [0, 1])
+def test_pooled_selection_equals_library_maximum_filter_and_full_sort(pool, keep):
+    # the ranking score against scipy's maximum filter (positions outside the sequence do not count: fill with -inf),
+    # the choice against a full sort, the forced window positions against their definition
+    from scipy.ndimage import maximum_filter1d
+
+    rng = np.random.RandomState(80 + pool)
+    B, L, H, n, w = 2, 2, 2, 131, 9
+    psi = (rng.randint(1, 40, size=(B, L, H, n)) / 64).astype(np.float32)  # many exact ties
+    mask = (rng.rand(B, n) < 0.6).astype(np.uint8)
+    sl = np.array([131, 77], np.int32)
+    budgets = rng.randint(0, 50, size=(B, L, H, 2)).astype(np.int32)
+    rc, kept_len, seg_off, kept_idx = oracle.select(psi, mask, sl, budgets, headroom=2, keep_window=keep, window=w,
+                                                    pool_kernel=pool)
+    assert rc == 0
+    u = 0
+    for b in range(B):
+        nb = int(sl[b])
+        win = set(range(max(0, nb - w), nb)) if keep else set()
+        for l in range(L):
+            for hh in range(H):
+                pooled = maximum_filter1d(psi[b, l, hh, :nb].astype(np.float64), size=pool, mode="constant", cval=-np.inf)
+                assert (pooled >= psi[b, l, hh, :nb]).all()
+                want = set(win)
+                for m, val in enumerate((1, 0)):
+                    pos = np.nonzero(mask[b, :nb] == val)[0]
+                    forced = [x for x in pos.tolist() if x in win]
+                    free = np.array([x for x in pos.tolist() if x not in win], np.int64)
+                    take = min(max(int(budgets[b, l, hh, m]), len(forced)), pos.size) - len(forced)
+                    order = np.lexsort((free, -pooled[free])) if free.size else np.zeros(0, np.int64)
+                    want |= set(free[order][:take].tolist())
+                got = kept_idx[seg_off[u]: seg_off[u] + kept_len[u]].tolist()
+                assert got == sorted(want), (b, l, hh)
+                assert win <= set(got)
+                u += 1
+
+
+def test_window_retention_floors_budgets_and_changes_nothing_else():
+    rng = np.random.RandomState(81)
+    B, L, H, n, w = 2, 4, 3, 150, 12
+    psi = rng.rand(B, L, H, n).astype(np.float32)
+    mask = (rng.rand(B, n) < 0.5).astype(np.uint8)
+    sl = np.array([150, 90], np.int32)
+    bud = np.array([10, 30], np.int32)
+    for mpa in (1, 0):
+        for mode in (0, 1, 2, 3):
+            base = oracle.allocate(psi, mask, sl, bud, 0.3, mpa=mpa, hcc_mode=mode)
+            kw = oracle.allocate(psi, mask, sl, bud, 0.3, mpa=mpa, hcc_mode=mode, keep_window=1, window=w)
+            for key in ("mass", "pref", "demand", "phi"):
+                assert np.array_equal(base[key], kw[key]), key
+            for b in range(B):
+                nb = int(sl[b])
+                win = mask[b, nb - w: nb]
+                lo = np.array([int(win.sum()), int(w - win.sum())]) if mpa else np.array([0, w])
+                assert (kw["budgets"][b] >= lo).all()
+                # a head's total: the layer budget, or the window size where that is larger
+                if mode != 3:
+                    Phi = np.clip(np.floor(base["phi"][b] + 0.5), 1, nb).astype(np.int64)
+                    tot = np.maximum(Phi, w)[:, None]
+                    assert (kw["budgets"][b].sum(-1) == np.broadcast_to(tot, (L, H))).all()
+                # where the base budgets already cover the window nothing changes
+                same = (base["budgets"][b] >= lo).all(-1)
+                assert np.array_equal(kw["budgets"][b][same], base["budgets"][b][same])
+            rc, kl, so, ki = oracle.select(psi, mask, sl, kw["budgets"], mpa=mpa, keep_window=1, window=w)
+            assert rc == 0 and np.array_equal(kl, kw["budgets"].reshape(-1, 2).sum(-1))
+
+
 def test_compact_is_row_gather():
     rng = np.random.RandomState(9)
     B, L, H, n, d = 1, 2, 2, 31, 64
