@@ -77,6 +77,12 @@ typedef struct madakv_config {
   int32_t max_new_tokens;   /* rows of headroom left after every ragged segment for Eq. 4 appends          */
   float theta;              /* threshold of Eq. 9, 0 <= theta <= 1                                        */
   float softmax_scale;      /* 0 means 1/sqrt(head_dim) (Eq. 5)                                           */
+  /* Two options of the selection step that the paper does not have (it defines no pooling and says nothing about
+   * retaining the proxy tokens); both are off in the paper-literal setting 0 / 1.                                 */
+  int32_t keep_window;      /* 1: the proxy tokens (the last min(w, seq_len) positions) are always kept; budgets
+                               are floored at their number per modality (madakv_allocate, madakv_select)          */
+  int32_t pool_kernel;      /* odd, 1..15. p > 1: stage 4a ranks tokens by the maximum of psi over the p positions
+                               centred on them (inside the sequence) instead of psi itself. 1 = no pooling        */
 } madakv_config;
 
 /* Strides in elements of a [B, L, H, tokens, d] tensor; d is contiguous. */
@@ -128,6 +134,9 @@ int madakv_score_lse(const madakv_config* cfg, const void* q_win, madakv_strides
  *   budgets[u][0] = floor(pref_v * Phi^l + 1/2), budgets[u][1] = Phi^l - budgets[u][0]; a modality with fewer
  *                  tokens than its share passes the surplus to the other one (both capped by their token counts).
  *                  With cfg->mpa = 0: budgets[u] = {0, min(Phi^l, n)}.
+ *                  With cfg->keep_window: lo_v, lo_t = visual / text tokens among the last min(w, n) positions,
+ *                  P' = max(Phi^l, lo_v + lo_t); the visual budget above is first brought into [lo_v, P' - lo_t] and
+ *                  the text budget is P' minus it (mpa = 0: {0, min(P', n)}). Nothing else changes.
  *   psi [B,L,H_kv,n_max] fp32; mask [B,n_max] uint8 (1 = visual token); seq_len [B]; budget [B] int32 >= 1
  *   mass, pref [B,L,H_kv,2] fp64 (mass = W_m / 2^32); demand, budgets [B,L,H_kv,2] int32; phi [B,L] fp64      */
 int madakv_allocate(const madakv_config* cfg, const float* psi, const uint8_t* mask, const int32_t* seq_len,
@@ -154,7 +163,11 @@ int madakv_allocate_layer(const madakv_config* cfg, int32_t layer, const float* 
  *   seg_off[u]  = sum_{u' < u} (kept_len[u'] + cfg->max_new_tokens), seg_off has B*L*H_kv + 1 entries (rows)
  *   kept_idx[seg_off[u] + j], j < kept_len[u]: the j-th kept position
  * With cfg->mpa = 0 the mask is ignored and budgets[u][1] positions are kept. A segment that would end beyond
- * `capacity` rows is not written and sets MADAKV_ECAPACITY in the status word.                             */
+ * `capacity` rows is not written and sets MADAKV_ECAPACITY in the status word.
+ * Options outside the paper: with cfg->pool_kernel = p > 1 "largest psi" reads "largest max of psi over positions
+ * i - (p-1)/2 .. i + (p-1)/2 inside the sequence" (only this ranking uses the pooled value). With cfg->keep_window
+ * the last min(w, seq_len) positions are kept whatever their score; they count towards their modality's budget, a
+ * budget smaller than their number acts as that number, and kept_len counts accordingly.                     */
 int madakv_select(const madakv_config* cfg, const float* psi, const uint8_t* mask, const int32_t* seq_len,
                   const int32_t* budgets, int32_t* kept_len, int64_t* seg_off, int32_t* kept_idx, int64_t capacity,
                   void* ws, size_t ws_bytes, void* stream);
@@ -209,7 +222,8 @@ int madakv_poll_status(void* ws, void* stream, int32_t* status_out);
 const char* madakv_status_string(int status);
 
 /* Library version, bumped when the ABI changes. 2: madakv_score_lse, madakv_allocate_layer and MADAKV_HCC_DEMAND added
- * (nothing that version 1 had was changed). */
+ * (nothing that version 1 had was changed). 3: madakv_config grew by keep_window and pool_kernel (struct_size is
+ * checked: a caller built against version 2 gets MADAKV_EINVAL, not a misread struct). */
 int madakv_abi_version(void);
 
 #ifdef __cplusplus

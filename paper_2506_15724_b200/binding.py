@@ -33,6 +33,7 @@ class MadakvConfig(ctypes.Structure):
         ("head_dim", ctypes.c_int32), ("max_seq_len", ctypes.c_int32), ("window", ctypes.c_int32),
         ("causal", ctypes.c_int32), ("mpa", ctypes.c_int32), ("hcc_mode", ctypes.c_int32),
         ("max_new_tokens", ctypes.c_int32), ("theta", ctypes.c_float), ("softmax_scale", ctypes.c_float),
+        ("keep_window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32),
     ]
 
 
@@ -81,10 +82,11 @@ def lib():
 
 
 def make_config(dtype, batch, n_layers, n_q_heads, n_kv_heads, head_dim, max_seq_len, window, causal=1, mpa=1,
-                hcc_mode=HCC_PAPER, max_new_tokens=0, theta=0.5, softmax_scale=0.0):
+                hcc_mode=HCC_PAPER, max_new_tokens=0, theta=0.5, softmax_scale=0.0, keep_window=0, pool_kernel=1):
     code = {torch.float32: MADAKV_F32, torch.bfloat16: MADAKV_BF16}.get(dtype, dtype)
     return MadakvConfig(ctypes.sizeof(MadakvConfig), code, batch, n_layers, n_q_heads, n_kv_heads, head_dim,
-                        max_seq_len, window, causal, mpa, hcc_mode, max_new_tokens, theta, softmax_scale)
+                        max_seq_len, window, causal, mpa, hcc_mode, max_new_tokens, theta, softmax_scale, keep_window,
+                        pool_kernel)
 
 
 def _ptr(t):

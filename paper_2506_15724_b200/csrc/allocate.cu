@@ -28,7 +28,7 @@ struct AllocParams {
   int32_t* demand;
   double* phi;
   int32_t* budgets;
-  int L, Hkv, n_max, mpa, hcc_mode;
+  int L, Hkv, n_max, mpa, hcc_mode, keep_window, window;
   u64 theta_fix;  // floor(theta * 2^32)
 };
 
@@ -309,19 +309,21 @@ __device__ __forceinline__ double next_phi(double ph, long long dem, int Hkv, in
 }
 // Eq. 8 integerised for one head: the visual share rounded half up, the rest to text, surplus of a modality with too
 // few tokens passed to the other. With `keep_demand` (mode DEMAND, every layer but the last) the head keeps what
-// Eq. 9 asked for instead.
+// Eq. 9 asked for instead. lo_v, lo_t: the proxy tokens of each modality when they are retained unconditionally
+// (cfg->keep_window), else 0: budgets are floored at them, the head's total at their sum.
 __device__ __forceinline__ void split_budget(const AllocParams& p, int64_t u, double Phi, int n, int n_v, int n_t,
-                                             bool keep_demand) {
+                                             int lo_v, int lo_t, bool keep_demand) {
   if (keep_demand) {
     const int dv = p.demand[u * 2], dt = p.demand[u * 2 + 1];
-    p.budgets[u * 2] = p.mpa ? dv : 0;
-    p.budgets[u * 2 + 1] = p.mpa ? dt : min(dv + dt, n);
+    p.budgets[u * 2] = p.mpa ? max(dv, lo_v) : 0;
+    p.budgets[u * 2 + 1] = p.mpa ? max(dt, lo_t) : min(max(dv + dt, lo_v + lo_t), n);
     return;
   }
-  const int P = (int)Phi;
+  const int P = max((int)Phi, lo_v + lo_t);
   int bv, bt;
   if (p.mpa) {
     bv = (int)floor(__dadd_rn(__dmul_rn(p.pref[u * 2], Phi), 0.5));  // Eq. 8, rounded half up
+    bv = min(max(bv, lo_v), P - lo_t);
     bt = P - bv;
     if (bv > n_v) { bt += bv - n_v; bv = n_v; }
     if (bt > n_t) { bv = min(n_v, bv + (bt - n_t)); bt = n_t; }
@@ -337,12 +339,14 @@ __device__ __forceinline__ void split_budget(const AllocParams& p, int64_t u, do
 __global__ void alloc_seq_kernel(AllocParams p) {
   extern __shared__ double s_Phi[];  // [L] rounded budgets, then [L] demand sums (as long long)
   long long* s_dem = reinterpret_cast<long long*>(s_Phi + p.L);
-  __shared__ int s_nv;
+  __shared__ int s_nv, s_wv;
   const int b = blockIdx.x;
   const int n = clamped_len(p.seq_len, b, p.n_max);
-  if (threadIdx.x == 0) s_nv = 0;
+  const int wlen = p.keep_window ? min(p.window, n) : 0;  // proxy tokens retained unconditionally
+  if (threadIdx.x == 0) s_nv = s_wv = 0;
   __syncthreads();
   count_visual(p.mask + (int64_t)b * p.n_max, n, &s_nv);
+  if (wlen > 0) count_visual(p.mask + (int64_t)b * p.n_max + (n - wlen), wlen, &s_wv);
   // Eq. 10's sum over heads, one warp per layer (integers: any order gives the same sum)
   for (int l = threadIdx.x >> 5; l < p.L; l += blockDim.x >> 5) {
     const long long dem = layer_demand(p.demand + ((int64_t)b * p.L + l) * p.Hkv * 2, p.Hkv);
@@ -350,6 +354,7 @@ __global__ void alloc_seq_kernel(AllocParams p) {
   }
   __syncthreads();
   const int n_v = s_nv, n_t = n - n_v;
+  const int lo_v = p.mpa ? s_wv : 0, lo_t = wlen - lo_v;
   if (threadIdx.x == 0) {
     const double lo = n >= 1 ? 1.0 : 0.0, hi = (double)n;
     double ph = (double)p.budget[b];
@@ -361,27 +366,30 @@ __global__ void alloc_seq_kernel(AllocParams p) {
   }
   __syncthreads();
   for (int x = threadIdx.x; x < p.L * p.Hkv; x += blockDim.x)
-    split_budget(p, (int64_t)b * p.L * p.Hkv + x, s_Phi[x / p.Hkv], n, n_v, n_t,
+    split_budget(p, (int64_t)b * p.L * p.Hkv + x, s_Phi[x / p.Hkv], n, n_v, n_t, lo_v, lo_t,
                  p.hcc_mode == MADAKV_HCC_DEMAND && x / p.Hkv + 1 < p.L);
 }
 
 // One block per sequence, one layer of a layer-by-layer pass: the same arithmetic as one trip of the scan above. The
 // per-layer arrays (pref, demand, budgets) hold this layer only; phi [B, depth] is the state carried between calls.
 __global__ void alloc_layer_kernel(AllocParams p, int depth, int layer) {
-  __shared__ int s_nv;
+  __shared__ int s_nv, s_wv;
   __shared__ double s_Phi;
   __shared__ long long s_dem;
   const int b = blockIdx.x;
   const int n = clamped_len(p.seq_len, b, p.n_max);
-  if (threadIdx.x == 0) s_nv = 0;
+  const int wlen = p.keep_window ? min(p.window, n) : 0;
+  if (threadIdx.x == 0) s_nv = s_wv = 0;
   __syncthreads();
   count_visual(p.mask + (int64_t)b * p.n_max, n, &s_nv);
+  if (wlen > 0) count_visual(p.mask + (int64_t)b * p.n_max + (n - wlen), wlen, &s_wv);
   if (threadIdx.x < 32) {
     const long long dem = layer_demand(p.demand + (int64_t)b * p.Hkv * 2, p.Hkv);
     if (threadIdx.x == 0) s_dem = dem;
   }
   __syncthreads();
   const int n_v = s_nv, n_t = n - n_v;
+  const int lo_v = p.mpa ? s_wv : 0, lo_t = wlen - lo_v;
   if (threadIdx.x == 0) {
     const double lo = n >= 1 ? 1.0 : 0.0, hi = (double)n;
     const int l = layer + 1;  // the paper counts layers from 1
@@ -397,7 +405,8 @@ __global__ void alloc_layer_kernel(AllocParams p, int depth, int layer) {
   }
   __syncthreads();
   for (int x = threadIdx.x; x < p.Hkv; x += blockDim.x)
-    split_budget(p, (int64_t)b * p.Hkv + x, s_Phi, n, n_v, n_t, p.hcc_mode == MADAKV_HCC_DEMAND && layer + 1 < depth);
+    split_budget(p, (int64_t)b * p.Hkv + x, s_Phi, n, n_v, n_t, lo_v, lo_t,
+                 p.hcc_mode == MADAKV_HCC_DEMAND && layer + 1 < depth);
 }
 
 }  // namespace
@@ -421,6 +430,8 @@ int launch_allocate(const madakv_config& c, const float* psi, const uint8_t* mas
   p.n_max = c.max_seq_len;
   p.mpa = c.mpa;
   p.hcc_mode = c.hcc_mode;
+  p.keep_window = c.keep_window;
+  p.window = c.window;
   p.theta_fix = (u64)((double)c.theta * 4294967296.0);
   const int units = c.batch * c.n_layers * c.n_kv_heads;
   alloc_unit_kernel<<<units, NT, 0, st>>>(p);
@@ -447,6 +458,8 @@ int launch_allocate_layer(const madakv_config& c, int layer, const float* psi, c
   p.n_max = c.max_seq_len;
   p.mpa = c.mpa;
   p.hcc_mode = c.hcc_mode;
+  p.keep_window = c.keep_window;
+  p.window = c.window;
   p.theta_fix = (u64)((double)c.theta * 4294967296.0);
   alloc_unit_kernel<<<c.batch * c.n_kv_heads, NT, 0, st>>>(p);
   alloc_layer_kernel<<<c.batch, 1024, 0, st>>>(p, c.n_layers, layer);

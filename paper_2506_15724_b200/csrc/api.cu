@@ -6,7 +6,7 @@ using namespace madakv;
 
 extern "C" {
 
-int madakv_abi_version(void) { return 2; }
+int madakv_abi_version(void) { return 3; }
 
 const char* madakv_status_string(int s) {
   switch (s) {

@@ -14,7 +14,8 @@ namespace madakv {
 // ---------------------------------------------------------------------------------------------------------------
 // Workspace layout (device memory owned by the caller)
 //   [0, 256)                 header: int32 status, then counters used by persistent kernels
-//   [256, ..)                stage 4 scratch: visual-token count per sequence [B] int32
+//   [256, ..)                stage 4 scratch: visual-token count per sequence [B] int32, visual tokens among the
+//                            proxy tokens per sequence [B] int32
 //   [.., .. + score)         stage 1 scratch: finished-item counters [units * rows] int32, log2-domain row
 //                            log-sum-exp [units * rows] fp32 (rows = g * w padded to a multiple of 32), per-chunk
 //                            partial (max, sum) pairs (see ws_layout)
@@ -48,7 +49,7 @@ inline WsLayout ws_layout(const madakv_config& c) {
   w.decode_splits = (c.max_seq_len + c.max_new_tokens + kDecodeChunk - 1) / kDecodeChunk;
   size_t off = kHeaderBytes;
   w.seq_nv_off = off;
-  off = align_up(off + (size_t)c.batch * sizeof(int32_t), 256);
+  off = align_up(off + 2 * (size_t)c.batch * sizeof(int32_t), 256);  // per sequence: visual tokens, visual proxy tokens
   const size_t rows_pad = (rows + 31) / 32 * 32;  // the tensor-core path pads the row count
   w.score_done_off = off;
   off = align_up(off + units * rows_pad * sizeof(int32_t), 256);
@@ -93,6 +94,9 @@ inline int check_config(const madakv_config* c) {
   if (c->max_new_tokens < 0) return MADAKV_ESHAPE;
   if (!(c->theta >= 0.0f && c->theta <= 1.0f)) return MADAKV_EINVAL;
   if (!(c->softmax_scale >= 0.0f)) return MADAKV_EINVAL;
+  if (c->keep_window != 0 && c->keep_window != 1) return MADAKV_EINVAL;
+  if (c->pool_kernel < 1 || c->pool_kernel % 2 == 0) return MADAKV_EINVAL;
+  if (c->pool_kernel > 15) return MADAKV_EUNSUPPORTED;
   return MADAKV_OK;
 }
 

@@ -8,6 +8,10 @@
 //                the lowest positions (block-wide prefix scans provide the tie ranks and the output slots).
 //                A thread owns KPT consecutive positions and keeps their keys in registers from the first pass to
 //                the sweep (sequences longer than one chunk are re-read from L2 chunk by chunk).
+// Two options outside the paper: with pooling the ranking key of a position is the maximum of the keys of the
+// positions around it (a maximum of fp32 values is exact, so nothing changes for the integer results); with
+// forced retention the proxy tokens are emitted by the sweep without taking part in the ranking, and the wanted
+// counts shrink by their number.
 // Integer work only: results are bit-exact functions of (psi bits, mask, budgets).
 #include "common.cuh"
 
@@ -30,27 +34,41 @@ struct SelParams {
   int64_t capacity;
   void* ws;
   int32_t* seq_nv;  // ws: visual-token count of every sequence
-  int units, B, L, Hkv, n_max, mpa, headroom;
+  int32_t* seq_wv;  // ws: visual tokens among the proxy tokens of every sequence (forced retention)
+  int units, B, L, Hkv, n_max, mpa, headroom, keep_window, window, pool_r;  // pool_r: (pool_kernel - 1) / 2
 };
 
 __global__ void __launch_bounds__(1024) seg_scan_kernel(SelParams p) {
   __shared__ long long warp_tot[32];
   __shared__ long long carry;
-  __shared__ int s_cnt;
+  __shared__ int s_cnt, s_wcnt;
   // visual tokens among the first seq_len[b] positions of every sequence
   for (int b = 0; b < p.B; ++b) {
     const int n = clamped_len(p.seq_len, b, p.n_max);
     const uint8_t* mask = p.mask + (int64_t)b * p.n_max;
-    if (threadIdx.x == 0) s_cnt = 0;
+    const int wfrom = p.keep_window ? max(n - p.window, 0) : n;  // first proxy token retained unconditionally
+    if (threadIdx.x == 0) s_cnt = s_wcnt = 0;
     __syncthreads();
-    int c = 0;
+    int c = 0, cw = 0;  // visual tokens, visual proxy tokens
     if (p.mpa)
-      for (int i = threadIdx.x; i < n; i += 1024) c += mask[i] ? 1 : 0;
+      for (int i = threadIdx.x; i < n; i += 1024)
+        if (mask[i]) {
+          ++c;
+          if (i >= wfrom) ++cw;
+        }
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) c += __shfl_xor_sync(kFull, c, off);
+    for (int off = 16; off >= 1; off >>= 1) {
+      c += __shfl_xor_sync(kFull, c, off);
+      cw += __shfl_xor_sync(kFull, cw, off);
+    }
     if ((threadIdx.x & 31) == 0 && c) atomicAdd(&s_cnt, c);
+    if ((threadIdx.x & 31) == 0 && cw) atomicAdd(&s_wcnt, cw);
     __syncthreads();
-    if (threadIdx.x == 0) p.seq_nv[b] = s_cnt;
+    if (threadIdx.x == 0) {
+      p.seq_nv[b] = s_cnt;
+      p.seq_wv[b] = s_wcnt;
+    }
+    __syncthreads();
   }
   if (threadIdx.x == 0) carry = 0;
   __syncthreads();  // also orders the seq_nv stores before the loads below (same block)
@@ -61,7 +79,8 @@ __global__ void __launch_bounds__(1024) seg_scan_kernel(SelParams p) {
       const int b = u / (p.Hkv * p.L);
       const int n = clamped_len(p.seq_len, b, p.n_max);
       const int n_v = p.seq_nv[b];
-      const int len = (p.mpa ? min(max(p.budgets[2 * u], 0), n_v) : 0) + min(max(p.budgets[2 * u + 1], 0), n - n_v);
+      const int lo_v = p.seq_wv[b], lo_t = (p.keep_window ? min(p.window, n) : 0) - lo_v;  // proxy tokens kept anyway
+      const int len = (p.mpa ? min(max(p.budgets[2 * u], lo_v), n_v) : 0) + min(max(p.budgets[2 * u + 1], lo_t), n - n_v);
       p.kept_len[u] = len;
       v = (long long)len + p.headroom;
     }
@@ -109,12 +128,35 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* warp_t
   return wbase + incl - v;
 }
 
-template <bool kVec>
-__device__ __forceinline__ void load_chunk(const float* psi, const uint8_t* mask, int n, int pos0, int mpa,
-                                           uint32_t (&key)[KPT], uint32_t& valid, uint32_t& vis) {
+constexpr int kMaxPoolR = 7;  // pool_kernel <= 15
+
+// Keys of KPT consecutive positions from pos0. valid: positions that take part in the ranking (inside the sequence
+// and not retained unconditionally); forced: proxy tokens retained unconditionally (positions wfrom .. n-1);
+// vis: visual tokens. With kPool the key of a position is the maximum over the 2 * pool_r + 1 positions around it.
+template <bool kVec, bool kPool>
+__device__ __forceinline__ void load_chunk(const float* psi, const uint8_t* mask, int n, int pos0, int mpa, int wfrom,
+                                           int pool_r, uint32_t (&key)[KPT], uint32_t& valid, uint32_t& vis,
+                                           uint32_t& forced) {
   valid = 0;
   vis = 0;
-  if (kVec && pos0 + KPT <= n) {
+  forced = 0;
+  if (kPool) {
+    uint32_t e[KPT + 2 * kMaxPoolR];  // keys of positions pos0 - 7 .. pos0 + KPT + 6 (0 outside the sequence)
+#pragma unroll
+    for (int x = 0; x < KPT + 2 * kMaxPoolR; ++x) {
+      const int pos = pos0 - kMaxPoolR + x;
+      e[x] = (pos >= 0 && pos < n) ? psi_key(__ldg(psi + pos)) : 0u;
+    }
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+      uint32_t m = e[j + kMaxPoolR];
+#pragma unroll
+      for (int d = 1; d <= kMaxPoolR; ++d)
+        if (d <= pool_r) m = max(m, max(e[j + kMaxPoolR - d], e[j + kMaxPoolR + d]));
+      key[j] = pos0 + j < n ? m : 0u;
+      if (pos0 + j < n) valid |= 1u << j;
+    }
+  } else if (kVec && pos0 + KPT <= n) {
 #pragma unroll
     for (int j = 0; j < KPT; j += 4) {
       const float4 v = __ldg(reinterpret_cast<const float4*>(psi + pos0 + j));
@@ -139,13 +181,19 @@ __device__ __forceinline__ void load_chunk(const float* psi, const uint8_t* mask
     for (int j = 0; j < KPT; ++j)
       if (pos0 + j < n && __ldg(mask + pos0 + j)) vis |= 1u << j;
   }
+  if (pos0 + KPT > wfrom) {  // proxy tokens retained unconditionally: out of the ranking, into the sweep's output
+#pragma unroll
+    for (int j = 0; j < KPT; ++j)
+      if (pos0 + j >= wfrom && pos0 + j < n) forced |= 1u << j;
+    valid &= ~forced;
+  }
 }
 
 // The radix digits are taken from t = kmax - key, starting at the highest bit in which the unit's keys differ
 // (kmax, kmin: largest and smallest key of the unit): importance values share their sign and most exponent bits,
 // so digits of the raw key would put nearly all keys into a handful of buckets and serialise the shared atomics.
 // Ascending t is descending importance.
-template <bool kVec>
+template <bool kVec, bool kPool>
 __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
   __shared__ unsigned int cnt[2][256];
   __shared__ uint32_t s_prefix[2];
@@ -160,15 +208,19 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
   const uint8_t* mask = p.mask + (int64_t)b * p.n_max;
   const int64_t off0 = p.seg_off[u];
   if (off0 + p.kept_len[u] + p.headroom > p.capacity) return;  // seg_scan has raised MADAKV_ECAPACITY
-  const int want0 = p.mpa ? max(p.budgets[2 * u], 0) : 0, want1 = max(p.budgets[2 * u + 1], 0);
+  // proxy tokens retained unconditionally (none without cfg->keep_window): they are emitted by the sweep and the
+  // ranking only has to find the rest of each modality's budget
+  const int wfrom = p.keep_window ? max(n - p.window, 0) : n;
+  const int lo_v = p.seq_wv[b], lo_t = (n - wfrom) - lo_v;
+  const int want0 = p.mpa ? max(p.budgets[2 * u] - lo_v, 0) : 0, want1 = max(p.budgets[2 * u + 1] - lo_t, 0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunks = (n + CHUNK - 1) / CHUNK;
 
   // range of the unit's keys (the chunk stays in registers when there is only one)
-  uint32_t key[KPT], valid = 0, vis = 0;
+  uint32_t key[KPT], valid = 0, vis = 0, forced = 0;
   uint32_t kmax = 0, kmin = 0xffffffffu;
   for (int c = 0; c < chunks; ++c) {
-    load_chunk<kVec>(psi, mask, n, c * CHUNK + (int)threadIdx.x * KPT, p.mpa, key, valid, vis);
+    load_chunk<kVec, kPool>(psi, mask, n, c * CHUNK + (int)threadIdx.x * KPT, p.mpa, wfrom, p.pool_r, key, valid, vis, forced);
 #pragma unroll
     for (int j = 0; j < KPT; ++j)
       if ((valid >> j) & 1u) {
@@ -209,7 +261,7 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
     const uint32_t pre0 = s_prefix[0], pre1 = s_prefix[1];
     for (int c = 0; c < chunks; ++c) {
       if (chunks > 1) {
-        load_chunk<kVec>(psi, mask, n, c * CHUNK + (int)threadIdx.x * KPT, p.mpa, key, valid, vis);
+        load_chunk<kVec, kPool>(psi, mask, n, c * CHUNK + (int)threadIdx.x * KPT, p.mpa, wfrom, p.pool_r, key, valid, vis, forced);
 #pragma unroll
         for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
       }
@@ -266,7 +318,7 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
   for (int c = 0; c < chunks; ++c) {
     const int pos0 = c * CHUNK + (int)threadIdx.x * KPT;
     if (chunks > 1) {
-      load_chunk<kVec>(psi, mask, n, pos0, p.mpa, key, valid, vis);
+      load_chunk<kVec, kPool>(psi, mask, n, pos0, p.mpa, wfrom, p.pool_r, key, valid, vis, forced);
 #pragma unroll
       for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
     }
@@ -286,7 +338,7 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
     // a threshold-valued key is kept while its rank among the modality's ties (in position order) is below ties[m]
     const int room0 = ties0 - (tie_run0 + (int)(eq_before & 0xffffu));
     const int room1 = ties1 - (tie_run1 + (int)(eq_before >> 16));
-    uint32_t keep_bits = gt_bits;
+    uint32_t keep_bits = gt_bits | forced;
     {
       uint32_t ev = eq_bits & vis, et = eq_bits & ~vis;
       for (int k = 0; k < room0 && ev && want0 > 0; ++k) {  // lowest positions first
@@ -335,10 +387,15 @@ int launch_select(const madakv_config& c, const float* psi, const uint8_t* mask,
   p.mpa = c.mpa;
   p.headroom = c.max_new_tokens;
   p.seq_nv = reinterpret_cast<int32_t*>((char*)ws + ws_layout(c).seq_nv_off);
+  p.seq_wv = p.seq_nv + c.batch;
+  p.keep_window = c.keep_window;
+  p.window = c.window;
+  p.pool_r = (c.pool_kernel - 1) / 2;
   seg_scan_kernel<<<1, 1024, 0, st>>>(p);
   // 16-byte loads of psi need every unit's row (n_max floats apart) to start on a 16-byte boundary
-  if (c.max_seq_len % 4 == 0) select_unit_kernel<true><<<p.units, NT, 0, st>>>(p);
-  else select_unit_kernel<false><<<p.units, NT, 0, st>>>(p);
+  if (c.pool_kernel > 1) select_unit_kernel<false, true><<<p.units, NT, 0, st>>>(p);
+  else if (c.max_seq_len % 4 == 0) select_unit_kernel<true, false><<<p.units, NT, 0, st>>>(p);
+  else select_unit_kernel<false, false><<<p.units, NT, 0, st>>>(p);
   return launch_status();
 }
 

@@ -42,10 +42,13 @@ def psi_close(got, want, rtol, atol=1e-9):
 
 def oracle_stages_from(wl, cfg, psi32, mask, seq_len, budget, k, v):
     """Oracle stages 2-4 run on a given fp32 psi (numpy inputs). Returns dict of numpy results."""
-    al = oracle.allocate(psi32, mask, seq_len, budget, float(np.float32(cfg.theta)), mpa=cfg.mpa, hcc_mode=cfg.hcc_mode)
+    al = oracle.allocate(psi32, mask, seq_len, budget, float(np.float32(cfg.theta)), mpa=cfg.mpa, hcc_mode=cfg.hcc_mode,
+                         keep_window=cfg.keep_window, window=cfg.window)
     cap = capacity_of(wl)
     rc, kept_len, seg_off, kept_idx = oracle.select(psi32, mask, seq_len, al["budgets"], mpa=cfg.mpa,
-                                                    headroom=cfg.max_new_tokens, capacity=cap)
+                                                    headroom=cfg.max_new_tokens, capacity=cap,
+                                                    keep_window=cfg.keep_window, window=cfg.window,
+                                                    pool_kernel=cfg.pool_kernel)
     assert rc == 0
     k_c, v_c = oracle.compact(dcode(wl), k, v, kept_idx, seg_off, kept_len, cap)
     al.update(kept_len=kept_len, seg_off=seg_off, kept_idx=kept_idx, k_c=k_c, v_c=v_c, capacity=cap)
@@ -89,6 +92,7 @@ def compare_with_pure_oracle(wl, cfg, want_psi, got, mask, seq_len, budget, tie_
     Nothing is skipped silently: the returned dict counts every use of a tie rule."""
     psi32 = np.ascontiguousarray(want_psi, np.float32)
     theta = float(np.float32(cfg.theta))
+    assert cfg.keep_window == 0 and cfg.pool_kernel == 1, "the tie rules are written for the paper-literal selection"
     pure = oracle.allocate(psi32, mask, seq_len, budget, theta, mpa=cfg.mpa, hcc_mode=cfg.hcc_mode)
     B, L, H, n = psi32.shape
     stats = dict(units=B * L * H, demand_ties=0, budget_rounding_ties=0, units_after_a_demand_tie=0, kept_ties=0,

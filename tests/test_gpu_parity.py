@@ -189,6 +189,61 @@ def test_staged_allocate_select_compact_are_bit_exact(name, mpa, hcc):
     assert_segments_equal(ref["kept_len"], ref["seg_off"], to_np(buf.v_c), ref["v_c"], "v_c")
 
 
+@pytest.mark.parametrize("name", ["tiny", "tiny_gqa_ragged", "bf16_gqa7", "tc_short_seqs", "tc_cluster4"])
+@pytest.mark.parametrize("pool,keep", [(3, 0), (1, 1), (7, 1), (15, 1)])
+@pytest.mark.parametrize("mpa,hcc", [(1, mk.HCC_PAPER), (0, mk.HCC_PAPER), (1, mk.HCC_DEMAND)])
+def test_pooling_and_window_retention_are_bit_exact(name, pool, keep, mpa, hcc):
+    """The two selection options outside the paper (score pooling, forced retention of the proxy tokens), staged on
+    the oracle's scores: budgets with the window floors, kept positions under the pooled ranking and compacted rows are
+    bit-exact against the oracle; so is the layer-by-layer allocation call."""
+    wl = SHAPES[name]
+    inp = make_case(wl)
+    cfg = config_of(wl, mpa=mpa, hcc_mode=hcc, keep_window=keep, pool_kernel=pool)
+    mask, sl, bud = to_np(inp["mask"]), to_np(inp["seq_len"]), to_np(inp["budget"])
+    if name == "tiny_gqa_ragged":
+        bud = np.array([2, 60, 3], np.int32)  # budgets below the window size: the floors bind
+    psi32 = oracle.score(dcode(wl), to_np(inp["q_win"]), to_np(inp["k"]), sl).astype(np.float32)
+    ref = oracle_stages_from(wl, cfg, psi32, mask, sl, bud, to_np(inp["k"]), to_np(inp["v"]))
+    g = dev(inp)
+    d_bud = torch.from_numpy(bud).cuda()
+    buf = mk.EvictionBuffers(cfg, ref["capacity"])
+    buf.psi.copy_(torch.from_numpy(psi32))
+    mk.madakv_allocate(cfg, buf.psi, g["mask"], g["seq_len"], d_bud, buf.mass, buf.pref, buf.demand, buf.phi,
+                       buf.budgets, buf.ws)
+    for key in ("mass", "pref", "demand", "phi", "budgets"):
+        assert np.array_equal(getattr(buf, key).cpu().numpy(), ref[key]), key
+    if keep:
+        for b in range(wl.B):
+            win = mask[b, max(int(sl[b]) - wl.w, 0): int(sl[b])]
+            lo = [int(win.sum()), int(win.size - win.sum())] if mpa else [0, int(win.size)]
+            assert (ref["budgets"][b] >= np.array(lo)).all()
+    mk.madakv_select(cfg, buf.psi, g["mask"], g["seq_len"], buf.budgets, buf.kept_len, buf.seg_off, buf.kept_idx,
+                     buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    assert np.array_equal(buf.kept_len.cpu().numpy(), ref["kept_len"])
+    assert np.array_equal(buf.seg_off.cpu().numpy(), ref["seg_off"])
+    got_idx = buf.kept_idx.cpu().numpy()
+    assert_segments_equal(ref["kept_len"], ref["seg_off"], got_idx, ref["kept_idx"], "kept_idx")
+    if keep:  # every proxy token of every unit is kept
+        for u in range(wl.units):
+            b = u // (wl.L * wl.Hkv)
+            a0 = int(ref["seg_off"][u])
+            seg = set(got_idx[a0: a0 + int(ref["kept_len"][u])].tolist())
+            assert set(range(max(int(sl[b]) - wl.w, 0), int(sl[b]))) <= seg
+    mk.madakv_compact(cfg, g["k"], g["v"], buf.kept_idx, buf.seg_off, buf.kept_len, buf.k_c, buf.v_c, buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    assert_segments_equal(ref["kept_len"], ref["seg_off"], to_np(buf.k_c), ref["k_c"], "k_c")
+    # the same budgets from the layer-by-layer call
+    if wl.L > 1 and hcc != mk.HCC_DEMAND:
+        cfg1 = config_of(synth.scaled(wl, L=1), mpa=mpa, hcc_mode=hcc, keep_window=keep, pool_kernel=pool)
+        one = mk.EvictionBuffers(cfg1, capacity_of(synth.scaled(wl, L=1)))
+        phi = torch.zeros((wl.B, wl.L), dtype=torch.float64, device="cuda")
+        for l in range(wl.L):
+            mk.madakv_allocate_layer(cfg, l, buf.psi[:, l:l + 1].contiguous(), g["mask"], g["seq_len"], d_bud, one.mass,
+                                     one.pref, one.demand, phi, one.budgets, buf.ws)
+            assert np.array_equal(one.budgets.cpu().numpy()[:, 0], ref["budgets"][:, l]), l
+
+
 @pytest.mark.parametrize("name", list(SHAPES))
 def test_end_to_end_pass_and_decode(name, record_property):
     wl = SHAPES[name]

@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol(lib):
     for name in declared:
         assert hasattr(lib, name), name
     assert declared == set(mk.EXPORTS)
-    assert lib.madakv_abi_version() == 2
+    assert lib.madakv_abi_version() == 3
     assert mk.madakv_status_string(mk.ECAPACITY) == "ragged cache capacity exceeded"
 
 
@@ -50,7 +50,12 @@ def test_workspace_bytes_and_config_validation(lib):
         (dict(causal=2), mk.EINVAL),
         (dict(hcc_mode=9), mk.EINVAL),
         (dict(max_new_tokens=-1), mk.ESHAPE),
+        (dict(pool_kernel=4), mk.EINVAL),       # the pooling width is odd
+        (dict(pool_kernel=0), mk.EINVAL),
+        (dict(pool_kernel=17), mk.EUNSUPPORTED),
+        (dict(keep_window=2), mk.EINVAL),
     ]
+    assert mk.madakv_workspace_bytes(_cfg(pool_kernel=7, keep_window=1)) > 256
     for kw, code in bad:
         with pytest.raises(mk.MadakvError) as e:
             mk.madakv_workspace_bytes(_cfg(**kw))
