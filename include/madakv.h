@@ -108,7 +108,12 @@ int madakv_workspace_bytes(const madakv_config* cfg, size_t* bytes_out);
  *   lse     [B, L, H_q, w] fp32, natural-log sum-exp of every window row's scaled logits. The call computes
  *           these values and stores them here when `lse` is non-null (may be null).
  *   psi     [B, L, H_kv, n_max] fp32, contiguous, written in full
- * Deterministic: a fixed reduction order, no floating-point atomics.                                       */
+ * Deterministic: a fixed reduction order, no floating-point atomics.
+ * The scoring kernels are persistent grids sized to the whole device. One of them (bf16, g * w <= 64, sequences too
+ * long for a thread-block cluster's tensor memory) lets a CTA wait, bounded, for results of other CTAs of the same
+ * launch: give this call the device to itself. If kernels of another stream keep part of its grid from being
+ * scheduled, the wait runs out and the call reports MADAKV_ETIMEOUT through the status word instead of scores
+ * (nothing hangs, the workspace stays usable).                                                              */
 int madakv_score(const madakv_config* cfg, const void* q_win, madakv_strides sq, const void* k, madakv_strides sk,
                  const int32_t* seq_len, float* lse, float* psi, void* ws, size_t ws_bytes, void* stream);
 

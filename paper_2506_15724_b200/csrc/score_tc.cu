@@ -52,6 +52,8 @@ struct TcParams {
   int32_t* status;   // ws header
   int units, L, Hq, Hkv, g, w, R, n_max, cpu, causal, lag;
   float scale2;
+  long long flag_wait_cycles;  // bound of the wait for another CTA's row flags (kWaitCycles unless a test shortens it)
+  int hold_flags;              // failure-path test only: the rows' log-sum-exps are computed but never flagged
 };
 
 // ------------------------------------------------------------------------------------------------ work list
@@ -390,7 +392,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
             if (v >= kReady) break;
             if (*abort_flag) break;
             __nanosleep(64);
-            if ((++spins & 255) == 0 && clock64() - t0 > kWaitCycles) {
+            if ((++spins & 255) == 0 && clock64() - t0 > p.flag_wait_cycles) {
               give_up(abort_flag, p.status, kSiteFlag);
               break;
             }
@@ -508,7 +510,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constan
               const int hq = h * p.g + row / p.w, wr = row % p.w;
               p.lse_out[((int64_t)bl * p.Hq + hq) * p.w + wr] = (Z > 0.f) ? lse2 * 0.6931471805599453f : -INFINITY;
             }
-            asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(cnt), "r"(kReady) : "memory");
+            if (!p.hold_flags)
+              asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(cnt), "r"(kReady) : "memory");
           }
         }
       } else {
@@ -623,6 +626,16 @@ int launch_score_tc(const madakv_config& c, const void* q, madakv_strides sq, co
   if (lag < p.cpu) lag = p.cpu;
   if (lag > 2 * grid) return MADAKV_EUNSUPPORTED;
   p.lag = lag;
+  // Failure-path test (no GPU fault involved): MADAKV_TEST_HOLD_FLAGS=1 withholds the row flags, so every phase-2 item
+  // runs into its bounded wait, and MADAKV_TEST_WAIT_CYCLES shortens that wait from ~2 s to the given number of clock
+  // cycles (at least 100 000). The kernel then records MADAKV_ETIMEOUT, drains and returns by itself.
+  p.flag_wait_cycles = kWaitCycles;
+  p.hold_flags = 0;
+  if (const char* e = getenv("MADAKV_TEST_WAIT_CYCLES")) {
+    const long long v = atoll(e);
+    if (v >= 100000 && v < kWaitCycles) p.flag_wait_cycles = v;
+  }
+  if (const char* e = getenv("MADAKV_TEST_HOLD_FLAGS")) p.hold_flags = atoi(e) == 1;
 
   CUtensorMap mk, mq;
   if (!make_map(&mk, k, c.head_dim, c.max_seq_len, c.n_kv_heads, c.n_layers, c.batch, sk, kTileKeys, 1) ||

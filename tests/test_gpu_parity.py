@@ -558,6 +558,33 @@ def test_decode_with_more_than_65535_segments():
     assert np.abs(out.cpu().numpy() - want).max() <= 2e-5
 
 
+def test_bounded_wait_runs_out_and_the_library_recovers(monkeypatch):
+    """Failure detection without a GPU fault: the two-phase scoring kernel's phase-2 items wait (bounded) for row flags
+    that phase 1 publishes. With the flags withheld and the bound shortened to ~1 ms the wait runs out: the kernel
+    records MADAKV_ETIMEOUT with the wait site, drains its copies and tensor-core work, frees its TMEM and returns;
+    nothing hangs or faults, and the next ordinary call on the same workspace gives the oracle's scores."""
+    wl = synth.scaled(TINY, dtype="bf16", L=1, Hq=2, Hkv=1, d=128, n=700, w=8, budget=90, theta=0.4)  # one CTA
+    inp = make_case(wl)
+    cfg = config_of(wl)
+    g = dev(inp)
+    buf = mk.EvictionBuffers(cfg, capacity_of(wl))
+    monkeypatch.setenv("MADAKV_SCORE_PATH", "twophase")
+    monkeypatch.setenv("MADAKV_TEST_HOLD_FLAGS", "1")
+    monkeypatch.setenv("MADAKV_TEST_WAIT_CYCLES", "2000000")
+    mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], None, buf.psi, buf.ws)
+    torch.cuda.synchronize()
+    site = int(buf.ws[4:8].view(torch.int32).item())
+    assert mk.madakv_poll_status(buf.ws) == mk.ETIMEOUT
+    assert site & 255 == 7 and site >> 8 == 0  # the wait for another item's row flags, in block 0
+    assert mk.madakv_poll_status(buf.ws) == 0   # cleared by the poll
+    monkeypatch.delenv("MADAKV_TEST_HOLD_FLAGS")
+    monkeypatch.delenv("MADAKV_TEST_WAIT_CYCLES")
+    mk.madakv_score(cfg, g["q_win"], g["k"], g["seq_len"], None, buf.psi, buf.ws)
+    assert mk.madakv_poll_status(buf.ws) == 0
+    want = oracle.score(1, to_np(inp["q_win"]), to_np(inp["k"]), to_np(inp["seq_len"]))
+    assert psi_close(buf.psi.cpu().numpy(), want, PSI_RTOL) < PSI_RTOL_SEEN
+
+
 def test_strided_kv_layout():
     # K/V stored per layer as [B, H, n, d] inside a larger allocation (token stride > d)
     wl = synth.scaled(TINY, dtype="bf16", L=2, Hq=4, Hkv=2, d=128, n=340, w=8, budget=50)
