@@ -431,79 +431,117 @@ class Bench:
 
     # ---- the layer-by-layer order (a layer is evicted right after its prefill): per layer single-pass scoring with
     # the prefill's log-sum-exps, madakv_allocate_layer carrying phi, selection and compaction of that layer.
-    # Scoring and compaction (HBM streams) run on one stream; allocation and selection of a layer (a few blocks,
-    # latency-bound) run on a second stream and overlap the scoring of the next layer. The only dependencies are
-    # score(l) -> allocate(l) -> select(l) -> compact(l) and phi(l) -> allocate(l + 1), both kept by events.
-    def time_streamed(self, steps=3, two_streams=True):
+    # Eager on one stream it is launch- and latency-bound (a layer's allocation and selection have only B * H_kv
+    # blocks). The overlapped form keeps several layers in flight: scoring on one stream, allocation + selection of
+    # layer l on stream l % NS, compaction on another; the dependencies score(l) -> allocate(l) -> select(l) ->
+    # compact(l), phi(l) -> allocate(l + 1) and the reuse of a layer's scratch are events. The whole pass is captured
+    # once into a CUDA graph and replayed, so the host's launch cost is out of the picture.
+    def time_streamed(self, steps=3, overlapped=True, NS=4):
         mk, wl, buf, inp = self.mk, self.wl, self.buf, self.inp
         cfg1 = mk.make_config(wl.torch_dtype, wl.B, 1, wl.Hq, wl.Hkv, wl.d, wl.n, wl.w,
                               max_new_tokens=wl.max_new_tokens, theta=wl.theta)
-        slots = 2 if two_streams else 1  # per-layer scratch in flight
-        one = [mk.EvictionBuffers(cfg1, self.cap // wl.L + wl.B * wl.Hkv, device=self.dev) for _ in range(slots)]
+        slots = NS if overlapped else 1  # layers in flight, each with its own scratch
+        # a single layer may be given far more than the nominal budget by the compensation of Eq. 10-11
+        per_layer = wl.B * wl.Hkv * (wl.n + wl.max_new_tokens)
+        one = [mk.EvictionBuffers(cfg1, per_layer, device=self.dev) for _ in range(slots)]
+        ws_side = [mk.new_workspace(buf.cfg, self.dev) for _ in range(slots)]  # allocate_layer's and select's workspace
         lse = torch.empty((wl.B, wl.L, wl.Hq, wl.w), dtype=torch.float32, device=self.dev)
         mk.madakv_score(buf.cfg, inp["q_win"], inp["k"], inp["seq_len"], lse, buf.psi, buf.ws)
         lse_l = [lse[:, l:l + 1].contiguous() for l in range(wl.L)]
         phi = torch.zeros((wl.B, wl.L), dtype=torch.float64, device=self.dev)
-        ws2 = mk.new_workspace(buf.cfg, self.dev)  # allocate_layer's workspace on the second stream
-        main = torch.cuda.current_stream()
-        side = torch.cuda.Stream() if two_streams else main
+        torch.cuda.synchronize()
 
-        def one_pass():
-            done_sel = [None] * slots
-            done_cmp = [None] * slots
+        def one_pass(main):
+            if not overlapped:
+                for l in range(wl.L):
+                    o = one[0]
+                    q_l, k_l, v_l = inp["q_win"][:, l:l + 1], inp["k"][:, l:l + 1], inp["v"][:, l:l + 1]
+                    mk.madakv_score_lse(cfg1, q_l, k_l, inp["seq_len"], lse_l[l], o.psi, o.ws)
+                    mk.madakv_allocate_layer(buf.cfg, l, o.psi, inp["mask"], inp["seq_len"], inp["budget"], o.mass,
+                                             o.pref, o.demand, phi, o.budgets, ws_side[0])
+                    mk.madakv_select(cfg1, o.psi, inp["mask"], inp["seq_len"], o.budgets, o.kept_len, o.seg_off,
+                                     o.kept_idx, ws_side[0])
+                    mk.madakv_compact(cfg1, k_l, v_l, o.kept_idx, o.seg_off, o.kept_len, o.k_c, o.v_c, o.ws)
+                return
+            side = [torch.cuda.Stream() for _ in range(slots)]
+            cmp_s = torch.cuda.Stream()
+            start = torch.cuda.Event()
+            start.record(main)
+            for st in side + [cmp_s]:
+                st.wait_event(start)
+            sel_done, cmp_done, alloc_done = {}, {}, {}
             for l in range(wl.L):
-                o = one[l % slots]
+                o, sd = one[l % slots], side[l % slots]
                 q_l, k_l, v_l = inp["q_win"][:, l:l + 1], inp["k"][:, l:l + 1], inp["v"][:, l:l + 1]
-                if two_streams and done_cmp[l % slots] is not None:
-                    pass  # same stream as the compaction that last read this slot: ordered already
-                if two_streams and done_sel[l % slots] is not None:
-                    main.wait_event(done_sel[l % slots])  # psi of this slot is free once its selection has run
+                if l - slots in sel_done:
+                    main.wait_event(sel_done[l - slots])  # psi of this scratch is free once its selection has run
                 mk.madakv_score_lse(cfg1, q_l, k_l, inp["seq_len"], lse_l[l], o.psi, o.ws)
                 scored = torch.cuda.Event()
                 scored.record(main)
-                with torch.cuda.stream(side):
-                    side.wait_event(scored)
-                    if two_streams and done_cmp[l % slots] is not None:
-                        side.wait_event(done_cmp[l % slots])  # kept_idx of this slot was read by its compaction
+                with torch.cuda.stream(sd):
+                    sd.wait_event(scored)
+                    if l - 1 in alloc_done:
+                        sd.wait_event(alloc_done[l - 1])  # phi^l comes from the layer before (Eq. 11)
+                    if l - slots in cmp_done:
+                        sd.wait_event(cmp_done[l - slots])  # the scratch's kept positions were read by its compaction
                     mk.madakv_allocate_layer(buf.cfg, l, o.psi, inp["mask"], inp["seq_len"], inp["budget"], o.mass,
-                                             o.pref, o.demand, phi, o.budgets, ws2)
+                                             o.pref, o.demand, phi, o.budgets, ws_side[l % slots])
+                    alloc_done[l] = torch.cuda.Event()
+                    alloc_done[l].record(sd)
                     mk.madakv_select(cfg1, o.psi, inp["mask"], inp["seq_len"], o.budgets, o.kept_len, o.seg_off,
-                                     o.kept_idx, ws2)
-                    sel = torch.cuda.Event()
-                    sel.record(side)
-                done_sel[l % slots] = sel
-                if two_streams:
-                    # compaction of the layer before runs behind this layer's scoring on the main stream
-                    if l > 0:
-                        p = one[(l - 1) % slots]
-                        main.wait_event(done_sel[(l - 1) % slots])
-                        mk.madakv_compact(cfg1, inp["k"][:, l - 1:l], inp["v"][:, l - 1:l], p.kept_idx, p.seg_off,
-                                          p.kept_len, p.k_c, p.v_c, p.ws)
-                        c = torch.cuda.Event()
-                        c.record(main)
-                        done_cmp[(l - 1) % slots] = c
-                else:
+                                     o.kept_idx, ws_side[l % slots])
+                    sel_done[l] = torch.cuda.Event()
+                    sel_done[l].record(sd)
+                with torch.cuda.stream(cmp_s):
+                    cmp_s.wait_event(sel_done[l])
                     mk.madakv_compact(cfg1, k_l, v_l, o.kept_idx, o.seg_off, o.kept_len, o.k_c, o.v_c, o.ws)
-            if two_streams:
-                l = wl.L - 1
-                p = one[l % slots]
-                main.wait_event(done_sel[l % slots])
-                mk.madakv_compact(cfg1, inp["k"][:, l:l + 1], inp["v"][:, l:l + 1], p.kept_idx, p.seg_off, p.kept_len,
-                                  p.k_c, p.v_c, p.ws)
+                    cmp_done[l] = torch.cuda.Event()
+                    cmp_done[l].record(cmp_s)
+            for st in side + [cmp_s]:  # join
+                e = torch.cuda.Event()
+                e.record(st)
+                main.wait_event(e)
 
-        for _ in range(2):
-            one_pass()
+        def statuses():
+            return [mk.madakv_poll_status(o.ws) for o in one] + [mk.madakv_poll_status(w) for w in ws_side] + \
+                   [mk.madakv_poll_status(buf.ws)]
+
+        cap_stream = torch.cuda.Stream()
+        with torch.cuda.stream(cap_stream):
+            one_pass(cap_stream)  # eager once: every kernel's attributes are set before the capture
         torch.cuda.synchronize()
-        bad = [mk.madakv_poll_status(o.ws) for o in one] + [mk.madakv_poll_status(ws2), mk.madakv_poll_status(buf.ws)]
-        if any(bad):
+        if any(statuses()):
+            return None
+        graph = None
+        if overlapped:
+            try:
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=cap_stream):
+                    one_pass(cap_stream)
+            except Exception:
+                graph = None
+                torch.cuda.synchronize()
+
+        def run():
+            if graph is not None:
+                graph.replay()
+            else:
+                with torch.cuda.stream(cap_stream):
+                    one_pass(cap_stream)
+
+        run()
+        torch.cuda.synchronize()
+        if any(statuses()):
             return None
         a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(steps):
-            one_pass()
-        z.record()
         torch.cuda.synchronize()
-        return a.elapsed_time(z) / steps
+        with torch.cuda.stream(cap_stream):
+            a.record()
+            for _ in range(steps):
+                run()
+            z.record()
+        torch.cuda.synchronize()
+        return {"ms": a.elapsed_time(z) / steps, "cuda_graph": graph is not None}
 
     def full_cache(self):
         """The same cache without eviction (budget = context length): what decode costs uncompressed."""
@@ -592,13 +630,15 @@ class Bench:
                 "frac_of_measured_peak": k_bytes / (single_ms * 1e-3) / 1e9 / peak,
                 "note": "madakv_score_lse: stage 1 with the rows' log-sum-exps supplied; not part of the step"}
             if with_streamed:
-                s2, s1 = self.time_streamed(two_streams=True), self.time_streamed(two_streams=False)
+                s2, s1 = self.time_streamed(overlapped=True), self.time_streamed(overlapped=False)
                 rec["streamed_pass"] = {
-                    "ms_two_streams": s2, "ms_one_stream": s1, "ratio_to_all_layer_pass":
-                    None if s2 is None else s2 / pass_ms, "launches": wl.L * 7,
+                    "ms_overlapped": None if s2 is None else s2["ms"],
+                    "overlapped_is_a_cuda_graph": None if s2 is None else s2["cuda_graph"],
+                    "ms_eager_one_stream": None if s1 is None else s1["ms"],
+                    "ratio_to_all_layer_pass": None if s2 is None else s2["ms"] / pass_ms, "launches": wl.L * 7,
                     "note": "stages 1-4 layer by layer (madakv_score_lse, madakv_allocate_layer, select and compact "
-                            "with one-layer configs); two streams: allocation and selection of a layer overlap the "
-                            "scoring of the next; not part of the step"}
+                            "with one-layer configs). overlapped: four layers in flight on their own streams (scoring, "
+                            "allocation + selection, compaction), replayed from one CUDA graph; not part of the step"}
         return rec
 
 
