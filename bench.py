@@ -32,9 +32,10 @@ METRIC = "prompt tokens evicted/sec"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
-# exp2 results per clock and SM of the special-function unit, measured on this machine's B200 with a register-only
-# kernel of independent ex2.approx chains (15.99 at 16 and at 32 warps per SM, CUDA events and clock64 agree)
-EXP2_PER_CLK_PER_SM = 15.99
+# exp2 results per clock and SM of the special-function unit: measured in the same run by the exp2-roof probe
+# (paper_2506_15724_b200/csrc/probe/exp2_roof.cu, a register-only kernel of independent ex2.approx chains); this is
+# the figure an earlier run of that probe gave on this machine's B200, used only if the probe cannot be run
+EXP2_PER_CLK_PER_SM_RECORDED = 15.99
 HEADLINE = "long"
 OTHER_WORKLOADS = ("llava", "qwen1024", "qwen", "qwen4096", "batched")
 
@@ -45,6 +46,18 @@ def measured_peaks():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def measure_exp2_roof():
+    """exp2 per clock and SM from the probe binary (built with the library), and how the figure was obtained."""
+    from paper_2506_15724_b200 import build as mkbuild
+
+    try:
+        out = subprocess.run([mkbuild.PROBE], capture_output=True, text=True, timeout=60).stdout
+        rec = json.loads(out.strip().splitlines()[-1])
+        return float(rec["exp2_per_clk_per_sm"]), "measured in this run by the exp2-roof probe", rec
+    except Exception as e:  # no binary, no device, unreadable output
+        return EXP2_PER_CLK_PER_SM_RECORDED, f"recorded from an earlier run of the exp2-roof probe ({type(e).__name__} now)", None
 
 
 def ncu_traffic(kernel, workload):
@@ -320,6 +333,7 @@ class Bench:
         self.dec = [synth.make_decode_step(wl_r, s, device=dev) for s in range(self.n_dec)]
         self.tokens = int(self.inp["seq_len"].sum().item())
         self.peak, self.peak_kind = measured_peaks()
+        self.exp2_roof = None  # (exp2 per clock and SM, how obtained, probe record): set by main() once per run
 
     def step(self, i, ev=None):
         mk, c, buf, inp = self.mk, self.cfg, self.buf, self.inp
@@ -579,13 +593,14 @@ class Bench:
         else:
             props = torch.cuda.get_device_properties(self.dev)
             sm_mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
-            exp_peak = props.multi_processor_count * EXP2_PER_CLK_PER_SM * sm_mhz * 1e6 / 1e12
+            per_clk, roof_how, _ = self.exp2_roof or (EXP2_PER_CLK_PER_SM_RECORDED, "recorded", None)
+            exp_peak = props.multi_processor_count * per_clk * sm_mhz * 1e6 / 1e12
             n_exp = 2.0 * wl.g * wl.w * float(self.tokens) * wl.L * wl.Hkv  # two passes over every logit
             achieved = n_exp / (stage_ms[0] * 1e-3) / 1e12
             roofline = {"bound": "alu", "kernel": "score_rows_kernel pass 1 + pass 2 (stage 1)", "achieved": achieved,
                         "peak": exp_peak, "unit": "Texp2/s", "frac": achieved / exp_peak,
                         "traffic": ncu_traffic("score_rows_kernel", wl.name),
-                        "peak_kind": f"measured: {EXP2_PER_CLK_PER_SM} exp2 per clock and SM (register-only probe) x "
+                        "peak_kind": f"{per_clk:.2f} exp2 per clock and SM ({roof_how}) x "
                                      f"{props.multi_processor_count} SMs x the median SM clock sampled in the timed "
                                      f"region ({sm_mhz:.0f} MHz)",
                         "algorithmic_exp2": n_exp,
@@ -696,8 +711,11 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    exp2_roof = measure_exp2_roof() if rank == 0 else None
+
     # ---- headline workload
     b = Bench(mk, wl, dev, rank)
+    b.exp2_roof = exp2_roof
     total_ms, stage_ms, clocks = b.timed_steps(args.steps, args.warmup, sync_all, local if rank == 0 else None)
     total_ms, tokens_all = reduce_over_ranks(total_ms, b.tokens, dev, world)
     ms_per_step = total_ms / args.steps
@@ -771,6 +789,7 @@ def main():
                 torch.cuda.empty_cache()
                 shared[key] = synth.make_inputs(rank_workload(w2, rank), device=dev)
             bb = Bench(mk, w2, dev, rank, inputs=shared[key])
+            bb.exp2_roof = exp2_roof
             t_ms, st_ms, clk = bb.timed_steps(max(args.steps, 20), args.warmup, sync_all, local)
             rec = bb.record(st_ms, clk, args)
             rec["ms_per_step"] = t_ms / max(args.steps, 20)
@@ -798,6 +817,7 @@ def main():
         "single_pass_score": head.get("single_pass_score"),
         "streamed_pass": head.get("streamed_pass"),
         "cpu_baseline": cpu,
+        "exp2_roof_probe": None if exp2_roof is None else exp2_roof[2],
         "workloads": workloads,
     }
     print(json.dumps(line))

@@ -7,6 +7,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libmadakv.so")
+PROBE_SRC = os.path.join(HERE, "csrc", "probe", "exp2_roof.cu")
+PROBE = os.path.join(HERE, "exp2_roof.bin")  # measures the exp2 roof (see the source); used by bench.py
 
 
 def sources():
@@ -21,7 +23,16 @@ def needs_build():
     return any(os.path.getmtime(f) > t for f in deps)
 
 
+def build_probe(force=False):
+    """The stand-alone exp2-roof probe (a small CUDA program, not part of the library)."""
+    if force or not os.path.exists(PROBE) or os.path.getmtime(PROBE) < os.path.getmtime(PROBE_SRC):
+        subprocess.check_call(["nvcc", "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
+                               "-o", PROBE, PROBE_SRC])
+    return PROBE
+
+
 def build(force=False, verbose=False):
+    build_probe(force)
     if not force and not needs_build():
         return LIB
     cmd = [

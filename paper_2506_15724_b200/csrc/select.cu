@@ -132,7 +132,9 @@ constexpr int kMaxPoolR = 7;  // pool_kernel <= 15
 
 // Keys of KPT consecutive positions from pos0. valid: positions that take part in the ranking (inside the sequence
 // and not retained unconditionally); forced: proxy tokens retained unconditionally (positions wfrom .. n-1);
-// vis: visual tokens. With kPool the key of a position is the maximum over the 2 * pool_r + 1 positions around it.
+// vis: visual tokens. kPool is the variant for the two options outside the paper: the key of a position is the maximum
+// over the 2 * pool_r + 1 positions around it (pool_r may be 0), and the proxy tokens from wfrom on are forced; without
+// kPool neither exists and the code is the plain paper-literal selection.
 template <bool kVec, bool kPool>
 __device__ __forceinline__ void load_chunk(const float* psi, const uint8_t* mask, int n, int pos0, int mpa, int wfrom,
                                            int pool_r, uint32_t (&key)[KPT], uint32_t& valid, uint32_t& vis,
@@ -181,7 +183,7 @@ __device__ __forceinline__ void load_chunk(const float* psi, const uint8_t* mask
     for (int j = 0; j < KPT; ++j)
       if (pos0 + j < n && __ldg(mask + pos0 + j)) vis |= 1u << j;
   }
-  if (pos0 + KPT > wfrom) {  // proxy tokens retained unconditionally: out of the ranking, into the sweep's output
+  if (kPool && pos0 + KPT > wfrom) {  // proxy tokens retained unconditionally: out of the ranking, into the output
 #pragma unroll
     for (int j = 0; j < KPT; ++j)
       if (pos0 + j >= wfrom && pos0 + j < n) forced |= 1u << j;
@@ -210,8 +212,8 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
   if (off0 + p.kept_len[u] + p.headroom > p.capacity) return;  // seg_scan has raised MADAKV_ECAPACITY
   // proxy tokens retained unconditionally (none without cfg->keep_window): they are emitted by the sweep and the
   // ranking only has to find the rest of each modality's budget
-  const int wfrom = p.keep_window ? max(n - p.window, 0) : n;
-  const int lo_v = p.seq_wv[b], lo_t = (n - wfrom) - lo_v;
+  const int wfrom = kPool && p.keep_window ? max(n - p.window, 0) : n;
+  const int lo_v = kPool ? p.seq_wv[b] : 0, lo_t = (n - wfrom) - lo_v;
   const int want0 = p.mpa ? max(p.budgets[2 * u] - lo_v, 0) : 0, want1 = max(p.budgets[2 * u + 1] - lo_t, 0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunks = (n + CHUNK - 1) / CHUNK;
@@ -338,7 +340,7 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
     // a threshold-valued key is kept while its rank among the modality's ties (in position order) is below ties[m]
     const int room0 = ties0 - (tie_run0 + (int)(eq_before & 0xffffu));
     const int room1 = ties1 - (tie_run1 + (int)(eq_before >> 16));
-    uint32_t keep_bits = gt_bits | forced;
+    uint32_t keep_bits = kPool ? (gt_bits | forced) : gt_bits;
     {
       uint32_t ev = eq_bits & vis, et = eq_bits & ~vis;
       for (int k = 0; k < room0 && ev && want0 > 0; ++k) {  // lowest positions first
@@ -393,7 +395,7 @@ int launch_select(const madakv_config& c, const float* psi, const uint8_t* mask,
   p.pool_r = (c.pool_kernel - 1) / 2;
   seg_scan_kernel<<<1, 1024, 0, st>>>(p);
   // 16-byte loads of psi need every unit's row (n_max floats apart) to start on a 16-byte boundary
-  if (c.pool_kernel > 1) select_unit_kernel<false, true><<<p.units, NT, 0, st>>>(p);
+  if (c.pool_kernel > 1 || c.keep_window) select_unit_kernel<false, true><<<p.units, NT, 0, st>>>(p);
   else if (c.max_seq_len % 4 == 0) select_unit_kernel<true, false><<<p.units, NT, 0, st>>>(p);
   else select_unit_kernel<false, false><<<p.units, NT, 0, st>>>(p);
   return launch_status();
