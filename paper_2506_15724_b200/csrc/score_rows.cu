@@ -235,45 +235,49 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   };
 
   if (warp == 0) {
-    // ================================================================ TMA producer
-    if (lane == 0) {
-      const uint64_t pol_k = l2_policy_evict_first();
-      const uint64_t pol_q = l2_policy_evict_last();
-      int stage = 0, cur_u = -1;
-      uint32_t stage_par = 0, q_par = 0;
-      bool ok = true;
-      for (ItemCursor c = cursor_begin(); ok && c.left > 0; cursor_next(c)) {
-        int u, split, key_begin, n;
-        cursor_item(p, c, u, split);
-        const int tiles = item_tiles(u, split, key_begin, n);
-        if (tiles == 0) continue;
-        const int h = u % p.Hkv, l = (u / p.Hkv) % p.L, b = u / (p.Hkv * p.L);
-        if (u != cur_u) {  // the unit changes: its queries (and, in pass 2, its shift rows)
-          cur_u = u;
-          ok = mbar_wait(qempty, q_par ^ 1, abort_flag, p.status, kSiteQEmpty);
-          if (!ok) break;
-          q_par ^= 1;
-          if (PASS == 2) {
-            // Row r of the shift operand: -lse_r / scale as the sum of three bf16 numbers (24 bits) in columns 0-2.
-            // Multiplied by the key side's ones in the extra contraction step, the accumulator holds q.k - lse / scale
-            // and the epilogue needs no per-row operand at all.
-            const float inv = 1.0f / p.scale2;
-            const float* src = p.lse2 + (int64_t)u * p.rs;
-            for (int r = 0; r < p.n16; ++r) {
-              const float v = src[r] * inv;
-              const float hi = __bfloat162float(__float2bfloat16_rn(v));
-              const float mid = __bfloat162float(__float2bfloat16_rn(v - hi));
-              const float low = __bfloat162float(__float2bfloat16_rn((v - hi) - mid));
-              const uint32_t w0 = (__float_as_uint(hi) >> 16) | (__float_as_uint(mid) & 0xffff0000u);
-              *reinterpret_cast<uint4*>(shift_s + r * 128 + (r & 7) * 16) =
-                  make_uint4(w0, __float_as_uint(low) >> 16, 0u, 0u);
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // ================================================================ TMA producer: lane 0 waits and issues the
+    // copies; the whole warp walks the items with it, because in pass 2 all 32 lanes write the unit's shift rows
+    const uint64_t pol_k = l2_policy_evict_first();
+    const uint64_t pol_q = l2_policy_evict_last();
+    int stage = 0, cur_u = -1;
+    uint32_t stage_par = 0, q_par = 0;
+    bool ok = true;
+    for (ItemCursor c = cursor_begin(); ok && c.left > 0; cursor_next(c)) {
+      int u, split, key_begin, n;
+      cursor_item(p, c, u, split);
+      const int tiles = item_tiles(u, split, key_begin, n);
+      if (tiles == 0) continue;
+      const int h = u % p.Hkv, l = (u / p.Hkv) % p.L, b = u / (p.Hkv * p.L);
+      if (u != cur_u) {  // the unit changes: its queries (and, in pass 2, its shift rows)
+        cur_u = u;
+        if (lane == 0) ok = mbar_wait(qempty, q_par ^ 1, abort_flag, p.status, kSiteQEmpty);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        q_par ^= 1;
+        if (PASS == 2) {
+          // Row r of the shift operand: -lse_r / scale as the sum of three bf16 numbers (24 bits) in columns 0-2.
+          // Multiplied by the key side's ones in the extra contraction step, the accumulator holds q.k - lse / scale
+          // and the epilogue needs no per-row operand at all.
+          const float inv = 1.0f / p.scale2;
+          const float* src = p.lse2 + (int64_t)u * p.rs;
+          for (int r = lane; r < p.n16; r += 32) {
+            const float v = src[r] * inv;
+            const float hi = __bfloat162float(__float2bfloat16_rn(v));
+            const float mid = __bfloat162float(__float2bfloat16_rn(v - hi));
+            const float low = __bfloat162float(__float2bfloat16_rn((v - hi) - mid));
+            const uint32_t w0 = (__float_as_uint(hi) >> 16) | (__float_as_uint(mid) & 0xffff0000u);
+            *reinterpret_cast<uint4*>(shift_s + r * 128 + (r & 7) * 16) = make_uint4(w0, __float_as_uint(low) >> 16, 0u, 0u);
           }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();  // every lane's rows are written (and fenced) before lane 0 signals the unit ready
+        }
+        if (lane == 0) {
           mbar_expect_tx(qfull, (uint32_t)(p.R * 128 * kKBlocks));
           for (int kb = 0; kb < kKBlocks; ++kb)
             tma_load_5d(q_s + kb * 256 * 128, &tmap_q, qfull, kb * 64, 0, h * p.g, l, b, pol_q);
         }
+      }
+      if (lane == 0) {
         for (int t = 0; t < tiles; ++t) {
           ok = mbar_wait(&empty[stage], stage_par ^ 1, abort_flag, p.status, kSiteStage);
           if (!ok) break;
@@ -287,10 +291,11 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
           }
         }
       }
-      if (!ok) {  // abandoned: give copies in flight time to land before the CTA's shared memory goes away
-        const long long t0 = clock64();
-        while (clock64() - t0 < 2000000ll) __nanosleep(1000);
-      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+    }
+    if (!ok && lane == 0) {  // abandoned: give copies in flight time to land before the CTA's shared memory goes away
+      const long long t0 = clock64();
+      while (clock64() - t0 < 2000000ll) __nanosleep(1000);
     }
   } else if (warp == 1) {
     // ================================================================ MMA issuer
