@@ -83,6 +83,128 @@ __device__ __forceinline__ uint64_t exp2_sum16(const uint64_t (&x)[8]) {
   return add2(add2(add2(e[0], e[1]), add2(e[2], e[3])), add2(add2(e[4], e[5]), add2(e[6], e[7])));
 }
 
+__device__ __forceinline__ float sum4(const uint64_t (&a)[4]) {
+  float lo, hi;
+  unpack2(add2(add2(a[0], a[1]), add2(a[2], a[3])), lo, hi);
+  return lo + hi;
+}
+__device__ __forceinline__ float block_max16(const uint32_t (&r)[16]) {
+  const float a0 = max3f(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
+  const float a1 = max3f(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
+  const float a2 = max3f(__uint_as_float(r[6]), __uint_as_float(r[7]), __uint_as_float(r[8]));
+  const float a3 = max3f(__uint_as_float(r[9]), __uint_as_float(r[10]), __uint_as_float(r[11]));
+  const float a4 = max3f(__uint_as_float(r[12]), __uint_as_float(r[13]), __uint_as_float(r[14]));
+  return max3f(max3f(a0, a1, a2), a3, fmaxf(a4, __uint_as_float(r[15])));
+}
+
+// A tile's NB blocks of 16 accumulator columns of this thread's TMEM lane, none of them masked, as a software
+// pipeline over steps of 8 columns: the exponentials of step s are queued on the special-function unit, then the
+// results of step s - 1 are added up and the inputs of step s + 1 prepared, so that a warp on its own keeps the unit
+// supplied (with the steps one after the other a lone warp kept it half busy, and at the end of every tile the
+// last warps of a scheduler are on their own). The TMEM load of block j + 1 is in flight during block j.
+//
+// Pass 2: acc += exp2(scale2 * column); the accumulator already holds q.k - lse / scale.
+template <int NB>
+__device__ __forceinline__ void psi_tile(uint32_t taddr, uint64_t sc2, uint64_t (&acc)[4]) {
+  uint32_t r[2][16];
+  uint64_t x[2][4], e[2][4];
+  tmem_ld16_issue(taddr, r[0]);
+  tmem_ld_wait16(r[0]);
+  if (NB > 1) tmem_ld16_issue(taddr + 16, r[1]);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) x[0][i] = mul2(pack2u(r[0][2 * i], r[0][2 * i + 1]), sc2);
+#pragma unroll
+  for (int s = 0; s < 2 * NB; ++s) {
+    const int cur = s & 1, nxt = cur ^ 1;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float lo, hi;
+      unpack2(x[cur][i], lo, hi);
+      e[cur][i] = pack2(ex2(lo), ex2(hi));
+    }
+    if (s > 0) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[i] = add2(acc[i], e[nxt][i]);
+    }
+    if (s + 1 < 2 * NB) {
+      const int blk = (s + 1) >> 1, half = (s + 1) & 1, b = blk & 1;
+      if (half == 0) {
+        tmem_ld_wait16(r[b]);
+        if (blk + 1 < NB) tmem_ld16_issue(taddr + (blk + 1) * 16, r[b ^ 1]);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) x[nxt][i] = mul2(pack2u(r[b][8 * half + 2 * i], r[b][8 * half + 2 * i + 1]), sc2);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) acc[i] = add2(acc[i], e[(2 * NB - 1) & 1][i]);
+}
+
+// Pass 1: the row's running maximum m (log2 domain) is checked once per block; it rarely grows once a few hundred
+// keys have been seen, so the rescaling sits behind a warp-uniform branch. acc holds the sum of exp2(scale2 * s - m)
+// of the item at hand, z_run that of the run's earlier items.
+template <int NB>
+__device__ __forceinline__ void stat_tile(uint32_t taddr, float scale2, uint64_t sc2, float& m, uint64_t (&acc)[4],
+                                          float& z_run) {
+  uint32_t r[2][16];
+  uint64_t x[2][4], e[2][4];
+  auto grow = [&](float bm) {
+    const float mn = fmaxf(m, bm);
+    const float f = ex2(m - mn);
+    const uint64_t f2 = pack2(f, f);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] = mul2(acc[i], f2);
+    z_run *= f;
+    m = mn;
+  };
+  tmem_ld16_issue(taddr, r[0]);
+  tmem_ld_wait16(r[0]);
+  if (NB > 1) tmem_ld16_issue(taddr + 16, r[1]);
+  {
+    const float bm = block_max16(r[0]) * scale2;
+    if (__any_sync(0xffffffffu, bm > m)) grow(bm);
+  }
+  uint64_t nm2 = pack2(-m, -m);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) x[0][i] = fma2(pack2u(r[0][2 * i], r[0][2 * i + 1]), sc2, nm2);
+#pragma unroll
+  for (int s = 0; s < 2 * NB; ++s) {
+    const int cur = s & 1, nxt = cur ^ 1;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float lo, hi;
+      unpack2(x[cur][i], lo, hi);
+      e[cur][i] = pack2(ex2(lo), ex2(hi));
+    }
+    if (s > 0) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[i] = add2(acc[i], e[nxt][i]);
+    }
+    if (s + 1 < 2 * NB) {
+      const int blk = (s + 1) >> 1, half = (s + 1) & 1, b = blk & 1;
+      if (half == 0) {
+        tmem_ld_wait16(r[b]);
+        if (blk + 1 < NB) tmem_ld16_issue(taddr + (blk + 1) * 16, r[b ^ 1]);
+        const float bm = block_max16(r[b]) * scale2;
+        if (__any_sync(0xffffffffu, bm > m)) {
+          // the exponentials just queued were taken against the old maximum: they go in before the rescaling
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            acc[i] = add2(acc[i], e[cur][i]);
+            e[cur][i] = 0ull;
+          }
+          grow(bm);
+          nm2 = pack2(-m, -m);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) x[nxt][i] = fma2(pack2u(r[b][8 * half + 2 * i], r[b][8 * half + 2 * i + 1]), sc2, nm2);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) acc[i] = add2(acc[i], e[(2 * NB - 1) & 1][i]);
+}
+
 // The CTA's share of the work: a contiguous range of the non-empty work items in (sequence, layer, KV head, split)
 // order. cursor = (sequence b, index r among the items of b); a sequence of n keys has L * Hkv * ceil(n / 2048) items.
 struct ItemCursor {
@@ -386,7 +508,8 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     // logit. The sum is kept on two levels (the item at hand, the run's earlier items): one accumulator over a whole
     // long sequence would lose the small terms to rounding.
     const int row = mb * 128 + quarter * 32 + lane;
-    float m = 4.f * kEmptyMax, z = 0.f, z_run = 0.f;
+    float m = 4.f * kEmptyMax, z_run = 0.f;
+    uint64_t zacc[4] = {0ull, 0ull, 0ull, 0ull};  // pass 1: the item's sum, as four packed partial sums
     float* xslot = xch + quarter * 32 + lane;  // pass 2: [buffer][share - 1][128 keys]
 
     for (ItemCursor c = cursor_begin(); ok && c.left > 0; cursor_next(c)) {
@@ -399,7 +522,7 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         m = 4.f * kEmptyMax;
         z_run = 0.f;
       }
-      z = 0.f;
+      zacc[0] = zacc[1] = zacc[2] = zacc[3] = 0ull;
       int vis = 0;  // pass 1: keys the row may see: [0, vis)
       if (PASS == 1 && row < p.R) {
         const int pos = n - p.w + row % p.w;
@@ -412,10 +535,10 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         tc_fence_after();
         const int key0 = key_begin + t * kTileKeys;
         const uint32_t taddr = tlane + buf * 256;
+        uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};  // pass 2: the key's sum over this warp's window rows
+        const int key = key0 + quarter * 32 + lane;  // pass 2: the thread's key
+        const bool plain = key0 + kTileKeys <= n - p.w;  // every row sees the whole tile: nothing to mask
         uint32_t ra[16], rb[16];
-        uint64_t acc = 0ull;  // pass 2: the key's sum over this warp's window rows
-        const int key = key0 + quarter * 32 + lane;                // pass 2: the thread's key
-        const bool plain = key0 + kTileKeys <= n - p.w;            // pass 2: every row sees the whole tile
         auto block = [&](uint32_t (&r)[16], int j) {  // block blk0 + j of the accumulator
           if (PASS == 1) {
             const int col0 = key0 + 16 * (blk0 + j);  // first key of the block
@@ -424,27 +547,21 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
               for (int i = 0; i < 16; ++i)
                 if (col0 + i >= vis) r[i] = __float_as_uint(kEmptyMax);
             }
-            const float a0 = max3f(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
-            const float a1 = max3f(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
-            const float a2 = max3f(__uint_as_float(r[6]), __uint_as_float(r[7]), __uint_as_float(r[8]));
-            const float a3 = max3f(__uint_as_float(r[9]), __uint_as_float(r[10]), __uint_as_float(r[11]));
-            const float a4 = max3f(__uint_as_float(r[12]), __uint_as_float(r[13]), __uint_as_float(r[14]));
-            const float bm = max3f(max3f(a0, a1, a2), a3, fmaxf(a4, __uint_as_float(r[15]))) * p.scale2;
-            // the running maximum rarely grows once a few hundred keys have been seen; the rescaling (one more
-            // exponential) is predicated on it
-            if (bm > m) {
-              const float f = ex2(m - bm);
-              z *= f;
+            const float bm = block_max16(r) * p.scale2;
+            if (__any_sync(0xffffffffu, bm > m)) {
+              const float mn = fmaxf(m, bm);
+              const float f = ex2(m - mn);
+              const uint64_t f2 = pack2(f, f);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) zacc[i] = mul2(zacc[i], f2);
               z_run *= f;
-              m = bm;
+              m = mn;
             }
             const uint64_t nm2 = pack2(-m, -m);
             uint64_t x[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) x[i] = fma2(pack2u(r[2 * i], r[2 * i + 1]), sc2, nm2);
-            float lo, hi;
-            unpack2(exp2_sum16(x), lo, hi);
-            z += lo + hi;
+            zacc[0] = add2(zacc[0], exp2_sum16(x));
           } else {
             if (!plain) {  // the tiles at the window: every logit is checked against what its row may see
 #pragma unroll
@@ -457,10 +574,23 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
             uint64_t x[8];  // the accumulator already holds q.k - lse / scale
 #pragma unroll
             for (int i = 0; i < 8; ++i) x[i] = mul2(pack2u(r[2 * i], r[2 * i + 1]), sc2);
-            acc = add2(acc, exp2_sum16(x));
+            acc[0] = add2(acc[0], exp2_sum16(x));
           }
         };
-        if (nblk > 0) {
+        if (plain) {  // all but the tiles at the window
+          if (PASS == 1) {
+            if (nblk == 4) stat_tile<4>(taddr, p.scale2, sc2, m, zacc, z_run);
+            else stat_tile<2>(taddr, p.scale2, sc2, m, zacc, z_run);
+          } else {
+            switch (nblk) {
+              case 4: psi_tile<4>(taddr, sc2, acc); break;
+              case 3: psi_tile<3>(taddr, sc2, acc); break;
+              case 2: psi_tile<2>(taddr, sc2, acc); break;
+              case 1: psi_tile<1>(taddr, sc2, acc); break;
+              default: break;
+            }
+          }
+        } else if (nblk > 0) {
           tmem_ld16_issue(taddr, ra);
 #pragma unroll 1
           for (int j = 0; j < nblk; j += 2) {
@@ -479,9 +609,7 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         if (PASS == 2) {
           // the four warps that share the key add up in a fixed order: shares 1-3 hand their sums to share 0 (a
           // slot is free once share 0 has taken the tile before last)
-          float lo, hi;
-          unpack2(acc, lo, hi);
-          float total = lo + hi;
+          float total = sum4(acc);
           const uint32_t xp = (uint32_t)(n_tile >> 1) & 1u;
           if (share) {
             ok = __all_sync(0xffffffffu, mbar_wait(&xempty[buf * 4 + quarter], xp ^ 1, abort_flag, p.status, kSiteFlag));
@@ -499,7 +627,7 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
       }
       if (!ok) break;
       if (PASS == 1) {
-        z_run += z;
+        z_run += sum4(zacc);
         if (row < p.R && tiles > 0) {
           // the pair goes out with the last item of the run (the next item is another unit's, holds no keys, or does
           // not exist); the run's other items leave an empty pair so that the merge finds every split that holds keys
