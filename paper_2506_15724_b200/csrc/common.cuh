@@ -35,7 +35,7 @@ struct WsHeader {
 static_assert(sizeof(WsHeader) == kHeaderBytes, "header size");
 
 struct WsLayout {
-  size_t seq_nv_off, score_done_off, score_lse_off, score_part_off, decode_off, total;
+  size_t seq_nv_off, score_done_off, score_lse_off, score_part_off, decode_off, decode_len_off, total;
   int score_chunks, score_tc_chunks, decode_splits;
 };
 
@@ -72,6 +72,8 @@ inline WsLayout ws_layout(const madakv_config& c) {
   w.decode_off = off;
   off = align_up(off + (size_t)c.batch * c.n_layers * c.n_q_heads * (size_t)w.decode_splits * (c.head_dim + 2) *
                            sizeof(float), 256);
+  w.decode_len_off = off;  // rows each segment's attention covered in an appending decode call
+  off = align_up(off + units * sizeof(int32_t), 256);
   w.total = off;
   return w;
 }

@@ -1,6 +1,7 @@
 // Stage 5: cache append (Eq. 4) and decode attention over the ragged per-head cache (Eq. 5).
 //
-//   append   copies k_new / v_new behind every segment of the layer(s) and bumps kept_len
+//   append   (Eq. 4) has no kernel of its own: the partial block whose share holds the new row copies it from
+//            k_new / v_new behind the segment and attends over it; the merge kernel bumps kept_len
 //   partial  up to kDecodeSlots blocks per segment, each taking an equal share of the segment's rows (the share is a
 //            function of the segment's length alone: short segments use fewer blocks, never fewer than kDecodeMinRows
 //            rows each): a group of LPR lanes owns a cache row (16 bytes per lane), the g query heads of the KV group
@@ -34,6 +35,7 @@ struct DecodeParams {
   void* out;
   float* lse_out;
   float* part;  // ws: [B*L*Hq, slots, D + 2]
+  int32_t* eff_len;  // ws: [units] rows each segment's attention covered (appending calls; else null)
   void* ws;
   int L, Hq, Hkv, g, layer, slots, n_sel, min_rows, slot_fast;
   float scale2;
@@ -77,25 +79,41 @@ __device__ __forceinline__ void block_rows(const DecodeParams& p, int len, int x
   row_end = min(len, row_begin + share);
 }
 
-template <int ROW_BYTES>
-__global__ void append_kernel(DecodeParams p, int n_sel) {
-  constexpr int LPR = ROW_BYTES / 16;
-  const int x = blockIdx.x * blockDim.x + threadIdx.x;
-  const int y = x / LPR, lane = x % LPR;
-  if (y >= n_sel) return;
-  const int u = unit_of(p, y);
-  const int len = p.kept_len[u];
-  const int64_t row = p.seg_off[u] + len;
-  if (segment_refused(p, u) || len < 0 || row + 1 > p.seg_off[u + 1]) {
-    if (lane == 0) set_status(p.ws, MADAKV_ECAPACITY);
-    return;
+// What a block of unit u works on. When the call appends (Eq. 4), the new row is part of the attention: the one block
+// whose share holds it copies it from k_new / v_new into the cache and reads it from there, all others see the old
+// rows only. kept_len itself is bumped by the merge kernel, after every block of both kernels has read the old value
+// (merge blocks read the length the partial kernel recorded in the workspace instead). A segment without room for the
+// row (or one that selection refused) is left as it is and MADAKV_ECAPACITY is recorded.
+struct SegView {
+  int len;      // rows attention covers, the appended one included
+  int new_row;  // its index in the segment, or -1
+};
+__device__ __forceinline__ SegView segment_view(const DecodeParams& p, int u, bool reporter) {
+  SegView v;
+  v.len = segment_rows(p, u);
+  v.new_row = -1;
+  if (p.k_new) {
+    const int len = p.kept_len[u];
+    if (segment_refused(p, u) || len < 0 || p.seg_off[u] + (int64_t)len + 1 > p.seg_off[u + 1]) {
+      if (reporter) set_status(p.ws, MADAKV_ECAPACITY);
+    } else {
+      v.new_row = len;
+      v.len = len + 1;
+    }
   }
-  const uint4 kv = *reinterpret_cast<const uint4*>((const char*)p.k_new + (int64_t)u * ROW_BYTES + lane * 16);
-  const uint4 vv = *reinterpret_cast<const uint4*>((const char*)p.v_new + (int64_t)u * ROW_BYTES + lane * 16);
-  *reinterpret_cast<uint4*>((char*)p.k_c + row * ROW_BYTES + lane * 16) = kv;
-  *reinterpret_cast<uint4*>((char*)p.v_c + row * ROW_BYTES + lane * 16) = vv;
-  __syncwarp(__activemask());
-  if (lane == 0) p.kept_len[u] = len + 1;
+  return v;
+}
+// The owner of the appended row (the block whose rows include it) stores it into the cache.
+template <int ROW_BYTES>
+__device__ __forceinline__ void store_new_row(const DecodeParams& p, int u, int64_t off, const SegView& v, int row_begin,
+                                              int row_end) {
+  constexpr int LPR = ROW_BYTES / 16;
+  if (v.new_row < row_begin || v.new_row >= row_end || (int)threadIdx.x >= LPR) return;
+  const int64_t row = off + v.new_row;
+  const uint4 kv = *reinterpret_cast<const uint4*>((const char*)p.k_new + (int64_t)u * ROW_BYTES + threadIdx.x * 16);
+  const uint4 vv = *reinterpret_cast<const uint4*>((const char*)p.v_new + (int64_t)u * ROW_BYTES + threadIdx.x * 16);
+  *reinterpret_cast<uint4*>((char*)p.k_c + row * ROW_BYTES + threadIdx.x * 16) = kv;
+  *reinterpret_cast<uint4*>((char*)p.v_c + row * ROW_BYTES + threadIdx.x * 16) = vv;
 }
 
 template <typename T>
@@ -134,13 +152,17 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
   __shared__ float s_o[GROUPS][G][D];
   __shared__ float s_m[GROUPS][G], s_l[GROUPS][G];
 
-  const int u = unit_of(p, p.slot_fast ? blockIdx.x / p.slots : blockIdx.x % p.n_sel);
-  const int len = segment_rows(p, u);
+  const int y = p.slot_fast ? blockIdx.x / p.slots : blockIdx.x % p.n_sel;
+  const int u = unit_of(p, y);
   const int slot = p.slot_fast ? blockIdx.x % p.slots : blockIdx.x / p.n_sel;
+  const SegView view = segment_view(p, u, slot == 0 && threadIdx.x == 0);
+  const int len = view.len;
+  if (slot == 0 && threadIdx.x == 0 && p.eff_len) p.eff_len[u] = len;
   if (slot >= segment_blocks(p, len)) return;
   int row_begin, row_end;
   block_rows(p, len, slot, row_begin, row_end);
   const int64_t off = p.seg_off[u];
+  store_new_row<ROW_BYTES>(p, u, off, view, row_begin, row_end);
   const int h = u % p.Hkv, bl = u / p.Hkv;
   const int lane = threadIdx.x % LPR, grp = threadIdx.x / LPR;
 
@@ -165,6 +187,9 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
   }
   const char* kc = (const char*)p.k_c + off * ROW_BYTES + lane * 16;
   const char* vc = (const char*)p.v_c + off * ROW_BYTES + lane * 16;
+  // the appended row is read from where it comes from, not from the cache row this block is writing
+  const char* kn = view.new_row >= 0 ? (const char*)p.k_new + (int64_t)u * ROW_BYTES + lane * 16 : nullptr;
+  const char* vn = view.new_row >= 0 ? (const char*)p.v_new + (int64_t)u * ROW_BYTES + lane * 16 : nullptr;
   // U rows per thread are in flight at a time: all their 16-byte K and V loads are issued before the first use, so a
   // block keeps GROUPS * U * 2 * ROW_BYTES bytes on the wire (the online-softmax chain below is short next to the
   // memory latency). Uniform trip count: the shuffles need full warps.
@@ -176,8 +201,9 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
       const int r = r0 + grp + GROUPS * j;
       kraw[j] = vraw[j] = make_uint4(0u, 0u, 0u, 0u);
       if (r < row_end) {
-        kraw[j] = __ldcs(reinterpret_cast<const uint4*>(kc + (int64_t)r * ROW_BYTES));
-        vraw[j] = __ldcs(reinterpret_cast<const uint4*>(vc + (int64_t)r * ROW_BYTES));
+        const bool fresh = r == view.new_row;
+        kraw[j] = __ldcs(reinterpret_cast<const uint4*>(fresh ? kn : kc + (int64_t)r * ROW_BYTES));
+        vraw[j] = __ldcs(reinterpret_cast<const uint4*>(fresh ? vn : vc + (int64_t)r * ROW_BYTES));
       }
     }
 #pragma unroll
@@ -316,12 +342,15 @@ __global__ void __launch_bounds__(kMmaWarps * 32, 3) decode_partial_mma_kernel(D
   extern __shared__ __align__(16) unsigned char dsmem[];
 
   const int u = unit_of(p, p.slot_fast ? blockIdx.x / p.slots : blockIdx.x % p.n_sel);
-  const int len = segment_rows(p, u);
   const int slot = p.slot_fast ? blockIdx.x % p.slots : blockIdx.x / p.n_sel;
+  const SegView view = segment_view(p, u, slot == 0 && threadIdx.x == 0);
+  const int len = view.len;
+  if (slot == 0 && threadIdx.x == 0 && p.eff_len) p.eff_len[u] = len;
   if (slot >= segment_blocks(p, len)) return;
   int row_begin, row_end;
   block_rows(p, len, slot, row_begin, row_end);
   const int64_t off = p.seg_off[u];
+  store_new_row<D * 2>(p, u, off, view, row_begin, row_end);
   const int h = u % p.Hkv, bl = u / p.Hkv;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int hr = lane / 4, t = lane % 4;  // fragment coordinates: row (head) hr and hr + 8, column pair t
@@ -343,6 +372,8 @@ __global__ void __launch_bounds__(kMmaWarps * 32, 3) decode_partial_mma_kernel(D
   }
   const char* kc = (const char*)p.k_c + off * ROW_BYTES;
   const char* vc = (const char*)p.v_c + off * ROW_BYTES;
+  const char* kn = view.new_row >= 0 ? (const char*)p.k_new + (int64_t)u * ROW_BYTES : nullptr;
+  const char* vn = view.new_row >= 0 ? (const char*)p.v_new + (int64_t)u * ROW_BYTES : nullptr;
   // per-lane shared-memory offsets of the matrix loads: lanes 8i..8i+7 address the rows of the i-th 8x8 matrix
   const int mi = lane / 8, mr = lane % 8;
   const uint32_t k_lane = ((mi >> 1) * 8 + mr) * MT::PITCH + (mi & 1) * 16;  // keys (mi/2)*8.., d half mi%2
@@ -361,8 +392,10 @@ __global__ void __launch_bounds__(kMmaWarps * 32, 3) decode_partial_mma_kernel(D
         const int rr = x / LPR, cc = x % LPR;
         const bool valid = r + rr < row_end;
         const int64_t src = (int64_t)(valid ? r + rr : r) * ROW_BYTES + cc * 16;  // row r itself is always valid
-        cp_async16(kd + rr * MT::PITCH + cc * 16, kc + src, valid);
-        cp_async16(vd + rr * MT::PITCH + cc * 16, vc + src, valid);
+        // (the appended row comes from k_new / v_new, not from the cache row this block is writing)
+        const bool fresh = valid && r + rr == view.new_row;
+        cp_async16(kd + rr * MT::PITCH + cc * 16, fresh ? kn + cc * 16 : kc + src, valid);
+        cp_async16(vd + rr * MT::PITCH + cc * 16, fresh ? vn + cc * 16 : vc + src, valid);
       }
     };
     if (row_begin + 16 * warp < row_end) load_chunk(row_begin + 16 * warp, 0);
@@ -488,7 +521,9 @@ __global__ void __launch_bounds__(D) decode_merge_kernel(DecodeParams p) {
   }
   const int bl = row / p.Hq, hq = row % p.Hq;
   const int u = bl * p.Hkv + hq / p.g;
-  const int len = segment_rows(p, u);
+  // an appending call: the length the partial kernel worked with; the first head of the group makes it the segment's
+  const int len = p.eff_len ? p.eff_len[u] : segment_rows(p, u);
+  if (p.eff_len && hq % p.g == 0 && threadIdx.x == 0 && len > p.kept_len[u]) p.kept_len[u] = len;
   const int used = segment_blocks(p, len);
   const float* part = p.part + (int64_t)row * p.slots * (D + 2);
   const int c = threadIdx.x;
@@ -523,17 +558,13 @@ int slot_order(int n_sel) {
 template <typename T, int D>
 int run(const DecodeParams& p, const madakv_config&, cudaStream_t st) {
   const int n_sel = p.n_sel;
-  // every host-side refusal comes before the first launch (the append below changes the cache)
+  // every host-side refusal comes before the first launch (an appending call changes the cache)
   const bool mma = sizeof(T) == 2 && p.g >= 3 && p.g <= 16;
   if (!mma && p.g > 8) return MADAKV_EUNSUPPORTED;
   if constexpr (sizeof(T) == 2) {
     if (mma && cudaFuncSetAttribute(decode_partial_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     MmaTile<D>::BYTES) != cudaSuccess)
       return MADAKV_ECUDA;
-  }
-  if (p.k_new) {
-    constexpr int LPR = D * (int)sizeof(T) / 16;
-    append_kernel<D * (int)sizeof(T)><<<(n_sel * LPR + 127) / 128, 128, 0, st>>>(p, n_sel);
   }
   const dim3 grid((unsigned)n_sel * p.slots);  // one dimension: no 65535 limit on the number of segments
   if constexpr (sizeof(T) == 2) {
@@ -566,6 +597,7 @@ int launch_decode(const madakv_config& c, int layer, const void* q, const void* 
   p.out = out;
   p.lse_out = lse_out;
   p.part = reinterpret_cast<float*>((char*)ws + wl.decode_off);
+  p.eff_len = k_new ? reinterpret_cast<int32_t*>((char*)ws + wl.decode_len_off) : nullptr;
   p.ws = ws;
   p.L = c.n_layers;
   p.Hq = c.n_q_heads;
@@ -650,7 +682,8 @@ extern "C" int madakv_decode_attn_static(const madakv_config* cfg, int32_t layer
   p.out = out;
   p.lse_out = lse_out;
   p.part = reinterpret_cast<float*>(scratch);
-  p.ws = nullptr;  // only the append kernel reports through the workspace
+  p.eff_len = nullptr;
+  p.ws = nullptr;  // only an appending call reports through the workspace
   p.L = c.n_layers;
   p.Hq = c.n_q_heads;
   p.Hkv = c.n_kv_heads;
