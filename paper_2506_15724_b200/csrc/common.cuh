@@ -41,6 +41,20 @@ struct WsLayout {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Wide-window scoring: its two passes run on at most kWideMaxGrid CTAs, each taking a contiguous, equally long range
+// of the 128-key tiles of all units; pass 1 leaves one partial per (unit, CTA that holds tiles of it). A unit of t
+// tiles meets at most ceil(t / floor(T / G)) + 1 of the G ranges (T tiles in all), and T >= L * Hkv * t, which
+// gives the bound below whatever the lengths in the batch are.
+constexpr int kWideMaxGrid = 160;
+inline int wide_max_runs(const madakv_config& c) {
+  const long long lh = (long long)c.n_layers * c.n_kv_heads;
+  long long runs = (2ll * kWideMaxGrid + lh - 1) / lh + 1;
+  const long long tiles = (c.max_seq_len + 127) / 128;
+  if (runs > kWideMaxGrid) runs = kWideMaxGrid;
+  if (runs > tiles) runs = tiles;
+  return (int)(runs < 1 ? 1 : runs);
+}
+
 inline WsLayout ws_layout(const madakv_config& c) {
   WsLayout w;
   const size_t units = (size_t)c.batch * c.n_layers * c.n_kv_heads;
@@ -63,9 +77,8 @@ inline WsLayout ws_layout(const madakv_config& c) {
   if (rows <= 64) {
     const size_t tc = units * rows_pad * (size_t)w.score_tc_chunks * 4 * sizeof(float2);
     part = tc > part ? tc : part;
-  } else if (rows <= 256) {  // wide-window path: per 2048-key split and padded row one pair for each column share
-    const size_t splits = ((size_t)c.max_seq_len + 2047) / 2048;
-    const size_t wide = units * splits * (rows <= 128 ? 4 : 2) * rows_pad * sizeof(float2);
+  } else if (rows <= 256) {  // wide-window path: per run of a unit and padded row one pair for each column share
+    const size_t wide = units * (size_t)wide_max_runs(c) * (rows <= 128 ? 4 : 2) * rows_pad * sizeof(float2);
     part = wide > part ? wide : part;
   }
   off = align_up(off + part, 256);

@@ -8,8 +8,8 @@
 // busy.
 //   pass 1  window rows on M (one or two blocks of 128 rows), the 128 keys of a tile on N: an epilogue thread owns
 //           ONE window row (a TMEM lane) and a share of the tile's columns and keeps a running (max, sum of exp2) of
-//           its row in registers, carried from tile to tile and from work item to work item for as long as the CTA
-//           stays with the same unit; one (max, sum) pair per row, column share and run goes to the workspace
+//           its row in registers, carried from tile to tile for as long as the CTA stays with the unit; one (max,
+//           sum) pair per row, column share and run goes to the workspace
 //   merge   per (unit, row): all pairs -> the row's log-sum-exp (a separate small kernel)
 //   pass 2  the tile turned back (128 keys on M, the window rows on N): a thread owns one key and a quarter of the
 //           window rows, and psi(i) = sum over rows of exp2(s - lse) is an in-thread sum over columns of its TMEM lane.
@@ -21,27 +21,30 @@
 //           fixed order.
 // In both passes all 16 epilogue warps work on the same tile while the MMAs of the next tile fill the other half of
 // the TMEM; the TMEM load of a warp's next 16 columns is in flight while it works on the present ones.
-// K is streamed twice. The passes are separate launches and no CTA ever waits for another CTA. Work items are
-// (unit, 2048 keys); a CTA takes a contiguous range of the non-empty items (equal counts, so ragged batches stay
-// balanced), which makes consecutive items share their unit: queries and log-sum-exps are reloaded only when the
-// unit changes. Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-17 epilogue; TMEM lane
-// quarter = warp % 4 throughout. Every wait is bounded: on expiry the kernel records MADAKV_ETIMEOUT, drains and returns.
+// K is streamed twice. The passes are separate launches and no CTA ever waits for another CTA. The work is the list
+// of all 128-key tiles in (sequence, layer, KV head, tile) order; a CTA takes a contiguous range of it, the same
+// number of tiles to within one for every CTA whatever the lengths in the batch. The part of a unit inside a CTA's
+// range is a run: queries and log-sum-exps are loaded once per run, and pass 1 leaves one pair per run, so a unit's
+// statistics come in as many pieces as CTAs share it (two or three for long sequences). Warp roles: warp 0 TMA
+// producer, warp 1 MMA issuer and TMEM owner, warps 2-17 epilogue; TMEM lane quarter = warp % 4 throughout. Every wait is bounded: on expiry the kernel records MADAKV_ETIMEOUT, drains and returns.
 #include "tc_common.cuh"
 
 namespace madakv {
 namespace {
 
 constexpr int kRowThreads = 576;  // 2 + 16 warps
-constexpr int kSplitKeys = 2048;  // keys per work item (16 tiles)
-constexpr int kMaxSeqScan = 1024; // batches up to this size get the exact (ragged-aware) item partition
+constexpr int kMaxSeqScan = 1024; // batches up to this size get the exact (ragged-aware) tile partition
+constexpr int kFoldTiles = 16;    // pass 1 moves a row's sum to its second level every this many tiles
 
 struct RowParams {
   const int32_t* seq_len;
   float* psi;        // [units, n_max]
-  float2* part;      // ws: [units, splits, cparts, rs] (max, sum) of every row over a column share of a run of items
+  float2* part;      // ws: [units, smax, cparts, rs] (max, sum) of every row over a column share of one CTA's run
   const float* lse2; // ws: [units, rs] NEGATED log2-domain log-sum-exp, padding rows hold kEmptyMax (pass 2)
   int32_t* status;   // ws header
-  int B, units, L, Hq, Hkv, g, w, R, n_max, causal, splits, rs, mblocks, cparts, n16;  // n16: R rounded up to 16
+  int B, units, L, Hq, Hkv, g, w, R, n_max, causal, rs, mblocks, cparts, n16;  // n16: R rounded up to 16
+  int smax;          // runs (CTAs) a unit's tiles can be spread over at most: wide_max_runs()
+  int grid;          // CTAs of the two passes (the merge kernel needs the partition)
   float scale2;
 };
 
@@ -60,7 +63,7 @@ struct RowSmem {
   // full[kStages], empty[kStages], qfull, qempty, tfull[2], tempty[2], drain, xfull[8], xempty[8]
   static constexpr int kNumBars = 2 * kStages + 2 + 4 + 1 + 16;
   static constexpr int kMiscOff = (kBarOff + kNumBars * 8 + 15) / 16 * 16;
-  static constexpr int kColOff = kMiscOff + 32;            // window position (row % w) of every row [256]
+  static constexpr int kColOff = kMiscOff + 48;            // window position (row % w) of every row [256]
   static constexpr int kXchOff = kColOff + 256 * 4;        // pass 2: partial psi of column shares 1-3 [2][3][128]
   static constexpr int kTotal = kXchOff + 6 * 128 * 4;
   static constexpr int kAlloc = kTotal + 1024;
@@ -205,17 +208,29 @@ __device__ __forceinline__ void stat_tile(uint32_t taddr, float scale2, uint64_t
   for (int i = 0; i < 4; ++i) acc[i] = add2(acc[i], e[(2 * NB - 1) & 1][i]);
 }
 
-// The CTA's share of the work: a contiguous range of the non-empty work items in (sequence, layer, KV head, split)
-// order. cursor = (sequence b, index r among the items of b); a sequence of n keys has L * Hkv * ceil(n / 2048) items.
-struct ItemCursor {
-  int b, r, per_b, s_b, left;  // per_b: items of sequence b; s_b: splits of sequence b; left: items still to do
+// The CTA's share of the work: a contiguous range of the 128-key tiles of all units, in (sequence, layer, KV head,
+// tile) order, cut at tile granularity (every CTA gets the same number of tiles to within one, whatever the batch's
+// length mix). The part of one unit inside a CTA's range is a run: the queries are loaded once per run, and pass 1
+// leaves one (max, sum) pair per run, row and column share. Sequence b has L * Hkv * tiles_of(b) tiles.
+struct TileCursor {
+  int b;        // sequence
+  int r;        // index among the tiles of sequence b
+  int tb;       // tiles per unit of sequence b
+  int per_b;    // tiles of sequence b
+  int left;     // tiles of the range still to do
+  int done;     // tiles of the range already done
+};
+struct Run {
+  int u, b, n;  // unit, its sequence and that sequence's length
+  int t0, cnt;  // first tile of the run within the unit, tiles in the run (what the partition counts)
+  int tiles;    // tiles of the run that hold keys (fewer than cnt only in the uniform partition of very large batches)
 };
 
-__device__ __forceinline__ int splits_of(const RowParams& p, int b) {
-  return (clamped_len(p.seq_len, b, p.n_max) + kSplitKeys - 1) / kSplitKeys;
+__device__ __forceinline__ int tiles_of(const RowParams& p, int b, bool exact) {
+  return ((exact ? clamped_len(p.seq_len, b, p.n_max) : p.n_max) + kTileKeys - 1) / kTileKeys;
 }
-__device__ __forceinline__ void cursor_settle(const RowParams& p, ItemCursor& c, bool exact) {
-  // move on to the next sequence that has items
+__device__ __forceinline__ void cursor_settle(const RowParams& p, TileCursor& c, bool exact) {
+  // move on to the next sequence that has tiles
   while (c.left > 0 && c.r >= c.per_b) {
     c.r -= c.per_b;
     ++c.b;
@@ -223,14 +238,34 @@ __device__ __forceinline__ void cursor_settle(const RowParams& p, ItemCursor& c,
       c.left = 0;
       break;
     }
-    c.s_b = exact ? splits_of(p, c.b) : p.splits;
-    c.per_b = p.L * p.Hkv * c.s_b;
+    c.tb = tiles_of(p, c.b, exact);
+    c.per_b = p.L * p.Hkv * c.tb;
   }
 }
-__device__ __forceinline__ void cursor_item(const RowParams& p, const ItemCursor& c, int& u, int& split) {
-  const int ub = c.r / c.s_b;
-  split = c.r - ub * c.s_b;
-  u = c.b * p.L * p.Hkv + ub;
+__device__ __forceinline__ Run cursor_run(const RowParams& p, const TileCursor& c) {
+  Run r;
+  const int ub = c.r / c.tb;
+  r.t0 = c.r - ub * c.tb;
+  r.cnt = min(c.tb - r.t0, c.left);
+  r.b = c.b;
+  r.u = c.b * p.L * p.Hkv + ub;
+  r.n = clamped_len(p.seq_len, c.b, p.n_max);
+  const int real = (r.n + kTileKeys - 1) / kTileKeys;  // tiles of the unit that hold keys
+  r.tiles = max(0, min(r.t0 + r.cnt, real) - r.t0);
+  return r;
+}
+__device__ __forceinline__ void cursor_advance(const RowParams& p, TileCursor& c, const Run& r, bool exact) {
+  c.r += r.cnt;
+  c.left -= r.cnt;
+  c.done += r.cnt;
+  cursor_settle(p, c, exact);
+}
+// The CTA whose range [total * c / grid, total * (c + 1) / grid) holds tile x of the global order.
+__device__ __forceinline__ int cta_of(long long total, int grid, long long x) {
+  int c = (int)(x * grid / total);
+  while (c + 1 < grid && total * (c + 1) / grid <= x) ++c;
+  while (c > 0 && total * c / grid > x) --c;
+  return c;
 }
 
 template <int D, int PASS>
@@ -257,7 +292,7 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   uint64_t* xempty = xfull + 8;        // [2][4]    pass 2: share 0 -> shares 1-3
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(smem + SL::kMiscOff);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::kMiscOff + 4);
-  int* range_s = reinterpret_cast<int*>(smem + SL::kMiscOff + 8);  // first sequence, index in it, item count, exact
+  int* range_s = reinterpret_cast<int*>(smem + SL::kMiscOff + 8);  // first sequence, tile in it, tiles, exact, lo, total, CTAs in use
   int* rowpos = reinterpret_cast<int*>(smem + SL::kColOff);
   float* xch = reinterpret_cast<float*>(smem + SL::kXchOff);
 
@@ -281,26 +316,30 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    // this CTA's range of work items
+    // this CTA's range of tiles
     const bool exact = p.B <= kMaxSeqScan;
     long long total = 0;
     if (exact) {
-      for (int b = 0; b < p.B; ++b) total += (long long)p.L * p.Hkv * splits_of(p, b);
+      for (int b = 0; b < p.B; ++b) total += (long long)p.L * p.Hkv * tiles_of(p, b, true);
     } else {
-      total = (long long)p.units * p.splits;
+      total = (long long)p.units * tiles_of(p, 0, false);
     }
-    const long long lo = total * blockIdx.x / gridDim.x, hi = total * (blockIdx.x + 1) / gridDim.x;
+    // (a batch with fewer tiles than CTAs is spread over as many CTAs as it has tiles: no empty range lies between
+    // two CTAs that share a unit)
+    const long long ctas = total < (long long)gridDim.x ? total : (long long)gridDim.x;
+    const bool idle = (long long)blockIdx.x >= ctas;
+    const long long lo = idle ? total : total * blockIdx.x / ctas, hi = idle ? total : total * (blockIdx.x + 1) / ctas;
     int b0 = 0;
     long long r0 = lo;
     if (exact) {
       while (b0 < p.B) {
-        const long long per = (long long)p.L * p.Hkv * splits_of(p, b0);
+        const long long per = (long long)p.L * p.Hkv * tiles_of(p, b0, true);
         if (r0 < per) break;
         r0 -= per;
         ++b0;
       }
     } else {
-      const long long per = (long long)p.L * p.Hkv * p.splits;
+      const long long per = (long long)p.L * p.Hkv * tiles_of(p, 0, false);
       b0 = (int)(lo / per);
       r0 = lo - (long long)b0 * per;
     }
@@ -308,6 +347,9 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     range_s[1] = (int)r0;
     range_s[2] = (int)(hi - lo);
     range_s[3] = exact ? 1 : 0;
+    range_s[4] = (int)lo;     // (the host refuses shapes with 2^31 tiles or more)
+    range_s[5] = (int)total;
+    range_s[6] = (int)ctas;
   }
   // rows R..255 of the Q buffer are never written by TMA: keep them zero so their logits are 0. Pass 2: the operands
   // of the extra contraction step start out as zeros, the key side gets its three ones per row (128-byte rows with
@@ -334,26 +376,15 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   const bool exact = range_s[3] != 0;
 
   auto cursor_begin = [&]() {
-    ItemCursor c;
+    TileCursor c;
     c.b = range_s[0];
     c.r = range_s[1];
     c.left = c.b < p.B ? range_s[2] : 0;
-    c.s_b = c.left > 0 ? (exact ? splits_of(p, c.b) : p.splits) : 1;
-    c.per_b = p.L * p.Hkv * c.s_b;
+    c.done = 0;
+    c.tb = c.left > 0 ? tiles_of(p, c.b, exact) : 1;
+    c.per_b = p.L * p.Hkv * c.tb;
     cursor_settle(p, c, exact);
     return c;
-  };
-  auto cursor_next = [&](ItemCursor& c) {
-    ++c.r;
-    --c.left;
-    cursor_settle(p, c, exact);
-  };
-  // keys and tiles of an item
-  auto item_tiles = [&](int u, int split, int& key_begin, int& n) {
-    const int b = u / (p.Hkv * p.L);
-    n = clamped_len(p.seq_len, b, p.n_max);
-    key_begin = split * kSplitKeys;
-    return key_begin < n ? (min(n, key_begin + kSplitKeys) - key_begin + kTileKeys - 1) / kTileKeys : 0;
   };
 
   if (warp == 0) {
@@ -364,13 +395,13 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     int stage = 0, cur_u = -1;
     uint32_t stage_par = 0, q_par = 0;
     bool ok = true;
-    for (ItemCursor c = cursor_begin(); ok && c.left > 0; cursor_next(c)) {
-      int u, split, key_begin, n;
-      cursor_item(p, c, u, split);
-      const int tiles = item_tiles(u, split, key_begin, n);
+    for (TileCursor c = cursor_begin(); ok && c.left > 0;) {
+      const Run run = cursor_run(p, c);
+      cursor_advance(p, c, run, exact);
+      const int u = run.u, tiles = run.tiles, key_begin = run.t0 * kTileKeys;
       if (tiles == 0) continue;
       const int h = u % p.Hkv, l = (u / p.Hkv) % p.L, b = u / (p.Hkv * p.L);
-      if (u != cur_u) {  // the unit changes: its queries (and, in pass 2, its shift rows)
+      if (u != cur_u) {  // a new run: the unit's queries (and, in pass 2, its shift rows)
         cur_u = u;
         if (lane == 0) ok = mbar_wait(qempty, q_par ^ 1, abort_flag, p.status, kSiteQEmpty);
         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -428,10 +459,10 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
       int stage = 0, n_tile = 0, cur_u = -1;
       uint32_t stage_par = 0, q_par = 0;
       bool ok = true;
-      for (ItemCursor c = cursor_begin(); ok && c.left > 0; cursor_next(c)) {
-        int u, split, key_begin, n;
-        cursor_item(p, c, u, split);
-        const int tiles = item_tiles(u, split, key_begin, n);
+      for (TileCursor c = cursor_begin(); ok && c.left > 0;) {
+        const Run run = cursor_run(p, c);
+        cursor_advance(p, c, run, exact);
+        const int u = run.u, tiles = run.tiles;
         if (tiles == 0) continue;
         if (u != cur_u) {
           if (cur_u >= 0) umma_commit(qempty);  // the queries may be replaced once the MMAs issued so far are done
@@ -502,7 +533,7 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     }
     const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16) + (PASS == 1 ? mb * 128 : 0) + blk0 * 16;
     const uint64_t sc2 = pack2(p.scale2, p.scale2);
-    int n_tile = 0, cur_u = -1;
+    int n_tile = 0;
     bool ok = true;
     // pass 1 state: running maximum and sums of the thread's window row, log2 domain; m starts below any masked
     // logit. The sum is kept on two levels (the item at hand, the run's earlier items): one accumulator over a whole
@@ -512,16 +543,14 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     uint64_t zacc[4] = {0ull, 0ull, 0ull, 0ull};  // pass 1: the item's sum, as four packed partial sums
     float* xslot = xch + quarter * 32 + lane;  // pass 2: [buffer][share - 1][128 keys]
 
-    for (ItemCursor c = cursor_begin(); ok && c.left > 0; cursor_next(c)) {
-      int u, split, key_begin, n;
-      cursor_item(p, c, u, split);
-      const int tiles = item_tiles(u, split, key_begin, n);
+    for (TileCursor c = cursor_begin(); ok && c.left > 0;) {
+      const Run run = cursor_run(p, c);
+      const int run_first = range_s[4] + c.done;  // the run's first tile in the global order
+      cursor_advance(p, c, run, exact);
+      const int u = run.u, tiles = run.tiles, key_begin = run.t0 * kTileKeys, n = run.n;
       float* psi = p.psi + (int64_t)u * p.n_max;
-      if (PASS == 1 && u != cur_u) {
-        cur_u = u;
-        m = 4.f * kEmptyMax;
-        z_run = 0.f;
-      }
+      m = 4.f * kEmptyMax;  // pass 1: every run starts its own statistics
+      z_run = 0.f;
       zacc[0] = zacc[1] = zacc[2] = zacc[3] = 0ull;
       int vis = 0;  // pass 1: keys the row may see: [0, vis)
       if (PASS == 1 && row < p.R) {
@@ -606,6 +635,10 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         }
         tc_fence_before();
         mbar_arrive(&tempty[buf]);
+        if (PASS == 1 && (t % kFoldTiles) == kFoldTiles - 1) {  // second level of the row's sum
+          z_run += sum4(zacc);
+          zacc[0] = zacc[1] = zacc[2] = zacc[3] = 0ull;
+        }
         if (PASS == 2) {
           // the four warps that share the key add up in a fixed order: shares 1-3 hand their sums to share 0 (a
           // slot is free once share 0 has taken the tile before last)
@@ -628,27 +661,19 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
       if (!ok) break;
       if (PASS == 1) {
         z_run += sum4(zacc);
-        if (row < p.R && tiles > 0) {
-          // the pair goes out with the last item of the run (the next item is another unit's, holds no keys, or does
-          // not exist); the run's other items leave an empty pair so that the merge finds every split that holds keys
-          ItemCursor nx = c;
-          cursor_next(nx);
-          bool last = nx.left <= 0;
-          if (!last) {
-            int u2, s2, kb2, n2;
-            cursor_item(p, nx, u2, s2);
-            last = u2 != u || item_tiles(u2, s2, kb2, n2) == 0;
-          }
-          // a row that saw no visible key only summed masked entries: it is recorded as empty
-          const bool none = m < 0.5f * kEmptyMax * p.scale2;
-          p.part[(((int64_t)u * p.splits + split) * p.cparts + share) * p.rs + row] =
-              (!last || none) ? make_float2(kEmptyMax, 0.f) : make_float2(m, z_run);
+        if (row < p.R) {
+          // one pair per run: slot = this CTA's place among the CTAs that the unit's tiles are spread over (the merge
+          // kernel walks the same partition). A row that saw no visible key only summed masked entries: it is
+          // recorded as empty, and so is a run without keys (the uniform partition of very large batches has those).
+          const long long total = range_s[5];
+          const int k = (int)blockIdx.x - cta_of(total, range_s[6], (long long)run_first - run.t0);
+          const bool none = tiles == 0 || m < 0.5f * kEmptyMax * p.scale2;
+          if (k >= 0 && k < p.smax)
+            p.part[(((int64_t)u * p.smax + k) * p.cparts + share) * p.rs + row] =
+                none ? make_float2(kEmptyMax, 0.f) : make_float2(m, z_run);
+          else
+            set_status(p.status, MADAKV_ESHAPE);  // cannot happen: smax bounds the runs of a unit
         }
-      } else {
-        // keys of the item beyond its last tile (the remainder of psi's padding is cleared by the kernel that
-        // prepares the log-sum-exps)
-        for (int k2 = key_begin + tiles * kTileKeys + ew * 32 + lane; k2 < min(key_begin + kSplitKeys, p.n_max); k2 += 512)
-          psi[k2] = 0.f;
       }
     }
   }
@@ -662,16 +687,16 @@ score_rows_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   }
 }
 
-// psi of the keys no work item covers: everything from the first split that lies wholly beyond the sequence
+// psi of the keys no tile covers: everything from the end of the sequence's last tile
 __device__ __forceinline__ void clear_tail(const RowParams& p, int u, int row) {
   const int b = u / (p.Hkv * p.L);
   const int n = clamped_len(p.seq_len, b, p.n_max);
-  const int from = (n + kSplitKeys - 1) / kSplitKeys * kSplitKeys;
+  const int from = (n + kTileKeys - 1) / kTileKeys * kTileKeys;
   float* psi = p.psi + (int64_t)u * p.n_max;
   for (int key = from + row; key < p.n_max; key += p.rs) psi[key] = 0.f;
 }
 
-// merge: per (unit, row) the (max, sum) pairs of all splits and column shares, in a fixed order -> log2-domain
+// merge: per (unit, row) the (max, sum) pairs of all runs and column shares, in a fixed order -> log2-domain
 // log-sum-exp, stored negated (pass 2 adds it inside a fused multiply-add); padding rows get a shift that turns
 // every weight into 0
 __global__ void score_rows_merge_kernel(RowParams p, float* nlse2, float* lse_out, int total) {
@@ -684,8 +709,27 @@ __global__ void score_rows_merge_kernel(RowParams p, float* nlse2, float* lse_ou
     return;
   }
   const int b = u / (p.Hkv * p.L);
-  const int entries = p.cparts * splits_of(p, b);  // the splits that hold keys of this sequence
-  const float2* part = p.part + (int64_t)u * p.cparts * p.splits * p.rs + row;
+  // the CTAs of pass 1 that the unit's tiles were spread over: the same partition as in the kernel
+  const bool exact = p.B <= kMaxSeqScan;
+  long long all_tiles = 0, first = 0;  // tiles of the batch; the unit's first tile in the global order
+  const int tb = tiles_of(p, b, exact);
+  if (exact) {
+    for (int b2 = 0; b2 < p.B; ++b2) {
+      const long long per = (long long)p.L * p.Hkv * tiles_of(p, b2, true);
+      if (b2 < b) first += per;
+      all_tiles += per;
+    }
+  } else {
+    all_tiles = (long long)p.units * tb;
+    first = (long long)b * p.L * p.Hkv * tb;
+  }
+  first += (long long)(u - b * p.L * p.Hkv) * tb;
+  int entries = 0;
+  if (tb > 0) {
+    const int ctas = (int)(all_tiles < p.grid ? all_tiles : p.grid);
+    entries = p.cparts * min(p.smax, cta_of(all_tiles, ctas, first + tb - 1) - cta_of(all_tiles, ctas, first) + 1);
+  }
+  const float2* part = p.part + (int64_t)u * p.cparts * p.smax * p.rs + row;
   float M = kEmptyMax;
   for (int s = 0; s < entries; ++s) M = fmaxf(M, part[(int64_t)s * p.rs].x);
   float Z = 0.f;
@@ -756,7 +800,7 @@ static bool rows_setup(const madakv_config& c, const void* q, madakv_strides sq,
   p.R = R;
   p.n_max = c.max_seq_len;
   p.causal = c.causal;
-  p.splits = (c.max_seq_len + kSplitKeys - 1) / kSplitKeys;
+  p.smax = wide_max_runs(c);
   p.rs = (R + 31) / 32 * 32;  // row stride of the workspace arrays
   p.mblocks = R <= 128 ? 1 : 2;
   p.cparts = R <= 128 ? 4 : 2;
@@ -768,9 +812,11 @@ static bool rows_setup(const madakv_config& c, const void* q, madakv_strides sq,
     rc = MADAKV_ECUDA;
     return false;
   }
-  const long long items = (long long)p.units * p.splits;
-  if (items > 0x3fffffff) return false;
-  grid = (int)(items < sms ? items : sms);
+  const long long tiles = (long long)p.units * ((c.max_seq_len + kTileKeys - 1) / kTileKeys);
+  if (tiles > 0x3fffffff) return false;
+  if (sms > kWideMaxGrid) sms = kWideMaxGrid;
+  grid = (int)(tiles < sms ? tiles : sms);
+  p.grid = grid;
   if (!make_map(&mk, k, c.head_dim, c.max_seq_len, c.n_kv_heads, c.n_layers, c.batch, sk, kTileKeys, 1) ||
       !make_map(&mq, q, c.head_dim, c.window, c.n_q_heads, c.n_layers, c.batch, sq, c.window, g))
     return false;
