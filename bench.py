@@ -450,7 +450,7 @@ class Bench:
     # layer l on stream l % NS, compaction on another; the dependencies score(l) -> allocate(l) -> select(l) ->
     # compact(l), phi(l) -> allocate(l + 1) and the reuse of a layer's scratch are events. The whole pass is captured
     # once into a CUDA graph and replayed, so the host's launch cost is out of the picture.
-    def time_streamed(self, steps=3, overlapped=True, NS=4):
+    def time_streamed(self, steps=3, overlapped=True, NS=8):
         mk, wl, buf, inp = self.mk, self.wl, self.buf, self.inp
         cfg1 = mk.make_config(wl.torch_dtype, wl.B, 1, wl.Hq, wl.Hkv, wl.d, wl.n, wl.w,
                               max_new_tokens=wl.max_new_tokens, theta=wl.theta)
@@ -494,11 +494,14 @@ class Bench:
                 scored.record(main)
                 with torch.cuda.stream(sd):
                     sd.wait_event(scored)
+                    # masses, preferences and demands (Eq. 6, 9) do not depend on the layer before ...
+                    mk.madakv_demand_layer(buf.cfg, o.psi, inp["mask"], inp["seq_len"], o.mass, o.pref, o.demand,
+                                           ws_side[l % slots])
                     if l - 1 in alloc_done:
-                        sd.wait_event(alloc_done[l - 1])  # phi^l comes from the layer before (Eq. 11)
+                        sd.wait_event(alloc_done[l - 1])  # ... phi^l does (Eq. 11)
                     if l - slots in cmp_done:
                         sd.wait_event(cmp_done[l - slots])  # the scratch's kept positions were read by its compaction
-                    mk.madakv_allocate_layer(buf.cfg, l, o.psi, inp["mask"], inp["seq_len"], inp["budget"], o.mass,
+                    mk.madakv_allocate_layer(buf.cfg, l, None, inp["mask"], inp["seq_len"], inp["budget"], o.mass,
                                              o.pref, o.demand, phi, o.budgets, ws_side[l % slots])
                     alloc_done[l] = torch.cuda.Event()
                     alloc_done[l].record(sd)
@@ -652,8 +655,10 @@ class Bench:
                     "ms_eager_one_stream": None if s1 is None else s1["ms"],
                     "ratio_to_all_layer_pass": None if s2 is None else s2["ms"] / pass_ms, "launches": wl.L * 7,
                     "note": "stages 1-4 layer by layer (madakv_score_lse, madakv_allocate_layer, select and compact "
-                            "with one-layer configs). overlapped: four layers in flight on their own streams (scoring, "
-                            "allocation + selection, compaction), replayed from one CUDA graph; not part of the step"}
+                            "with one-layer configs). overlapped: eight layers in flight on their own streams (scoring; "
+                            "madakv_demand_layer, then madakv_allocate_layer without scores once the layer before "
+                            "has passed phi on, selection; compaction), replayed from one CUDA graph; not part of "
+                            "the step"}
         return rec
 
 

@@ -161,6 +161,15 @@ int madakv_allocate_layer(const madakv_config* cfg, int32_t layer, const float* 
                           const int32_t* seq_len, const int32_t* budget, double* mass, double* pref, int32_t* demand,
                           double* phi, int32_t* budgets, void* ws, size_t ws_bytes, void* stream);
 
+/* The part of madakv_allocate_layer that does not depend on the budget state: mass, pref and demand of one layer
+ * (Eq. 6, the ratio of Eq. 8, Eq. 9) from that layer's psi. Only Eq. 10-11 chain the layers together, so a caller
+ * that keeps several layers in flight runs this call for layer l + 1 while layer l is still being allocated, and
+ * then calls madakv_allocate_layer with psi = NULL, which takes mass, pref and demand as given and does the rest
+ * (Phi^l, phi^{l+1}, budgets). The two calls together write exactly what madakv_allocate_layer alone writes.
+ *   psi [B,H_kv,n_max]; mass, pref [B,H_kv,2] fp64; demand [B,H_kv,2] int32 (cfg as for madakv_allocate_layer)   */
+int madakv_demand_layer(const madakv_config* cfg, const float* psi, const uint8_t* mask, const int32_t* seq_len,
+                        double* mass, double* pref, int32_t* demand, void* ws, size_t ws_bytes, void* stream);
+
 /* Stage 4a (Section 3.3: modality-specific eviction for each head). For every unit keep, of each modality m,
  * the budgets[u][m] tokens with the largest psi (equal psi: the lower position wins) and list the kept positions
  * in ascending order:
@@ -228,7 +237,8 @@ const char* madakv_status_string(int status);
 
 /* Library version, bumped when the ABI changes. 2: madakv_score_lse, madakv_allocate_layer and MADAKV_HCC_DEMAND added
  * (nothing that version 1 had was changed). 3: madakv_config grew by keep_window and pool_kernel (struct_size is
- * checked: a caller built against version 2 gets MADAKV_EINVAL, not a misread struct). */
+ * checked: a caller built against version 2 gets MADAKV_EINVAL, not a misread struct). 4: madakv_demand_layer
+ * added, madakv_allocate_layer accepts psi = NULL (nothing that version 3 had was changed). */
 int madakv_abi_version(void);
 
 #ifdef __cplusplus

@@ -21,7 +21,7 @@ STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = [
     "madakv_abi_version", "madakv_status_string", "madakv_workspace_bytes", "madakv_score", "madakv_score_lse",
-    "madakv_allocate", "madakv_allocate_layer",
+    "madakv_allocate", "madakv_allocate_layer", "madakv_demand_layer",
     "madakv_select", "madakv_compact", "madakv_decode_attn", "madakv_decode_attn_static", "madakv_poll_status",
 ]
 
@@ -69,6 +69,7 @@ def lib():
         L.madakv_score_lse.argtypes = [cfgp, vp, MadakvStrides, vp, MadakvStrides, vp, vp, vp, vp, sz, vp]
         L.madakv_allocate.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.madakv_allocate_layer.argtypes = [cfgp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.madakv_demand_layer.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.madakv_select.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, i64, vp, sz, vp]
         L.madakv_compact.argtypes = [cfgp, vp, vp, MadakvStrides, vp, vp, vp, vp, vp, i64, vp, sz, vp]
         L.madakv_decode_attn.argtypes = [cfgp, i32, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, sz, vp]
@@ -135,7 +136,14 @@ def madakv_allocate(cfg, psi, mask, seq_len, budget, mass, pref, demand, phi, bu
                                                     _ptr(budgets), _ptr(ws), ws.numel(), _stream()))
 
 
+def madakv_demand_layer(cfg, psi, mask, seq_len, mass, pref, demand, ws):
+    _check("madakv_demand_layer", lib().madakv_demand_layer(ctypes.byref(cfg), _ptr(psi), _ptr(mask), _ptr(seq_len),
+                                                            _ptr(mass), _ptr(pref), _ptr(demand), _ptr(ws), ws.numel(),
+                                                            _stream()))
+
+
 def madakv_allocate_layer(cfg, layer, psi, mask, seq_len, budget, mass, pref, demand, phi, budgets, ws):
+    """psi may be None: mass, pref and demand then come from madakv_demand_layer."""
     _check("madakv_allocate_layer", lib().madakv_allocate_layer(ctypes.byref(cfg), int(layer), _ptr(psi), _ptr(mask),
                                                                 _ptr(seq_len), _ptr(budget), _ptr(mass), _ptr(pref),
                                                                 _ptr(demand), _ptr(phi), _ptr(budgets), _ptr(ws),

@@ -461,8 +461,33 @@ int launch_allocate_layer(const madakv_config& c, int layer, const float* psi, c
   p.keep_window = c.keep_window;
   p.window = c.window;
   p.theta_fix = (u64)((double)c.theta * 4294967296.0);
-  alloc_unit_kernel<<<c.batch * c.n_kv_heads, NT, 0, st>>>(p);
+  if (psi) alloc_unit_kernel<<<c.batch * c.n_kv_heads, NT, 0, st>>>(p);  // else: done by launch_demand_layer
   alloc_layer_kernel<<<c.batch, 1024, 0, st>>>(p, c.n_layers, layer);
+  return launch_status();
+}
+
+int launch_demand_layer(const madakv_config& c, const float* psi, const uint8_t* mask, const int32_t* seq_len,
+                        double* mass, double* pref, int32_t* demand, void* ws, cudaStream_t st) {
+  (void)ws;
+  AllocParams p;
+  p.psi = psi;
+  p.mask = mask;
+  p.seq_len = seq_len;
+  p.budget = nullptr;
+  p.mass = mass;
+  p.pref = pref;
+  p.demand = demand;
+  p.phi = nullptr;
+  p.budgets = nullptr;
+  p.L = 1;  // the per-layer arrays hold one layer
+  p.Hkv = c.n_kv_heads;
+  p.n_max = c.max_seq_len;
+  p.mpa = c.mpa;
+  p.hcc_mode = c.hcc_mode;
+  p.keep_window = c.keep_window;
+  p.window = c.window;
+  p.theta_fix = (u64)((double)c.theta * 4294967296.0);
+  alloc_unit_kernel<<<c.batch * c.n_kv_heads, NT, 0, st>>>(p);
   return launch_status();
 }
 

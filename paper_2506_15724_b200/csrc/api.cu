@@ -6,7 +6,7 @@ using namespace madakv;
 
 extern "C" {
 
-int madakv_abi_version(void) { return 3; }
+int madakv_abi_version(void) { return 4; }
 
 const char* madakv_status_string(int s) {
   switch (s) {
@@ -75,13 +75,26 @@ int madakv_allocate_layer(const madakv_config* cfg, int32_t layer, const float* 
   int rc = check_config(cfg);
   if (rc) return rc;
   if (layer < 0 || layer >= cfg->n_layers) return MADAKV_ESHAPE;
-  if (!psi || !mask || !seq_len || !budget || !mass || !pref || !demand || !phi || !budgets) return MADAKV_EINVAL;
+  // psi may be null: mass, pref and demand of the layer then come from madakv_demand_layer
+  if (!mask || !seq_len || !budget || !mass || !pref || !demand || !phi || !budgets) return MADAKV_EINVAL;
   if (!aligned16(psi) || ((uintptr_t)mass & 7) || ((uintptr_t)pref & 7) || ((uintptr_t)phi & 7) ||
       ((uintptr_t)demand & 7) || ((uintptr_t)budgets & 7) || ((uintptr_t)seq_len & 3) || ((uintptr_t)budget & 3))
     return MADAKV_EALIGN;
   if ((rc = check_ws(*cfg, ws, ws_bytes))) return rc;
   return launch_allocate_layer(*cfg, layer, psi, mask, seq_len, budget, mass, pref, demand, phi, budgets, ws,
                                (cudaStream_t)stream);
+}
+
+int madakv_demand_layer(const madakv_config* cfg, const float* psi, const uint8_t* mask, const int32_t* seq_len,
+                        double* mass, double* pref, int32_t* demand, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (!psi || !mask || !seq_len || !mass || !pref || !demand) return MADAKV_EINVAL;
+  if (!aligned16(psi) || ((uintptr_t)mass & 7) || ((uintptr_t)pref & 7) || ((uintptr_t)demand & 7) ||
+      ((uintptr_t)seq_len & 3))
+    return MADAKV_EALIGN;
+  if ((rc = check_ws(*cfg, ws, ws_bytes))) return rc;
+  return launch_demand_layer(*cfg, psi, mask, seq_len, mass, pref, demand, ws, (cudaStream_t)stream);
 }
 
 int madakv_select(const madakv_config* cfg, const float* psi, const uint8_t* mask, const int32_t* seq_len,

@@ -186,6 +186,8 @@ int launch_allocate(const madakv_config& c, const float* psi, const uint8_t* mas
 int launch_allocate_layer(const madakv_config& c, int layer, const float* psi, const uint8_t* mask,
                           const int32_t* seq_len, const int32_t* budget, double* mass, double* pref, int32_t* demand,
                           double* phi, int32_t* budgets, void* ws, cudaStream_t st);
+int launch_demand_layer(const madakv_config& c, const float* psi, const uint8_t* mask, const int32_t* seq_len,
+                        double* mass, double* pref, int32_t* demand, void* ws, cudaStream_t st);
 int launch_select(const madakv_config& c, const float* psi, const uint8_t* mask, const int32_t* seq_len,
                   const int32_t* budgets, int32_t* kept_len, int64_t* seg_off, int32_t* kept_idx, int64_t capacity,
                   void* ws, cudaStream_t st);

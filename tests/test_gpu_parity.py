@@ -365,11 +365,14 @@ def test_allocate_and_select_on_crafted_scores(kind, n):
 
 @pytest.mark.parametrize("name", ["tiny_gqa_ragged", "bf16_d128", "bf16_gqa7", "tc_short_seqs"])
 @pytest.mark.parametrize("hcc", [mk.HCC_PAPER, mk.HCC_LITERAL, mk.HCC_DEMAND])
-def test_layer_by_layer_pass_equals_the_all_layer_pass(name, hcc):
+@pytest.mark.parametrize("split", [False, True])
+def test_layer_by_layer_pass_equals_the_all_layer_pass(name, hcc, split):
     """The streaming use of the library: layer after layer, single-pass scoring with given log-sum-exps, then
     madakv_allocate_layer carrying phi, then selection and compaction with one-layer configs on slices of K/V. Given
     the same fp32 scores everything downstream is bit-identical to the all-layer calls; the single-pass scores
-    themselves agree with the two-pass ones to rounding."""
+    themselves agree with the two-pass ones to rounding. split: masses, preferences and demands of ALL layers come
+    from madakv_demand_layer first (they do not depend on the budget state), then madakv_allocate_layer without
+    scores walks the layers."""
     wl = SHAPES[name]
     inp = make_case(wl)
     g = dev(inp)
@@ -384,14 +387,19 @@ def test_layer_by_layer_pass_equals_the_all_layer_pass(name, hcc):
     r_idx, r_kc, r_vc = ref.kept_idx.cpu().numpy(), ref.k_c, ref.v_c
     phi = torch.zeros((wl.B, wl.L), dtype=torch.float64, device="cuda")
     cap1 = capacity_of(synth.scaled(wl, L=1))
+    ones = [mk.EvictionBuffers(cfg1, cap1) for _ in range(wl.L)]
+    if split:
+        for l in range(wl.L):
+            mk.madakv_demand_layer(cfg, ref.psi[:, l:l + 1].contiguous(), g["mask"], g["seq_len"], ones[l].mass,
+                                   ones[l].pref, ones[l].demand, ref.ws)
     for l in range(wl.L):
-        one = mk.EvictionBuffers(cfg1, cap1)
+        one = ones[l]
         q_l, k_l, v_l = g["q_win"][:, l:l + 1], g["k"][:, l:l + 1], g["v"][:, l:l + 1]  # views: strides go through
         mk.madakv_score_lse(cfg1, q_l, k_l, g["seq_len"], ref.lse[:, l:l + 1].contiguous(), one.psi, one.ws)
         assert psi_close(one.psi.cpu().numpy(), ref.psi[:, l:l + 1].cpu().numpy().astype(np.float64), 1e-4) < 1e-4
         psi_l = ref.psi[:, l:l + 1].contiguous()  # from here on the same scores as the all-layer pass
-        mk.madakv_allocate_layer(cfg, l, psi_l, g["mask"], g["seq_len"], g["budget"], one.mass, one.pref, one.demand,
-                                 phi, one.budgets, ref.ws)
+        mk.madakv_allocate_layer(cfg, l, None if split else psi_l, g["mask"], g["seq_len"], g["budget"], one.mass,
+                                 one.pref, one.demand, phi, one.budgets, ref.ws)
         for key in ("mass", "pref", "demand", "budgets"):
             assert torch.equal(getattr(one, key)[:, 0], getattr(ref, key)[:, l]), (key, l)
         mk.madakv_select(cfg1, psi_l, g["mask"], g["seq_len"], one.budgets, one.kept_len, one.seg_off, one.kept_idx,

@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol(lib):
     for name in declared:
         assert hasattr(lib, name), name
     assert declared == set(mk.EXPORTS)
-    assert lib.madakv_abi_version() == 3
+    assert lib.madakv_abi_version() == 4
     assert mk.madakv_status_string(mk.ECAPACITY) == "ragged cache capacity exceeded"
 
 
@@ -90,6 +90,11 @@ def test_entry_points_reject_bad_arguments_before_launch(lib):
                                      None) == mk.ESHAPE
     assert lib.madakv_allocate_layer(cref, 0, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, None, FAKE, FAKE, need,
                                      None) == mk.EINVAL
+    # the budget-free half of the per-layer allocation needs its score array; the other half may go without
+    assert lib.madakv_demand_layer(cref, None, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, need, None) == mk.EINVAL
+    assert lib.madakv_demand_layer(cref, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, need - 1, None) == mk.EWORKSPACE
+    assert lib.madakv_allocate_layer(cref, 0, None, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, need - 1,
+                                     None) == mk.EWORKSPACE
     # misaligned pointer / stride
     assert lib.madakv_score(cref, odd, good, FAKE, good, FAKE, None, FAKE, FAKE, need, None) == mk.EALIGN
     assert lib.madakv_score(cref, FAKE, st, FAKE, good, FAKE, None, FAKE, FAKE, need, None) == mk.EALIGN
