@@ -702,6 +702,7 @@ def test_full_size_workload(name, record_property):
     assert mk.madakv_poll_status(buf.ws) == 0
     out = buf.out.float().cpu().numpy().reshape(wl.B * wl.L, wl.Hq, wl.d)
     q3 = q.view(wl.B * wl.L, wl.Hq, wl.d)
+    worst_dec = 0.0
     for u in rng.choice(wl.units, size=6, replace=False).tolist() + [0, wl.units - 1]:
         a, b = int(seg_off[u]), int(seg_off[u] + kept_len[u])
         kc, vc = to_np(buf.k_c[a:b]), to_np(buf.v_c[a:b])
@@ -709,7 +710,9 @@ def test_full_size_workload(name, record_property):
         heads = slice(h * wl.g, (h + 1) * wl.g)
         rc, want_o, _ = oracle.decode(1, to_np(q3[bl, heads]).reshape(1, 1, wl.g, wl.d), None, None, kc, vc,
                                       np.array([0, b - a], np.int64), np.array([b - a], np.int32), Hkv=1)
-        assert np.abs(out[bl, heads] - want_o.reshape(wl.g, wl.d)).max() <= DEC_ATOL["bf16"], u
+        worst_dec = max(worst_dec, float(np.abs(out[bl, heads] - want_o.reshape(wl.g, wl.d)).max()))
+        assert worst_dec <= DEC_ATOL["bf16"], u
+    record_property("worst_decode_abs_error", worst_dec)
 
 
 @pytest.mark.parametrize("name", ["batched", "long"])
