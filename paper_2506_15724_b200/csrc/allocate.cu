@@ -135,15 +135,33 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
 
   uint32_t key[KPT];
   uint32_t flags = 0;  // bit j: key j exists; bit 16 + j: key j is a visual token
+  // a thread takes KPT consecutive keys of a round (which keys a thread holds does not matter: all sums are exact);
+  // a full, aligned stretch comes in four 16-byte loads of scores and one of mask bytes
+  const bool vec = (p.n_max & 3) == 0 && (reinterpret_cast<uintptr_t>(mask) & 15) == 0;
   auto load_round = [&](int r) {
     flags = 0;
+    const int i0 = r * ROUND + (int)threadIdx.x * KPT;
+    if (vec && i0 + KPT <= n) {
 #pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-      const int i = r * ROUND + j * NT + (int)threadIdx.x;
-      key[j] = 0;
-      if (i < n) {
-        key[j] = psi_key(__ldg(psi + i));
-        flags |= (1u << j) | (__ldg(mask + i) ? (0x10000u << j) : 0u);
+      for (int j = 0; j < KPT; j += 4) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(psi + i0 + j));
+        key[j] = psi_key(v.x);
+        key[j + 1] = psi_key(v.y);
+        key[j + 2] = psi_key(v.z);
+        key[j + 3] = psi_key(v.w);
+      }
+      const uint4 mv = __ldg(reinterpret_cast<const uint4*>(mask + i0));
+      flags = 0xffffu | ((nonzero_bytes(mv.x) | (nonzero_bytes(mv.y) << 4) | (nonzero_bytes(mv.z) << 8) |
+                          (nonzero_bytes(mv.w) << 12)) << 16);
+    } else {
+#pragma unroll
+      for (int j = 0; j < KPT; ++j) {
+        const int i = i0 + j;
+        key[j] = 0;
+        if (i < n) {
+          key[j] = psi_key(__ldg(psi + i));
+          flags |= (1u << j) | (__ldg(mask + i) ? (0x10000u << j) : 0u);
+        }
       }
     }
   };

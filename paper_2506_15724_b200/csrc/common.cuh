@@ -155,6 +155,11 @@ __device__ __forceinline__ int clamped_len(const int32_t* seq_len, int b, int n_
   return max(0, min(seq_len[b], n_max));
 }
 __device__ __forceinline__ uint32_t psi_key(float x) { return x > 0.0f ? __float_as_uint(x) : 0u; }
+// Bit i of the result: byte i of the word is not zero (four mask bytes at a time).
+__device__ __forceinline__ uint32_t nonzero_bytes(uint32_t w) {
+  const uint32_t x = ((((w & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w) & 0x80808080u) >> 7;  // bits 0, 8, 16, 24
+  return (x & 1u) | ((x >> 7) & 2u) | ((x >> 14) & 4u) | ((x >> 21) & 8u);
+}
 // floor(x * 2^32) of a key produced by psi_key.
 __device__ __forceinline__ unsigned long long psi_fix(uint32_t key) {
   return key ? __float2ull_rz(__uint_as_float(key) * 4294967296.0f) : 0ull;

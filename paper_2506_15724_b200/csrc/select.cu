@@ -179,9 +179,17 @@ __device__ __forceinline__ void load_chunk(const float* psi, const uint8_t* mask
     }
   }
   if (mpa) {
+    if (kVec && pos0 + KPT <= n && (reinterpret_cast<uintptr_t>(mask + pos0) & 15) == 0) {  // 16 mask bytes per load
 #pragma unroll
-    for (int j = 0; j < KPT; ++j)
-      if (pos0 + j < n && __ldg(mask + pos0 + j)) vis |= 1u << j;
+      for (int j = 0; j < KPT; j += 16) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(mask + pos0 + j));
+        vis |= (nonzero_bytes(v.x) | (nonzero_bytes(v.y) << 4) | (nonzero_bytes(v.z) << 8) | (nonzero_bytes(v.w) << 12)) << j;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < KPT; ++j)
+        if (pos0 + j < n && __ldg(mask + pos0 + j)) vis |= 1u << j;
+    }
   }
   if (kPool && pos0 + KPT > wfrom) {  // proxy tokens retained unconditionally: out of the ranking, into the output
 #pragma unroll
