@@ -50,12 +50,19 @@ __global__ void __launch_bounds__(1024) seg_scan_kernel(SelParams p) {
     if (threadIdx.x == 0) s_cnt = s_wcnt = 0;
     __syncthreads();
     int c = 0, cw = 0;  // visual tokens, visual proxy tokens
-    if (p.mpa)
-      for (int i = threadIdx.x; i < n; i += 1024)
-        if (mask[i]) {
-          ++c;
-          if (i >= wfrom) ++cw;
+    if (p.mpa) {
+      int done = 0;
+      if ((reinterpret_cast<uintptr_t>(mask) & 15) == 0) {  // 16 mask bytes per load
+        const int n16 = n >> 4;
+        for (int i = threadIdx.x; i < n16; i += 1024) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(mask) + i);
+          c += __popc(nonzero_bytes(v.x) | (nonzero_bytes(v.y) << 4) | (nonzero_bytes(v.z) << 8) | (nonzero_bytes(v.w) << 12));
         }
+        done = n16 << 4;
+      }
+      for (int i = done + threadIdx.x; i < n; i += 1024) c += mask[i] ? 1 : 0;
+      for (int i = wfrom + threadIdx.x; i < n; i += 1024) cw += mask[i] ? 1 : 0;  // (no proxy tokens: wfrom = n)
+    }
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) {
       c += __shfl_xor_sync(kFull, c, off);
