@@ -138,8 +138,36 @@ inline int launch_status() {
   return MADAKV_ECUDA;
 }
 
+// Launch with programmatic stream serialisation: the grid may be scheduled while the kernel before it in the stream is
+// still running, which hides its launch latency. A kernel launched this way calls pdl_wait() before it touches global
+// memory (the call returns once the kernels before it have completed and their writes are visible; it is a no-op in a
+// kernel launched the ordinary way) and pdl_go() to let the kernel after it be scheduled.
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  // a stream that is being captured gets the ordinary launch (full serialisation: the waits in the kernels are no-ops)
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) cap = cudaStreamCaptureStatusActive;
+  if (cap == cudaStreamCaptureStatusNone) {
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---------------------------------------------------------------------------------------------------------------
 // Device helpers
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_go() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
 // ---------------------------------------------------------------------------------------------------------------
 #ifdef __CUDACC__
 __device__ __forceinline__ float ld_f32(const float* p) { return *p; }

@@ -152,6 +152,8 @@ __global__ void __launch_bounds__(NT) decode_partial_kernel(DecodeParams p) {
   __shared__ float s_o[GROUPS][G][D];
   __shared__ float s_m[GROUPS][G], s_l[GROUPS][G];
 
+  pdl_wait();
+  pdl_go();
   const int y = p.slot_fast ? blockIdx.x / p.slots : blockIdx.x % p.n_sel;
   const int u = unit_of(p, y);
   const int slot = p.slot_fast ? blockIdx.x % p.slots : blockIdx.x / p.n_sel;
@@ -341,6 +343,8 @@ __global__ void __launch_bounds__(kMmaWarps * 32, 3) decode_partial_mma_kernel(D
   constexpr int NB = D / 8;            // 8-column blocks of the output
   extern __shared__ __align__(16) unsigned char dsmem[];
 
+  pdl_wait();
+  pdl_go();
   const int u = unit_of(p, p.slot_fast ? blockIdx.x / p.slots : blockIdx.x % p.n_sel);
   const int slot = p.slot_fast ? blockIdx.x % p.slots : blockIdx.x / p.n_sel;
   const SegView view = segment_view(p, u, slot == 0 && threadIdx.x == 0);
@@ -512,6 +516,8 @@ __global__ void __launch_bounds__(kMmaWarps * 32, 3) decode_partial_mma_kernel(D
 template <typename T, int D>
 __global__ void __launch_bounds__(D) decode_merge_kernel(DecodeParams p) {
   // blockIdx.x enumerates the query heads of the selected layer(s)
+  pdl_wait();
+  pdl_go();
   int row;
   if (p.layer < 0) {
     row = blockIdx.x;
@@ -568,14 +574,15 @@ int run(const DecodeParams& p, const madakv_config&, cudaStream_t st) {
   }
   const dim3 grid((unsigned)n_sel * p.slots);  // one dimension: no 65535 limit on the number of segments
   if constexpr (sizeof(T) == 2) {
-    if (mma) decode_partial_mma_kernel<D><<<grid, kMmaWarps * 32, MmaTile<D>::BYTES, st>>>(p);
+    if (mma) launch_pdl(decode_partial_mma_kernel<D>, grid, dim3(kMmaWarps * 32), MmaTile<D>::BYTES, st, p);
   }
   if (mma) {
-  } else if (p.g == 1) decode_partial_kernel<T, D, 1><<<grid, NT, 0, st>>>(p);
-  else if (p.g == 2) decode_partial_kernel<T, D, 2><<<grid, NT, 0, st>>>(p);
-  else if (p.g <= 4) decode_partial_kernel<T, D, 4><<<grid, NT, 0, st>>>(p);
-  else decode_partial_kernel<T, D, 8><<<grid, NT, 0, st>>>(p);
-  decode_merge_kernel<T, D><<<n_sel * p.g, D, 0, st>>>(p);
+  } else if (p.g == 1) launch_pdl(decode_partial_kernel<T, D, 1>, grid, dim3(NT), 0, st, p);
+  else if (p.g == 2) launch_pdl(decode_partial_kernel<T, D, 2>, grid, dim3(NT), 0, st, p);
+  else if (p.g <= 4) launch_pdl(decode_partial_kernel<T, D, 4>, grid, dim3(NT), 0, st, p);
+  else launch_pdl(decode_partial_kernel<T, D, 8>, grid, dim3(NT), 0, st, p);
+  // (the merge may be scheduled while the partial kernel runs; it waits for its completion before reading anything)
+  launch_pdl(decode_merge_kernel<T, D>, dim3(n_sel * p.g), dim3(D), 0, st, p);
   return launch_status();
 }
 
