@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
   const int top = max(32 - __clz(kmax - kmin), 1);
   if (rounds == 1) {
 #pragma unroll
-    for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
+    for (int j = 0; j < KPT; ++j) key[j] = (flags >> j) & 1u ? kmax - key[j] : 0xffffffffu;  // (see the passes)
   }
 
   // state of the descent, kept by warp m (all lanes alike) for modality m
@@ -219,13 +219,16 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
         if (rounds > 1) {
           load_round(r);
 #pragma unroll
-          for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
+          for (int j = 0; j < KPT; ++j) key[j] = (flags >> j) & 1u ? kmax - key[j] : 0xffffffffu;
         }
+        // One comparison per key: t of an existing key is below 2^top <= 2^31, a slot without a key holds all ones,
+        // and a modality that is done gets a prefix no shifted t can equal (rem >= 1).
+        const uint32_t want0 = act0 ? pre0 : 0xffffffffu, want1 = act1 ? pre1 : 0xffffffffu;
 #pragma unroll
         for (int j = 0; j < KPT; ++j) {
-          const int m = (flags >> (16 + j)) & 1u ? 0 : 1;
-          if (((flags >> j) & 1u) && (m == 0 ? act0 : act1) && (key[j] >> rem) == (m == 0 ? pre0 : pre1))
-            hist_add(hist, m * 256 + (int)((key[j] >> shift) & dmask), psi_fix(kmax - key[j]));
+          const bool vis = (flags >> (16 + j)) & 1u;
+          if ((key[j] >> rem) == (vis ? want0 : want1))
+            hist_add(hist, (vis ? 0 : 256) + (int)((key[j] >> shift) & dmask), psi_fix(kmax - key[j]));
         }
       }
     }

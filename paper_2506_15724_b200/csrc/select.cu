@@ -265,7 +265,7 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
   const int top = 32 - __clz(kmax - kmin);  // significant bits of t; 0 when all keys are equal
   if (chunks == 1) {
 #pragma unroll
-    for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
+    for (int j = 0; j < KPT; ++j) key[j] = (valid >> j) & 1u ? kmax - key[j] : 0xffffffffu;
   }
 
   // radix select: when all bits of t are resolved, s_prefix[m] is the t of the want[m]-th largest key of modality m
@@ -280,13 +280,12 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
       if (chunks > 1) {
         load_chunk<kVec, kPool>(psi, mask, n, c * CHUNK + (int)threadIdx.x * KPT, p.mpa, wfrom, p.pool_r, key, valid, vis, forced);
 #pragma unroll
-        for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
+        for (int j = 0; j < KPT; ++j) key[j] = (valid >> j) & 1u ? kmax - key[j] : 0xffffffffu;
       }
 #pragma unroll
-      for (int j = 0; j < KPT; ++j) {
+      for (int j = 0; j < KPT; ++j) {  // (a position outside the ranking holds all ones: no prefix equals its shifted t)
         const int m = (vis >> j) & 1u ? 0 : 1;
-        if (((valid >> j) & 1u) && (key[j] >> rem) == (m == 0 ? pre0 : pre1))
-          atomicAdd(&cnt[m][(key[j] >> shift) & dmask], 1u);
+        if ((key[j] >> rem) == (m == 0 ? pre0 : pre1)) atomicAdd(&cnt[m][(key[j] >> shift) & dmask], 1u);
       }
     }
     __syncthreads();
@@ -337,17 +336,16 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
     if (chunks > 1) {
       load_chunk<kVec, kPool>(psi, mask, n, pos0, p.mpa, wfrom, p.pool_r, key, valid, vis, forced);
 #pragma unroll
-      for (int j = 0; j < KPT; ++j) key[j] = kmax - key[j];
+      for (int j = 0; j < KPT; ++j) key[j] = (valid >> j) & 1u ? kmax - key[j] : 0xffffffffu;
     }
     uint32_t eq_bits = 0, gt_bits = 0;
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
       const bool v = (vis >> j) & 1u;
       const uint32_t thr = v ? thr0 : thr1;
-      if ((valid >> j) & 1u) {
-        if (key[j] == thr) eq_bits |= 1u << j;
-        if (key[j] < thr && (v ? want0 : want1) > 0) gt_bits |= 1u << j;  // smaller t: larger importance
-      }
+      // (thresholds are below 2^31; a position outside the ranking holds all ones and is neither equal nor smaller)
+      if (key[j] == thr) eq_bits |= 1u << j;
+      if (key[j] < thr && (v ? want0 : want1) > 0) gt_bits |= 1u << j;  // smaller t: larger importance
     }
     const uint32_t eq_pack = (uint32_t)__popc(eq_bits & vis) | ((uint32_t)__popc(eq_bits & ~vis) << 16);
     uint32_t eq_total;
