@@ -2,7 +2,7 @@
 // (Eq. 10-11) and the integer per-head, per-modality budgets.
 //
 // All sums of psi are exact: psi is mapped to 2^-32 fixed point (psi_fix) and added as 64-bit integers, so the
-// results do not depend on the order of summation or on the launch shape. Eq. 9 is a "top-p" count: a 4-pass
+// results do not depend on the order of summation or on the launch shape. Eq. 9 is a "top-p" count: a three- or four-pass
 // radix descent over the order-preserving bit pattern of psi with per-bucket (count, mass) histograms in shared
 // memory finds the bucket in which the descending prefix mass reaches theta * W_m; ties inside the final bucket
 // share one value, so the remaining count is a division. The keys of a unit sit in registers between passes. The layer recurrence is a scalar fp64 scan per sequence
@@ -34,14 +34,23 @@ struct AllocParams {
 
 // Shared histograms of one radix pass: per (modality, digit) a count and an exact 64-bit mass kept as two 32-bit
 // words (32-bit shared atomics are native; the carry of the low word is detected from the value the atomic returns).
-// Bucket b sits at word b + b / 32: the bucket walk has lane j read buckets 8j .. 8j+7, which in a dense array would be
-// an 8-way bank conflict on every load; with the skew the 32 lanes of a load hit 32 different banks.
-constexpr int kHistWords = 512 + 16;
-__device__ __forceinline__ int hist_slot(int bucket) { return bucket + (bucket >> 5); }
+// A digit has DIG bits. Sequences of more than one round are re-read from L2 in every pass, and with 10-bit digits the
+// 30 bits in which importance values differ at most take three passes instead of four (long: allocation 0.26 -> 0.20
+// ms); a sequence that sits in registers gains nothing from that and pays for the larger histograms (llava 0.067 ->
+// 0.073 ms), so configs whose sequences fit one round keep 8-bit digits.
+// Bucket b sits at word b + b / kPerLane: the bucket walk has lane j read buckets kPerLane * j + i, which in a dense
+// array would be a many-way bank conflict on every load; with the skew the 32 lanes of a load hit 32 different banks.
+template <int DIG>
 struct Hist {
-  unsigned int cnt[kHistWords], mlo[kHistWords], mhi[kHistWords];
+  static constexpr int kBuckets = 1 << DIG;        // per modality
+  static constexpr int kPerLane = kBuckets / 32;   // buckets a lane of the walking warp owns
+  static constexpr int kWords = 2 * kBuckets + 2 * 32;
+  unsigned int cnt[kWords], mlo[kWords], mhi[kWords];
+  __device__ __forceinline__ static int slot(int bucket) { return bucket + bucket / kPerLane; }
 };
-__device__ __forceinline__ void hist_add(Hist& h, int bucket, u64 m) {
+#define hist_slot(b) (Hist<DIG>::slot(b))
+template <int DIG>
+__device__ __forceinline__ void hist_add(Hist<DIG>& h, int bucket, u64 m) {
   const int s = hist_slot(bucket);
   atomicAdd(&h.cnt[s], 1u);
   const unsigned int add = (unsigned int)m;
@@ -49,27 +58,29 @@ __device__ __forceinline__ void hist_add(Hist& h, int bucket, u64 m) {
   const unsigned int hi = (unsigned int)(m >> 32) + ((unsigned int)(old + add) < old ? 1u : 0u);
   if (hi) atomicAdd(&h.mhi[s], hi);  // rare: importance values are mostly below 1, carries are few
 }
-__device__ __forceinline__ u64 hist_mass(const Hist& h, int bucket) {
+template <int DIG>
+__device__ __forceinline__ u64 hist_mass(const Hist<DIG>& h, int bucket) {
   const int s = hist_slot(bucket);
   return ((u64)h.mhi[s] << 32) | h.mlo[s];
 }
 
-// One warp walks the 256 buckets of modality m in ascending digit order (digits are taken from kmax - key, so this
-// is descending importance): the first bucket at which the running mass `above + mass[dig]` reaches need_c is the
-// one the threshold falls into (the last bucket if none does). Lane j owns buckets 8j..8j+7; a warp prefix scan
-// supplies what lies before them. Returns the bucket, and updates above / above_c to the mass / count strictly
-// before it (identical in every lane).
-__device__ __forceinline__ int descend(const Hist& h, int m, u64 need_c, u64& above, unsigned int& above_c,
+// One warp walks the buckets of modality m in ascending digit order (digits are taken from kmax - key, so this is
+// descending importance): the first bucket at which the running mass `above + mass[dig]` reaches need_c is the one
+// the threshold falls into (the last bucket if none does). Lane j owns buckets kPerLane * j ..; a warp prefix scan of
+// the lanes' totals tells which lane holds that bucket, and that lane alone walks its buckets. Returns the bucket,
+// and updates above / above_c to the mass / count strictly before it (identical in every lane).
+template <int DIG>
+__device__ __forceinline__ int descend(const Hist<DIG>& h, int m, u64 need_c, u64& above, unsigned int& above_c,
                                        unsigned int& cnt_at) {
+  constexpr int kBuckets = Hist<DIG>::kBuckets, kPerLane = Hist<DIG>::kPerLane;
   const int lane = threadIdx.x & 31;
-  u64 ms[8], lm = 0;
-  unsigned int cs[8], lc = 0;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    ms[j] = hist_mass(h, m * 256 + lane * 8 + j);
-    cs[j] = h.cnt[hist_slot(m * 256 + lane * 8 + j)];
-    lm += ms[j];
-    lc += cs[j];
+  const int first = m * kBuckets + lane * kPerLane;
+  u64 lm = 0;
+  unsigned int lc = 0;
+#pragma unroll 8
+  for (int i = 0; i < kPerLane; ++i) {
+    lm += hist_mass(h, first + i);
+    lc += h.cnt[hist_slot(first + i)];
   }
   u64 sm = lm;
   unsigned int sc = lc;
@@ -82,33 +93,29 @@ __device__ __forceinline__ int descend(const Hist& h, int m, u64 need_c, u64& ab
       sc += tc;
     }
   }
-  // within the lane: the running mass before each of its buckets is monotone, so the first bucket that reaches the
-  // threshold is the number of buckets that do not (no data-dependent branches)
-  const u64 a0 = above + (sm - lm);
-  const unsigned int ac0 = above_c + (sc - lc);
-  u64 run = a0;
-  int below = 0;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    run += ms[j];
-    below += run < need_c ? 1 : 0;
-  }
-  int found = below < 8 ? below : (lane == 31 ? 7 : -1);
-  u64 a = a0;
-  unsigned int ac = ac0, c_at = 0;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const bool before = j < (found < 0 ? 8 : found);
-    a += before ? ms[j] : 0ull;
-    ac += before ? cs[j] : 0u;
-    c_at = j == found ? cs[j] : c_at;
-  }
-  const unsigned int hit = __ballot_sync(kFull, found >= 0);  // lane 31 always hits
+  // the lane whose buckets take the running mass to the threshold (lane 31 if none does)
+  u64 a = above + (sm - lm);
+  unsigned int ac = above_c + (sc - lc), c_at = 0;
+  const unsigned int hit = __ballot_sync(kFull, a + lm >= need_c || lane == 31);
   const int win = __ffs(hit) - 1;
+  int found = kPerLane - 1;
+  if (lane == win) {
+    for (int i = 0; i < kPerLane; ++i) {
+      const u64 mi = hist_mass(h, first + i);
+      const unsigned int ci = h.cnt[hist_slot(first + i)];
+      if (a + mi >= need_c || i == kPerLane - 1) {
+        found = i;
+        c_at = ci;
+        break;
+      }
+      a += mi;
+      ac += ci;
+    }
+  }
   above = __shfl_sync(kFull, a, win);
   above_c = __shfl_sync(kFull, ac, win);
   cnt_at = __shfl_sync(kFull, c_at, win);
-  return win * 8 + __shfl_sync(kFull, found, win);
+  return win * kPerLane + __shfl_sync(kFull, found, win);
 }
 
 // One block per unit. A thread keeps KPT keys in registers (loaded once when the sequence fits one round, else
@@ -118,8 +125,11 @@ __device__ __forceinline__ int descend(const Hist& h, int m, u64 need_c, u64& ab
 // the unit's keys differ (kmax, kmin: largest and smallest key of the unit). Importance values share their sign and
 // most exponent bits, so digits of the raw key would put nearly all keys into a handful of buckets and serialise
 // the shared atomics; the digits of t spread them over the whole histogram. Ascending t is descending importance.
+template <int DIG>
 __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
-  __shared__ Hist hist;
+  constexpr int kDigitBits = DIG, kBuckets = Hist<DIG>::kBuckets, kPerLane = Hist<DIG>::kPerLane;
+  constexpr int kHistWords = Hist<DIG>::kWords;
+  __shared__ Hist<DIG> hist;
   __shared__ uint32_t s_prefix[2];
   __shared__ int s_done[2];
   __shared__ u64 s_W[2];
@@ -204,7 +214,7 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
   // Eq. 9: radix descent, both modalities at once. The first pass sees every key, so its histogram also yields the
   // modality masses W_v, W_t of Eq. 6. `rem` counts the bits of t not yet resolved.
   for (int rem = top, pass = 0; rem > 0; ++pass) {
-    const int bits = min(rem, 8), shift = rem - bits;
+    const int bits = min(rem, kDigitBits), shift = rem - bits;
     const uint32_t dmask = (1u << bits) - 1u;
     for (int x = threadIdx.x; x < kHistWords; x += NT) {
       hist.cnt[x] = 0;
@@ -228,7 +238,7 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
         for (int j = 0; j < KPT; ++j) {
           const bool vis = (flags >> (16 + j)) & 1u;
           if ((key[j] >> rem) == (vis ? want0 : want1))
-            hist_add(hist, (vis ? 0 : 256) + (int)((key[j] >> shift) & dmask), psi_fix(kmax - key[j]));
+            hist_add(hist, (vis ? 0 : kBuckets) + (int)((key[j] >> shift) & dmask), psi_fix(kmax - key[j]));
         }
       }
     }
@@ -237,8 +247,8 @@ __global__ void __launch_bounds__(NT, 2) alloc_unit_kernel(AllocParams p) {
       const int m = warp;
       if (pass == 0) {
         u64 wsum = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) wsum += hist_mass(hist, m * 256 + lane * 8 + j);
+#pragma unroll 8
+        for (int j = 0; j < kPerLane; ++j) wsum += hist_mass(hist, m * kBuckets + lane * kPerLane + j);
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) wsum += __shfl_xor_sync(kFull, wsum, off);
         const u64 W = wsum;
@@ -430,6 +440,12 @@ __global__ void alloc_layer_kernel(AllocParams p, int depth, int layer) {
                  p.hcc_mode == MADAKV_HCC_DEMAND && layer + 1 < depth);
 }
 
+// 8-bit digits while every sequence fits one round of the kernel, 10-bit digits beyond
+void launch_alloc_unit(const madakv_config& c, const AllocParams& p, int units, cudaStream_t st) {
+  if (c.max_seq_len <= ROUND) alloc_unit_kernel<8><<<units, NT, 0, st>>>(p);
+  else alloc_unit_kernel<10><<<units, NT, 0, st>>>(p);
+}
+
 }  // namespace
 
 int launch_allocate(const madakv_config& c, const float* psi, const uint8_t* mask, const int32_t* seq_len,
@@ -455,7 +471,7 @@ int launch_allocate(const madakv_config& c, const float* psi, const uint8_t* mas
   p.window = c.window;
   p.theta_fix = (u64)((double)c.theta * 4294967296.0);
   const int units = c.batch * c.n_layers * c.n_kv_heads;
-  alloc_unit_kernel<<<units, NT, 0, st>>>(p);
+  launch_alloc_unit(c, p, units, st);
   alloc_seq_kernel<<<c.batch, 1024, c.n_layers * (sizeof(double) + sizeof(long long)), st>>>(p);
   return launch_status();
 }
@@ -482,7 +498,7 @@ int launch_allocate_layer(const madakv_config& c, int layer, const float* psi, c
   p.keep_window = c.keep_window;
   p.window = c.window;
   p.theta_fix = (u64)((double)c.theta * 4294967296.0);
-  if (psi) alloc_unit_kernel<<<c.batch * c.n_kv_heads, NT, 0, st>>>(p);  // else: done by launch_demand_layer
+  if (psi) launch_alloc_unit(c, p, c.batch * c.n_kv_heads, st);  // else: done by launch_demand_layer
   alloc_layer_kernel<<<c.batch, 1024, 0, st>>>(p, c.n_layers, layer);
   return launch_status();
 }
@@ -508,7 +524,7 @@ int launch_demand_layer(const madakv_config& c, const float* psi, const uint8_t*
   p.keep_window = c.keep_window;
   p.window = c.window;
   p.theta_fix = (u64)((double)c.theta * 4294967296.0);
-  alloc_unit_kernel<<<c.batch * c.n_kv_heads, NT, 0, st>>>(p);
+  launch_alloc_unit(c, p, c.batch * c.n_kv_heads, st);
   return launch_status();
 }
 

@@ -2,7 +2,7 @@
 //
 //   seg_scan     one block: visual-token count of every sequence, kept_len[u] = b_v + b_t and the exclusive scan
 //                seg_off (rows, with headroom)
-//   select_unit  one block per unit: a 4-pass shared-memory radix select over the order-preserving bit pattern of
+//   select_unit  one block per unit: a three- or four-pass shared-memory radix select over the order-preserving bit pattern of
 //                psi finds, for both modalities at once, the budget-th largest value and how many of its ties are
 //                still needed; an ordered sweep then emits the kept positions in ascending order, giving ties to
 //                the lowest positions (block-wide prefix scans provide the tie ranks and the output slots).
@@ -22,6 +22,10 @@ constexpr int NT = 256;
 constexpr int KPT = 32;                // consecutive positions per thread
 constexpr int CHUNK = NT * KPT;        // 8192 positions per chunk
 constexpr unsigned int kFull = 0xffffffffu;
+// A radix digit has DIG bits: 10 for configs whose sequences are longer than one chunk (they are re-read from L2 in
+// every pass, and the 30 bits in which importance values differ at most then take three passes instead of four),
+// 8 for those that sit in registers (the larger histograms only cost there). Bucket b of a modality sits at word
+// b + b / kPerLane, so that the lanes of the walking warp (lane j owns buckets kPerLane * j ..) read 32 different banks.
 
 struct SelParams {
   const float* psi;
@@ -210,9 +214,11 @@ __device__ __forceinline__ void load_chunk(const float* psi, const uint8_t* mask
 // (kmax, kmin: largest and smallest key of the unit): importance values share their sign and most exponent bits,
 // so digits of the raw key would put nearly all keys into a handful of buckets and serialise the shared atomics.
 // Ascending t is descending importance.
-template <bool kVec, bool kPool>
+template <bool kVec, bool kPool, int DIG>
 __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
-  __shared__ unsigned int cnt[2][256];
+  constexpr int kDigitBits = DIG, kBuckets = 1 << DIG, kPerLane = kBuckets / 32, kCntWords = kBuckets + 32;
+  auto cnt_slot = [](uint32_t digit) { return (int)(digit + digit / kPerLane); };
+  __shared__ unsigned int cnt[2][kCntWords];
   __shared__ uint32_t s_prefix[2];
   __shared__ unsigned int s_above[2];
   __shared__ uint32_t warp_tot[NT / 32];
@@ -271,9 +277,9 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
   // radix select: when all bits of t are resolved, s_prefix[m] is the t of the want[m]-th largest key of modality m
   // (if that many exist) and s_above[m] counts the keys strictly above it. `rem` counts the bits not yet resolved.
   for (int rem = top; rem > 0;) {
-    const int bits = min(rem, 8), shift = rem - bits;
+    const int bits = min(rem, kDigitBits), shift = rem - bits;
     const uint32_t dmask = (1u << bits) - 1u;
-    for (int x = threadIdx.x; x < 512; x += NT) (&cnt[0][0])[x] = 0;
+    for (int x = threadIdx.x; x < 2 * kCntWords; x += NT) (&cnt[0][0])[x] = 0;
     __syncthreads();
     const uint32_t pre0 = s_prefix[0], pre1 = s_prefix[1];
     for (int c = 0; c < chunks; ++c) {
@@ -285,20 +291,19 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
 #pragma unroll
       for (int j = 0; j < KPT; ++j) {  // (a position outside the ranking holds all ones: no prefix equals its shifted t)
         const int m = (vis >> j) & 1u ? 0 : 1;
-        if ((key[j] >> rem) == (m == 0 ? pre0 : pre1)) atomicAdd(&cnt[m][(key[j] >> shift) & dmask], 1u);
+        if ((key[j] >> rem) == (m == 0 ? pre0 : pre1)) atomicAdd(&cnt[m][cnt_slot((key[j] >> shift) & dmask)], 1u);
       }
     }
     __syncthreads();
     if (warp < 2) {
-      // warp m walks modality m's buckets in ascending digit order; lane j owns buckets 8j..8j+7
+      // warp m walks modality m's buckets in ascending digit order: a prefix scan of the lanes' totals tells which
+      // lane holds the bucket that takes the running count to `want` (lane 31 if none does), and that lane alone
+      // walks its buckets
       const int m = warp;
       const unsigned int want = (unsigned int)(m == 0 ? want0 : want1);
-      unsigned int cs[8], lc = 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        cs[j] = cnt[m][lane * 8 + j];
-        lc += cs[j];
-      }
+      unsigned int lc = 0;
+#pragma unroll 8
+      for (int i = 0; i < kPerLane; ++i) lc += cnt[m][cnt_slot(lane * kPerLane + i)];
       unsigned int sc = lc;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
@@ -306,19 +311,20 @@ __global__ void __launch_bounds__(NT) select_unit_kernel(SelParams p) {
         if (lane >= off) sc += t;
       }
       unsigned int above = s_above[m] + (sc - lc);
-      int found = -1;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if (found < 0) {
-          if (above + cs[j] >= want || (lane == 31 && j == 7)) found = j;
-          else above += cs[j];
-        }
-      }
-      const unsigned int hit = __ballot_sync(kFull, found >= 0);  // lane 31 always hits
+      const unsigned int hit = __ballot_sync(kFull, above + lc >= want || lane == 31);
       if (lane == __ffs(hit) - 1) {
+        int found = kPerLane - 1;
+        for (int i = 0; i < kPerLane; ++i) {
+          const unsigned int ci = cnt[m][cnt_slot(lane * kPerLane + i)];
+          if (above + ci >= want || i == kPerLane - 1) {
+            found = i;
+            break;
+          }
+          above += ci;
+        }
         // buckets beyond the pass's digit range are empty; landing there means "fewer keys than wanted"
         s_above[m] = above;
-        s_prefix[m] = (s_prefix[m] << bits) | min((uint32_t)(lane * 8 + found), dmask);
+        s_prefix[m] = (s_prefix[m] << bits) | min((uint32_t)(lane * kPerLane + found), dmask);
       }
     }
     __syncthreads();
@@ -408,9 +414,17 @@ int launch_select(const madakv_config& c, const float* psi, const uint8_t* mask,
   p.pool_r = (c.pool_kernel - 1) / 2;
   seg_scan_kernel<<<1, 1024, 0, st>>>(p);
   // 16-byte loads of psi need every unit's row (n_max floats apart) to start on a 16-byte boundary
-  if (c.pool_kernel > 1 || c.keep_window) select_unit_kernel<false, true><<<p.units, NT, 0, st>>>(p);
-  else if (c.max_seq_len % 4 == 0) select_unit_kernel<true, false><<<p.units, NT, 0, st>>>(p);
-  else select_unit_kernel<false, false><<<p.units, NT, 0, st>>>(p);
+  const bool wide = c.max_seq_len > CHUNK;  // 10-bit digits when sequences can be longer than one chunk
+  if (c.pool_kernel > 1 || c.keep_window) {
+    if (wide) select_unit_kernel<false, true, 10><<<p.units, NT, 0, st>>>(p);
+    else select_unit_kernel<false, true, 8><<<p.units, NT, 0, st>>>(p);
+  } else if (c.max_seq_len % 4 == 0) {
+    if (wide) select_unit_kernel<true, false, 10><<<p.units, NT, 0, st>>>(p);
+    else select_unit_kernel<true, false, 8><<<p.units, NT, 0, st>>>(p);
+  } else {
+    if (wide) select_unit_kernel<false, false, 10><<<p.units, NT, 0, st>>>(p);
+    else select_unit_kernel<false, false, 8><<<p.units, NT, 0, st>>>(p);
+  }
   return launch_status();
 }
 
