@@ -542,6 +542,43 @@ def test_decode_refusals_come_before_the_append():
     assert int(kept_len[0]) == 10 and not k_c.any() and not v_c.any()
 
 
+@pytest.mark.parametrize("name", ["bf16_d128", "bf16_gqa7"])
+def test_decode_steps_replayed_from_a_cuda_graph(name):
+    """Two decode steps with append, captured into a CUDA graph and replayed, give the cache and the outputs of the
+    same two steps launched eagerly (the decode kernels are launched with programmatic stream serialisation outside a
+    capture and in the ordinary way inside one; both orders of execution must be the same)."""
+    wl = SHAPES[name]
+    g = dev(make_case(wl))
+    cfg = config_of(wl)
+    steps = [tuple(t.cuda() for t in synth.make_decode_step(wl, s)) for s in range(2)]
+
+    def prepared():
+        buf = mk.EvictionBuffers(cfg, capacity_of(wl))
+        buf.run_eviction(g["q_win"], g["k"], g["v"], g["mask"], g["seq_len"], g["budget"])
+        return buf
+
+    eager, outs = prepared(), []
+    for q, kn, vn in steps:
+        eager.run_decode(q, kn, vn)
+        outs.append(eager.out.clone())
+    assert mk.madakv_poll_status(eager.ws) == 0
+    graphed = prepared()
+    out2 = [torch.empty_like(graphed.out) for _ in steps]
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for (q, kn, vn), o in zip(steps, out2):
+            mk.madakv_decode_attn(cfg, -1, q, kn, vn, graphed.k_c, graphed.v_c, graphed.seg_off, graphed.kept_len, o, None,
+                                  graphed.ws)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert mk.madakv_poll_status(graphed.ws) == 0
+    assert torch.equal(graphed.kept_len, eager.kept_len)
+    assert torch.equal(graphed.k_c, eager.k_c) and torch.equal(graphed.v_c, eager.v_c)
+    for a, b in zip(outs, out2):
+        assert torch.equal(a, b)
+
+
 def test_decode_with_more_than_65535_segments():
     # 70 000 short segments in one call (a grid dimension of 65 535 must not be the limit); every unit against the oracle
     wl = synth.scaled(TINY, B=70, L=100, Hq=10, Hkv=10, d=64, n=16, w=4, budget=8, max_new_tokens=2)
