@@ -403,20 +403,36 @@ class Bench:
     # ---- the decode run of the workload: max_new_tokens steps, each appending one row per KV head (Eq. 4) and
     # attending over the grown cache (Eq. 5); per-step device times. `layerwise` issues the L dependent per-layer
     # calls a model makes (layer l + 1's query depends on layer l's output) instead of one all-layer call.
-    def time_decode_run(self, b, layerwise=False, max_steps=None):
+    def time_decode_run(self, b, layerwise=False, max_steps=None, graph=False):
+        """Decode steps with append, one event per step. graph: one step (its L per-layer calls) is captured into a
+        CUDA graph once and replayed, as a serving loop would do; the step's inputs are then the same every time."""
         mk, wl = self.mk, self.wl
         n_steps = wl.max_new_tokens if max_steps is None else min(max_steps, wl.max_new_tokens)
         keep = b.kept_len.clone()
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps + 1)]
-        torch.cuda.synchronize()
-        evs[0].record()
-        for s in range(n_steps):
-            q, kn, vn = self.dec[s % self.n_dec]
+
+        def one_step(q, kn, vn):
             if layerwise:
                 for l in range(wl.L):
                     mk.madakv_decode_attn(b.cfg, l, q, kn, vn, b.k_c, b.v_c, b.seg_off, b.kept_len, b.out, None, b.ws)
             else:
                 mk.madakv_decode_attn(b.cfg, -1, q, kn, vn, b.k_c, b.v_c, b.seg_off, b.kept_len, b.out, None, b.ws)
+
+        g = None
+        if graph:
+            one_step(*self.dec[0])  # everything the calls set up on the host has happened before the capture
+            torch.cuda.synchronize()
+            b.kept_len.copy_(keep)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                one_step(*self.dec[0])
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps + 1)]
+        torch.cuda.synchronize()
+        evs[0].record()
+        for s in range(n_steps):
+            if g is not None:
+                g.replay()
+            else:
+                one_step(*self.dec[s % self.n_dec])
             evs[s + 1].record()
         torch.cuda.synchronize()
         grown = int((b.kept_len - keep).min().item()), int((b.kept_len - keep).max().item())
@@ -631,11 +647,15 @@ class Bench:
         dec["run_with_append"] = {"compressed": self.time_decode_run(buf), "full": None}
         dec["us_per_step_layer_sequential"] = {"compressed": self.time_decode_run(buf, layerwise=True, max_steps=16),
                                                "full": None}
+        dec["us_per_step_layer_sequential_cuda_graph"] = {
+            "compressed": self.time_decode_run(buf, layerwise=True, max_steps=16, graph=True), "full": None}
         if not args.no_full_cache:
             full = self.full_cache()
             dec["us_per_step"]["full"] = self.time_decode(full, steps=5)
             dec["run_with_append"]["full"] = self.time_decode_run(full, max_steps=32)
             dec["us_per_step_layer_sequential"]["full"] = self.time_decode_run(full, layerwise=True, max_steps=4)
+            dec["us_per_step_layer_sequential_cuda_graph"]["full"] = self.time_decode_run(full, layerwise=True, max_steps=4,
+                                                                                         graph=True)
             full_bytes = 2 * int(full.kept_len.sum().item()) * wl.d * e
             dec["full_cache_gbs"] = full_bytes / (dec["us_per_step"]["full"] * 1e-6) / 1e9
             dec["speedup_compressed_vs_full"] = dec["us_per_step"]["full"] / us

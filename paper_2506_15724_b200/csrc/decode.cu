@@ -550,6 +550,16 @@ __global__ void __launch_bounds__(D) decode_merge_kernel(DecodeParams p) {
   if (p.lse_out && c == 0) p.lse_out[row] = Lsum > 0.f ? (M + log2f(Lsum)) * kLn2 : -INFINITY;
 }
 
+// Smallest share of a segment that a block takes. 512 rows when there are segments enough to fill the GPU (shorter
+// shares leave a block's load pipeline no time to fill and cost more merge work: measured 5-8 % at 256 rows); a call
+// with few segments (one layer of a long-context model: 8 segments) is bound by the latency of its longest block,
+// and there shorter shares spread a segment over more blocks: 128 rows for the scalar kernel (one layer of the llava
+// workload: 747 -> 488 us for the 32 layers of a step), 256 for the tensor-core kernel, whose four warps take 64
+// rows per iteration (at 128 rows it lost more in merge work than it gained: long 429 -> 471 us, at 256: 426).
+int min_share_rows(int n_sel, bool tensor_core_kernel) {
+  return n_sel >= 64 ? kDecodeMinRows : (tensor_core_kernel ? 256 : 128);
+}
+
 // Block order of the grid. With many segments a segment's blocks follow one another (neighbouring blocks stream
 // neighbouring rows); with fewer segments than SMs the grid is a wave or two, and then the blocks are ordered by slot so
 // that every segment's last and shortest block is scheduled last.
@@ -613,7 +623,7 @@ int launch_decode(const madakv_config& c, int layer, const void* q, const void* 
   p.layer = layer;
   p.slots = wl.decode_splits < kDecodeSlots ? wl.decode_splits : kDecodeSlots;
   p.n_sel = (layer < 0 ? c.batch * c.n_layers : c.batch) * c.n_kv_heads;
-  p.min_rows = kDecodeMinRows;
+  p.min_rows = min_share_rows(p.n_sel, c.dtype == MADAKV_BF16 && p.g >= 3 && p.g <= 16);
   p.slot_fast = slot_order(p.n_sel);
   p.scale2 = scale_of(c) * kLog2e;
   if (c.dtype == MADAKV_F32) return c.head_dim == 64 ? run<float, 64>(p, c, st) : run<float, 128>(p, c, st);
@@ -698,7 +708,7 @@ extern "C" int madakv_decode_attn_static(const madakv_config* cfg, int32_t layer
   p.layer = layer;
   p.slots = splits < kDecodeSlots ? splits : kDecodeSlots;  // what the kernels use of the (larger) documented bound
   p.n_sel = (layer < 0 ? c.batch * c.n_layers : c.batch) * c.n_kv_heads;
-  p.min_rows = kDecodeMinRows;
+  p.min_rows = min_share_rows(p.n_sel, c.dtype == MADAKV_BF16 && p.g >= 3 && p.g <= 16);
   p.slot_fast = slot_order(p.n_sel);
   p.scale2 = scale_of(c) * kLog2e;
   cudaStream_t st = (cudaStream_t)stream;
