@@ -2,7 +2,7 @@
 //
 //   append   (Eq. 4) has no kernel of its own: the partial block whose share holds the new row copies it from
 //            k_new / v_new behind the segment and attends over it; the merge kernel bumps kept_len
-//   partial  up to kDecodeSlots blocks per segment, each taking an equal share of the segment's rows (the share is a
+//   partial  up to 8, 16 or 32 blocks per segment (blocks_per_segment), each taking an equal share of the segment's rows (the share is a
 //            function of the segment's length alone: short segments use fewer blocks, never fewer than kDecodeMinRows
 //            rows each): a group of LPR lanes owns a cache row (16 bytes per lane), the g query heads of the KV group
 //            share every K/V row read; online softmax in the log2 domain, fp32 accumulation; the block's row groups
@@ -560,6 +560,15 @@ int min_share_rows(int n_sel, bool tensor_core_kernel) {
   return n_sel >= 64 ? kDecodeMinRows : (tensor_core_kernel ? 256 : 128);
 }
 
+// Blocks launched per segment (the grid is segments x this number, and a block whose share of its segment is empty
+// returns at once). With segments enough to fill the GPU 8 is plenty, and the thousands of blocks that 32 per segment
+// launched only to return cost a tenth of the call (batched 246 -> 219 us, qwen 26.6 -> 23.8); a long segment then
+// simply gets longer shares. A call with few segments keeps 32 (scalar kernel) or 16 (tensor-core kernel).
+int blocks_per_segment(int n_sel, bool tensor_core_kernel, int splits) {
+  const int want = n_sel >= 64 ? 8 : (tensor_core_kernel ? 16 : kDecodeSlots);
+  return splits < want ? splits : want;
+}
+
 // Block order of the grid. With many segments a segment's blocks follow one another (neighbouring blocks stream
 // neighbouring rows); with fewer segments than SMs the grid is a wave or two, and then the blocks are ordered by slot so
 // that every segment's last and shortest block is scheduled last.
@@ -621,9 +630,10 @@ int launch_decode(const madakv_config& c, int layer, const void* q, const void* 
   p.Hkv = c.n_kv_heads;
   p.g = c.n_q_heads / c.n_kv_heads;
   p.layer = layer;
-  p.slots = wl.decode_splits < kDecodeSlots ? wl.decode_splits : kDecodeSlots;
   p.n_sel = (layer < 0 ? c.batch * c.n_layers : c.batch) * c.n_kv_heads;
-  p.min_rows = min_share_rows(p.n_sel, c.dtype == MADAKV_BF16 && p.g >= 3 && p.g <= 16);
+  const bool tc = c.dtype == MADAKV_BF16 && p.g >= 3 && p.g <= 16;
+  p.slots = blocks_per_segment(p.n_sel, tc, wl.decode_splits);
+  p.min_rows = min_share_rows(p.n_sel, tc);
   p.slot_fast = slot_order(p.n_sel);
   p.scale2 = scale_of(c) * kLog2e;
   if (c.dtype == MADAKV_F32) return c.head_dim == 64 ? run<float, 64>(p, c, st) : run<float, 128>(p, c, st);
@@ -706,9 +716,10 @@ extern "C" int madakv_decode_attn_static(const madakv_config* cfg, int32_t layer
   p.Hkv = c.n_kv_heads;
   p.g = c.n_q_heads / c.n_kv_heads;
   p.layer = layer;
-  p.slots = splits < kDecodeSlots ? splits : kDecodeSlots;  // what the kernels use of the (larger) documented bound
   p.n_sel = (layer < 0 ? c.batch * c.n_layers : c.batch) * c.n_kv_heads;
-  p.min_rows = min_share_rows(p.n_sel, c.dtype == MADAKV_BF16 && p.g >= 3 && p.g <= 16);
+  const bool tc = c.dtype == MADAKV_BF16 && p.g >= 3 && p.g <= 16;
+  p.slots = blocks_per_segment(p.n_sel, tc, splits);  // what the kernels use of the (larger) documented bound
+  p.min_rows = min_share_rows(p.n_sel, tc);
   p.slot_fast = slot_order(p.n_sel);
   p.scale2 = scale_of(c) * kLog2e;
   cudaStream_t st = (cudaStream_t)stream;
