@@ -9,6 +9,7 @@ namespace {
 
 constexpr int NT = 256;
 constexpr int ROWS_PER_BLOCK = 128;
+constexpr int kMaxBlocksX = 64;  // blocks per unit at most
 
 struct CompactParams {
   const char* k;
@@ -28,8 +29,7 @@ template <int LPR>  // 16-byte lanes per row
 __global__ void __launch_bounds__(NT) compact_kernel(CompactParams p) {
   const int u = blockIdx.y;
   const int len = p.kept_len[u];
-  const int row0 = blockIdx.x * ROWS_PER_BLOCK;
-  if (row0 >= len) return;
+  if ((int)blockIdx.x * ROWS_PER_BLOCK >= len) return;
   const int64_t off = p.seg_off[u];
   // a segment that selection refused (MADAKV_ECAPACITY: it would end beyond the cache) has no index list: skip it
   if (off + len + p.headroom > p.capacity) return;
@@ -37,6 +37,10 @@ __global__ void __launch_bounds__(NT) compact_kernel(CompactParams p) {
   const int64_t src_base = b * p.stride_b + l * p.stride_l + h * p.stride_h;
   const int lane = threadIdx.x % LPR, sub = threadIdx.x / LPR;
   constexpr int RPI = NT / LPR;  // rows per block iteration
+  // a block takes every gridDim.x-th stretch of ROWS_PER_BLOCK rows (the grid has at most kMaxBlocksX blocks per
+  // unit: with one block per stretch of the longest possible segment nearly all blocks of a long-context call were
+  // launched only to return)
+  for (int row0 = blockIdx.x * ROWS_PER_BLOCK; row0 < len; row0 += gridDim.x * ROWS_PER_BLOCK) {
   const int row_end = min(len, row0 + ROWS_PER_BLOCK);
 #pragma unroll 2
   for (int r = row0 + sub; r < row_end; r += RPI) {
@@ -48,6 +52,7 @@ __global__ void __launch_bounds__(NT) compact_kernel(CompactParams p) {
     const uint4 vv = __ldg(reinterpret_cast<const uint4*>(p.v + src));
     *reinterpret_cast<uint4*>(p.k_c + dst) = kv;
     *reinterpret_cast<uint4*>(p.v_c + dst) = vv;
+  }
   }
 }
 
@@ -79,7 +84,8 @@ int launch_compact(const madakv_config& c, const void* k, const void* v, madakv_
   p.headroom = c.max_new_tokens;
   const int units = c.batch * c.n_layers * c.n_kv_heads;
   if (units > 65535) return MADAKV_EUNSUPPORTED;
-  const dim3 grid((c.max_seq_len + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK, units);
+  const int stretches = (c.max_seq_len + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK;
+  const dim3 grid(stretches < kMaxBlocksX ? stretches : kMaxBlocksX, units);
   switch (p.row_bytes / 16) {
     case 8: compact_kernel<8><<<grid, NT, 0, st>>>(p); break;
     case 16: compact_kernel<16><<<grid, NT, 0, st>>>(p); break;
